@@ -1,0 +1,153 @@
+"""Float64 CPU oracle for the Pulsar Attention context-encoding path.
+
+TEST INFRASTRUCTURE ONLY: the checker that the CUDA library is compared with.
+Nothing in the product path may import this package; it imports nothing from
+the product either.  The arithmetic lives in ``pulsar_oracle.c`` (plain C,
+float64, OpenMP over independent query rows); this module compiles it with gcc
+on first use and marshals numpy arrays through ctypes.
+
+Each wrapper names the passage of the paper its C function follows:
+
+* :func:`maxidf_select` -- Section 3.1 Eq. 2-3, Algorithm 1 line 6, Eq. 4
+* :func:`phase1_attn`   -- Eq. 1 over the assembled input of Eq. 4
+* :func:`phase2_attn`   -- Section 3.2 / Appendix H (single global softmax)
+* :func:`lse_merge`     -- Appendix H Eq. 12-13, iterated
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "pulsar_oracle.c")
+_LIB = os.path.join(_HERE, "liboracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle into ``oracle/liboracle.so`` (gcc, -O2, OpenMP)."""
+    with _lock:
+        stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+        if force or stale:
+            tmp = _LIB + f".tmp{os.getpid()}"
+            subprocess.check_call(
+                ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", tmp, _SRC, "-lm"])
+            os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        i32, i64, f64, vp = ctypes.c_int32, ctypes.c_int64, ctypes.c_double, ctypes.c_void_p
+        lib.oracle_maxidf_select.argtypes = [vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
+        lib.oracle_maxidf_select.restype = ctypes.c_int
+        lib.oracle_phase1_attn.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, vp, vp, i32, f64,
+                                           vp, i64, vp, vp]
+        lib.oracle_phase1_attn.restype = ctypes.c_int
+        lib.oracle_phase2_attn.argtypes = [vp, i32, vp, vp, i32, i32, i32, i32, i32, f64,
+                                           vp, vp, vp, vp]
+        lib.oracle_phase2_attn.restype = ctypes.c_int
+        lib.oracle_lse_merge.argtypes = [vp, vp, i32, i64, i32, vp, vp]
+        lib.oracle_lse_merge.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _bits(x) -> np.ndarray:
+    """bf16 payload as a C-contiguous uint16 array (torch.bfloat16 or uint16 ndarray)."""
+    if isinstance(x, np.ndarray):
+        assert x.dtype == np.uint16
+        return np.ascontiguousarray(x)
+    import torch  # only to reinterpret a CPU bf16 tensor's bits
+    assert x.dtype == torch.bfloat16 and x.device.type == "cpu"
+    return np.ascontiguousarray(x.contiguous().view(torch.int16).numpy().view(np.uint16))
+
+
+def num_threads() -> int:
+    """Threads the OpenMP regions use (OMP_NUM_THREADS if set, else all cores)."""
+    env = os.environ.get("OMP_NUM_THREADS")
+    return int(env) if env else (os.cpu_count() or 1)
+
+
+def maxidf_select(token_ids, vocab_size, block_size, chunk, k, sink):
+    """Max-IDF summary selection.  Returns a dict with ``sel_chunks`` [B,k],
+    ``prefix_idx`` [sink+(B-1)*k*chunk], ``prefix_len`` [B], ``df`` [V] (uint32),
+    ``idf`` [V] and ``score`` [B, block_size/chunk] (float64)."""
+    ids = np.ascontiguousarray(np.asarray(token_ids, dtype=np.uint32))
+    L = ids.shape[0]
+    B, C = L // block_size, block_size // chunk
+    sel = np.zeros((B, k), np.int32)
+    pidx = np.zeros(sink + max(B - 1, 0) * k * chunk, np.int32)
+    plen = np.zeros(B, np.int32)
+    df = np.zeros(vocab_size, np.uint32)
+    idf = np.zeros(vocab_size, np.float64)
+    score = np.zeros((B, C), np.float64)
+    rc = _load().oracle_maxidf_select(_ptr(ids), L, vocab_size, block_size, chunk, k, sink,
+                                      _ptr(sel), _ptr(pidx), _ptr(plen), _ptr(df), _ptr(idf),
+                                      _ptr(score))
+    if rc != 0:
+        raise ValueError(f"oracle_maxidf_select rejected the shape (rc={rc})")
+    return dict(sel_chunks=sel, prefix_idx=pidx, prefix_len=plen, df=df, idf=idf, score=score)
+
+
+def phase1_attn(Q, K, V, block_size, prefix_idx, prefix_len, scale=0.0, rows=None):
+    """Phase-1 prefix-block attention for the query positions ``rows`` (all if
+    None).  Q [L,Hq,d], K,V [L,Hkv,d] bf16.  Returns (O [n,Hq,d], LSE [n,Hq]) float64."""
+    q, kk, v = _bits(Q), _bits(K), _bits(V)
+    L, Hq, d = q.shape
+    Hkv = kk.shape[1]
+    pidx = np.ascontiguousarray(np.asarray(prefix_idx, dtype=np.int32))
+    plen = np.ascontiguousarray(np.asarray(prefix_len, dtype=np.int32))
+    r = None if rows is None else np.ascontiguousarray(np.asarray(rows, dtype=np.int64))
+    n = L if r is None else r.shape[0]
+    O = np.zeros((n, Hq, d), np.float64)
+    LSE = np.zeros((n, Hq), np.float64)
+    rc = _load().oracle_phase1_attn(_ptr(q), _ptr(kk), _ptr(v), L, Hq, Hkv, d, block_size,
+                                    _ptr(pidx), _ptr(plen), pidx.shape[0], float(scale),
+                                    _ptr(r), n, _ptr(O), _ptr(LSE))
+    if rc != 0:
+        raise ValueError(f"oracle_phase1_attn rejected its arguments (rc={rc})")
+    return O, LSE
+
+
+def phase2_attn(Qq, K, V, n_blocks, block_size, scale=0.0, partials=False):
+    """Phase-2 query attention over all retained KV.  Qq [nq,Hq,d], K,V
+    [n_blocks*block_size,Hkv,d] bf16.  Returns (O, LSE) or, with ``partials``,
+    (O, LSE, part_O [B,nq,Hq,d], part_LSE [B,nq,Hq]); all float64."""
+    q, kk, v = _bits(Qq), _bits(K), _bits(V)
+    nq, Hq, d = q.shape
+    Hkv = kk.shape[1]
+    assert kk.shape[0] == n_blocks * block_size
+    O = np.zeros((nq, Hq, d), np.float64)
+    LSE = np.zeros((nq, Hq), np.float64)
+    pO = np.zeros((n_blocks, nq, Hq, d), np.float64) if partials else None
+    pL = np.zeros((n_blocks, nq, Hq), np.float64) if partials else None
+    rc = _load().oracle_phase2_attn(_ptr(q), nq, _ptr(kk), _ptr(v), n_blocks, block_size,
+                                    Hq, Hkv, d, float(scale), _ptr(O), _ptr(LSE), _ptr(pO), _ptr(pL))
+    if rc != 0:
+        raise ValueError(f"oracle_phase2_attn rejected its arguments (rc={rc})")
+    return (O, LSE, pO, pL) if partials else (O, LSE)
+
+
+def lse_merge(part_O, part_LSE):
+    """Iterated online-softmax merge.  part_O [J,rows,d], part_LSE [J,rows] float64."""
+    pO = np.ascontiguousarray(np.asarray(part_O, dtype=np.float64))
+    pL = np.ascontiguousarray(np.asarray(part_LSE, dtype=np.float64))
+    J, rows, d = pO.shape
+    O = np.zeros((rows, d), np.float64)
+    LSE = np.zeros(rows, np.float64)
+    rc = _load().oracle_lse_merge(_ptr(pO), _ptr(pL), J, rows, d, _ptr(O), _ptr(LSE))
+    if rc != 0:
+        raise ValueError(f"oracle_lse_merge rejected its arguments (rc={rc})")
+    return O, LSE

@@ -1,0 +1,302 @@
+/*
+ * Pulsar Attention context-encoding oracle: plain, slow, float64 CPU code.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the checker the CUDA library is
+ * compared against; it shares no code, header, table or helper with the CUDA
+ * path and the product never calls it.  Each function writes out the paper's
+ * definition of the operation directly:
+ *
+ *   oracle_maxidf_select   Section 3.1 Eq. 2-3, Algorithm 1 lines 3 and 6,
+ *                          Appendix C.1 (Eq. 5) and C.5 (Eq. 9), Eq. 4 / Eq. 14
+ *   oracle_phase1_attn     Eq. 1 applied to the assembled input of Eq. 4
+ *                          (Algorithm 1 lines 7-8), block rows only
+ *   oracle_phase2_attn     Section 3.2 / Appendix H: one softmax over the
+ *                          concatenated retained KV, plus per-block partials
+ *   oracle_lse_merge       Appendix H Eq. 12-13, applied iteratively
+ *
+ * Readings taken where the paper is silent: natural logarithm; N = number of
+ * logical blocks; equal chunk scores are ranked by the lower chunk index;
+ * duplicates between the sink and the first summary are kept (each occurrence
+ * counts once); query head h reads KV head h / (Hq/Hkv); softmax scale
+ * 1/sqrt(d) unless the caller gives one; LSE is the natural log of the sum of
+ * exponentials of the scaled logits.
+ *
+ * Parity pins (tests, CPU only): brute-force selection on tiny inputs, needle
+ * property, Table 6 lengths, dense attention with a materialised multiplicity
+ * mask, library causal attention for block 0, single softmax over all keys for
+ * Phase 2.  Parity unpinned (no statement in the paper): the tie-break rule
+ * and the keeping of duplicates; both are the readings above.
+ *
+ * bf16 inputs arrive as raw 16-bit patterns and are widened exactly.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+static double bf16_to_double(uint16_t h) {
+    uint32_t u = ((uint32_t)h) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Selection                                                                 */
+/* ------------------------------------------------------------------------ */
+
+/*
+ * df(t)  = number of blocks that contain token t          (Section 3.1)
+ * IDF(t) = ln(N / max(df(t), 1)),  N = number of blocks    (Eq. 3 / Eq. 5)
+ * score(chunk) = max over its tokens of IDF                (Eq. 2 / Eq. 9)
+ * Sigma_b = the k best chunks of block b, in positional order (Alg. 1 l.6)
+ * prefix  = [sink | Sigma_0 | ... | Sigma_{B-2}], block i uses its first
+ *           prefix_len[i] = sink + i*k*chunk entries (0 for i = 0) (Eq. 4, 14)
+ *
+ * Outputs (any may be NULL): sel_chunks [B*k], prefix_idx [sink+(B-1)*k*chunk],
+ * prefix_len [B], df_out [vocab], idf_out [vocab], score_out [B*C].
+ * Returns 0, or -1 on a shape that the definition does not cover.
+ */
+int oracle_maxidf_select(const uint32_t *token_ids, int64_t L, int32_t vocab_size,
+                         int32_t block_size, int32_t chunk, int32_t k, int32_t sink,
+                         int32_t *sel_chunks, int32_t *prefix_idx, int32_t *prefix_len,
+                         uint32_t *df_out, double *idf_out, double *score_out) {
+    if (L <= 0 || block_size <= 0 || chunk <= 0 || vocab_size <= 0) return -1;
+    if (L % block_size != 0 || block_size % chunk != 0) return -1;
+    const int64_t B = L / block_size;
+    const int64_t C = block_size / chunk;
+    if (k < 0 || k > C || sink < 0 || sink > block_size) return -1;
+    for (int64_t p = 0; p < L; ++p)
+        if (token_ids[p] >= (uint32_t)vocab_size) return -1;
+
+    uint32_t *df = (uint32_t *)calloc((size_t)vocab_size, sizeof(uint32_t));
+    int64_t *last_block = (int64_t *)malloc((size_t)vocab_size * sizeof(int64_t));
+    double *idf = (double *)malloc((size_t)vocab_size * sizeof(double));
+    double *score = (double *)malloc((size_t)C * sizeof(double));
+    char *taken = (char *)malloc((size_t)C);
+    if (!df || !last_block || !idf || !score || !taken) return -2;
+
+    /* document frequency: a block counts once however often the token occurs */
+    for (int64_t t = 0; t < vocab_size; ++t) last_block[t] = -1;
+    for (int64_t b = 0; b < B; ++b)
+        for (int64_t p = b * block_size; p < (b + 1) * block_size; ++p) {
+            uint32_t t = token_ids[p];
+            if (last_block[t] != b) { last_block[t] = b; df[t] += 1; }
+        }
+    for (int64_t t = 0; t < vocab_size; ++t) {
+        uint32_t f = df[t] > 1 ? df[t] : 1;
+        idf[t] = log((double)B / (double)f);
+    }
+
+    if (prefix_idx) for (int32_t j = 0; j < sink; ++j) prefix_idx[j] = j;
+
+    for (int64_t b = 0; b < B; ++b) {
+        for (int64_t c = 0; c < C; ++c) {
+            double s = -INFINITY;
+            for (int64_t p = 0; p < chunk; ++p) {
+                double v = idf[token_ids[b * block_size + c * chunk + p]];
+                if (v > s) s = v;
+            }
+            score[c] = s;
+            if (score_out) score_out[b * C + c] = s;
+        }
+        /* top-k: take the best remaining chunk k times; a strict comparison
+           scanning upward leaves equal scores to the lower index */
+        memset(taken, 0, (size_t)C);
+        for (int32_t j = 0; j < k; ++j) {
+            int64_t best = -1;
+            for (int64_t c = 0; c < C; ++c)
+                if (!taken[c] && (best < 0 || score[c] > score[best])) best = c;
+            if (best >= 0) taken[best] = 1;
+        }
+        /* positional order */
+        int32_t j = 0;
+        for (int64_t c = 0; c < C; ++c) {
+            if (!taken[c]) continue;
+            if (sel_chunks) sel_chunks[b * k + j] = (int32_t)c;
+            if (prefix_idx && b < B - 1)
+                for (int64_t p = 0; p < chunk; ++p)
+                    prefix_idx[sink + (b * k + j) * chunk + p] =
+                        (int32_t)(b * block_size + c * chunk + p);
+            ++j;
+        }
+        if (prefix_len) prefix_len[b] = b == 0 ? 0 : (int32_t)(sink + b * k * chunk);
+    }
+
+    if (df_out) memcpy(df_out, df, (size_t)vocab_size * sizeof(uint32_t));
+    if (idf_out) memcpy(idf_out, idf, (size_t)vocab_size * sizeof(double));
+    free(df); free(last_block); free(idf); free(score); free(taken);
+    return 0;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Attention over an explicit key list                                       */
+/* ------------------------------------------------------------------------ */
+
+/* softmax(q.k_j * scale) V over keys key[0..n) of KV head kv; out[d], *lse.
+   z is caller scratch of n doubles. */
+static void attend_list(const double *q, const float *Kf, const float *Vf,
+                        const int64_t *key, int64_t n, int32_t Hkv, int32_t kv,
+                        int32_t d, double scale, double *z, double *out, double *lse) {
+    double zmax = -INFINITY;
+    for (int64_t j = 0; j < n; ++j) {
+        const float *kr = Kf + ((size_t)key[j] * Hkv + kv) * d;
+        double acc = 0.0;
+        for (int32_t e = 0; e < d; ++e) acc += q[e] * (double)kr[e];
+        z[j] = acc * scale;
+        if (z[j] > zmax) zmax = z[j];
+    }
+    double denom = 0.0;
+    for (int32_t e = 0; e < d; ++e) out[e] = 0.0;
+    for (int64_t j = 0; j < n; ++j) {
+        double w = exp(z[j] - zmax);
+        denom += w;
+        const float *vr = Vf + ((size_t)key[j] * Hkv + kv) * d;
+        for (int32_t e = 0; e < d; ++e) out[e] += w * (double)vr[e];
+    }
+    for (int32_t e = 0; e < d; ++e) out[e] /= denom;
+    *lse = zmax + log(denom);
+}
+
+static float *widen(const uint16_t *x, size_t n) {
+    float *f = (float *)malloc(n * sizeof(float));
+    if (!f) return NULL;
+    for (size_t i = 0; i < n; ++i) f[i] = (float)bf16_to_double(x[i]);
+    return f;
+}
+
+/*
+ * Phase 1 (Eq. 1 over Input_i of Eq. 4).  Query row at global position
+ * p = i*block_size + r, head h, sees the keys prefix_idx[0 .. prefix_len[i])
+ * followed by the block's own rows i*block_size .. p (causal).  A key that is
+ * listed twice is attended twice.
+ *
+ * Q [L,Hq,d], K,V [L,Hkv,d] bf16 bit patterns.  rows: n_rows global query
+ * positions to compute (NULL = all L, in order).  O [n_rows,Hq,d] and
+ * LSE [n_rows,Hq] in float64.  scale <= 0 selects 1/sqrt(d).
+ */
+int oracle_phase1_attn(const uint16_t *Q, const uint16_t *K, const uint16_t *V,
+                       int64_t L, int32_t Hq, int32_t Hkv, int32_t d, int32_t block_size,
+                       const int32_t *prefix_idx, const int32_t *prefix_len,
+                       int32_t prefix_total, double scale,
+                       const int64_t *rows, int64_t n_rows, double *O, double *LSE) {
+    if (L <= 0 || block_size <= 0 || L % block_size || Hkv <= 0 || Hq % Hkv || d <= 0) return -1;
+    const int64_t B = L / block_size;
+    for (int64_t i = 0; i < B; ++i) {
+        if (prefix_len[i] < 0 || prefix_len[i] > prefix_total) return -1;
+        for (int32_t j = 0; j < prefix_len[i]; ++j)
+            if (prefix_idx[j] < 0 || prefix_idx[j] >= i * block_size) return -1;
+    }
+    if (!rows) n_rows = L;
+    if (scale <= 0.0) scale = 1.0 / sqrt((double)d);
+    const int32_t g = Hq / Hkv;
+    float *Kf = widen(K, (size_t)L * Hkv * d);
+    float *Vf = widen(V, (size_t)L * Hkv * d);
+    if (!Kf || !Vf) return -2;
+    int err = 0;
+
+#pragma omp parallel
+    {
+        int64_t *key = (int64_t *)malloc((size_t)(prefix_total + block_size) * sizeof(int64_t));
+        double *z = (double *)malloc((size_t)(prefix_total + block_size) * sizeof(double));
+        double *q = (double *)malloc((size_t)d * sizeof(double));
+        if (!key || !z || !q) {
+#pragma omp atomic write
+            err = -2;
+        } else {
+#pragma omp for schedule(dynamic, 1)
+            for (int64_t s = 0; s < n_rows; ++s) {
+                const int64_t p = rows ? rows[s] : s;
+                const int64_t i = p / block_size;
+                int64_t n = 0;
+                for (int32_t j = 0; j < prefix_len[i]; ++j) key[n++] = prefix_idx[j];
+                for (int64_t j = i * block_size; j <= p; ++j) key[n++] = j;
+                for (int32_t h = 0; h < Hq; ++h) {
+                    for (int32_t e = 0; e < d; ++e)
+                        q[e] = bf16_to_double(Q[((size_t)p * Hq + h) * d + e]);
+                    attend_list(q, Kf, Vf, key, n, Hkv, h / g, d, scale, z,
+                                O + ((size_t)s * Hq + h) * d, LSE + (size_t)s * Hq + h);
+                }
+            }
+        }
+        free(key); free(z); free(q);
+    }
+    free(Kf); free(Vf);
+    return err;
+}
+
+/*
+ * Phase 2.  Every query row attends to all L = B*block_size retained keys of
+ * its KV head with one softmax (the result the LSE merge must reproduce), and,
+ * if part_O/part_LSE are given, to each block's block_size keys separately
+ * (A_h, l_h of Algorithm 1 line 12).
+ *
+ * Qq [nq,Hq,d], K,V [B*block_size,Hkv,d] bf16 bit patterns.
+ * O [nq,Hq,d], LSE [nq,Hq]; part_O [B,nq,Hq,d], part_LSE [B,nq,Hq] or NULL.
+ */
+int oracle_phase2_attn(const uint16_t *Qq, int32_t nq, const uint16_t *K, const uint16_t *V,
+                       int32_t B, int32_t block_size, int32_t Hq, int32_t Hkv, int32_t d,
+                       double scale, double *O, double *LSE, double *part_O, double *part_LSE) {
+    if (nq <= 0 || B <= 0 || block_size <= 0 || Hkv <= 0 || Hq % Hkv || d <= 0) return -1;
+    const int64_t L = (int64_t)B * block_size;
+    if (scale <= 0.0) scale = 1.0 / sqrt((double)d);
+    const int32_t g = Hq / Hkv;
+    float *Kf = widen(K, (size_t)L * Hkv * d);
+    float *Vf = widen(V, (size_t)L * Hkv * d);
+    if (!Kf || !Vf) return -2;
+    int err = 0;
+
+#pragma omp parallel
+    {
+        int64_t *key = (int64_t *)malloc((size_t)L * sizeof(int64_t));
+        double *z = (double *)malloc((size_t)L * sizeof(double));
+        double *q = (double *)malloc((size_t)d * sizeof(double));
+        if (!key || !z || !q) {
+#pragma omp atomic write
+            err = -2;
+        } else {
+            for (int64_t j = 0; j < L; ++j) key[j] = j;
+#pragma omp for schedule(dynamic, 1) collapse(2)
+            for (int32_t r = 0; r < nq; ++r)
+                for (int32_t h = 0; h < Hq; ++h) {
+                    for (int32_t e = 0; e < d; ++e)
+                        q[e] = bf16_to_double(Qq[((size_t)r * Hq + h) * d + e]);
+                    attend_list(q, Kf, Vf, key, L, Hkv, h / g, d, scale, z,
+                                O + ((size_t)r * Hq + h) * d, LSE + (size_t)r * Hq + h);
+                    if (part_O && part_LSE)
+                        for (int32_t b = 0; b < B; ++b)
+                            attend_list(q, Kf, Vf, key + (int64_t)b * block_size, block_size,
+                                        Hkv, h / g, d, scale, z,
+                                        part_O + (((size_t)b * nq + r) * Hq + h) * d,
+                                        part_LSE + ((size_t)b * nq + r) * Hq + h);
+                }
+        }
+        free(key); free(z); free(q);
+    }
+    free(Kf); free(Vf);
+    return err;
+}
+
+/*
+ * Online-softmax merge, Appendix H Eq. 12-13, folded over the parts in order:
+ *   l' = l + ln(1 + e^{l_h - l}),  o' = e^{l - l'} o + e^{l_h - l'} o_h.
+ * part_O [n_parts,rows,d], part_LSE [n_parts,rows] -> O [rows,d], LSE [rows].
+ */
+int oracle_lse_merge(const double *part_O, const double *part_LSE, int32_t n_parts,
+                     int64_t rows, int32_t d, double *O, double *LSE) {
+    if (n_parts <= 0 || rows < 0 || d <= 0) return -1;
+    for (int64_t r = 0; r < rows; ++r) {
+        double l = part_LSE[r];
+        for (int32_t e = 0; e < d; ++e) O[r * d + e] = part_O[r * d + e];
+        for (int32_t h = 1; h < n_parts; ++h) {
+            double lh = part_LSE[(size_t)h * rows + r];
+            double ln = l + log(1.0 + exp(lh - l));
+            double a = exp(l - ln), bw = exp(lh - ln);
+            const double *oh = part_O + ((size_t)h * rows + r) * d;
+            for (int32_t e = 0; e < d; ++e) O[r * d + e] = a * O[r * d + e] + bw * oh[e];
+            l = ln;
+        }
+        LSE[r] = l;
+    }
+    return 0;
+}
