@@ -1,0 +1,186 @@
+/*
+ * pulsar.h -- C ABI of the B200 (sm_100a) Pulsar Attention context-encoding library.
+ *
+ * Three operations of the method, one call each, plus the merge on its own:
+ *
+ *   pulsar_maxidf_select   Max-IDF summary selection      (Section 3.1, Eq. 2-4; Alg. 1 l.3, l.6)
+ *   pulsar_phase1_attn     Phase-1 prefix-block attention (Eq. 1 over Input_i of Eq. 4; Alg. 1 l.7-8)
+ *   pulsar_phase2_attn     Phase-2 query attention + merge (Section 3.2; Alg. 1 l.12-13; App. H)
+ *   pulsar_lse_merge       online-softmax merge alone      (Appendix H, Eq. 12-13)
+ *
+ * Conventions that hold for every call
+ * ------------------------------------
+ *  - All data pointers are DEVICE pointers unless the comment says "host".  Tensors are
+ *    contiguous in the stated layout, 16-byte aligned.  "bf16" is the raw 16-bit bfloat16
+ *    pattern (uint16_t here).
+ *  - The caller owns all memory.  The library allocates and frees no device memory and keeps
+ *    no pointer after the work enqueued on `stream` has finished.  Scratch comes from the
+ *    `workspace` argument, whose minimum size the matching *_workspace_bytes function returns
+ *    (256-byte aligned base required).  The workspace may be reused by the next call on the
+ *    same stream.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls
+ *    only enqueue work and never synchronise the host; inputs and outputs must stay alive
+ *    until the stream reaches the end of the call.
+ *  - The return value is a pulsar_status_t.  Arguments are validated on the host before
+ *    anything is launched: a call that returns non-zero has launched nothing.
+ *  - Errors that depend on device data (a token id >= vocab_size, a prefix index that is not
+ *    before its block, a device-side wait that ran out) are OR-ed into `*device_status`
+ *    (device int32, may be NULL; the caller zeroes it and reads it after synchronising).
+ *    The kernels never trap: offending elements are skipped or clamped, every wait is bounded.
+ *  - Only compute capability 10.0 devices are accepted (PULSAR_ERR_UNSUPPORTED_DEVICE otherwise).
+ *    There is no CPU path.
+ */
+#ifndef PULSAR_H_
+#define PULSAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum pulsar_status {
+    PULSAR_OK = 0,
+    PULSAR_ERR_INVALID_ARG = 1,        /* NULL where data is required, negative size          */
+    PULSAR_ERR_SHAPE = 2,              /* shape outside what the kernels cover                */
+    PULSAR_ERR_ALIGNMENT = 3,          /* pointer not 16-byte (workspace: 256-byte) aligned   */
+    PULSAR_ERR_WORKSPACE = 4,          /* workspace_bytes below the *_workspace_bytes value   */
+    PULSAR_ERR_UNSUPPORTED_DEVICE = 5, /* current device is not sm_100                        */
+    PULSAR_ERR_CUDA = 6,               /* a CUDA runtime/driver call failed (launch, tensor map) */
+    PULSAR_ERR_TIMEOUT = 7,            /* device_status bit: a bounded device wait gave up    */
+    PULSAR_ERR_DEVICE_CHECK = 8        /* device_status bit: data-dependent check failed      */
+} pulsar_status_t;
+
+/* Bits OR-ed into *device_status by the kernels. */
+#define PULSAR_DEV_BAD_TOKEN   0x1 /* token id >= vocab_size (token ignored)                 */
+#define PULSAR_DEV_BAD_PREFIX  0x2 /* prefix index outside [0, first row of its block) (row 0 used) */
+#define PULSAR_DEV_TIMEOUT     0x4 /* an mbarrier wait exceeded its bound (results invalid)   */
+#define PULSAR_DEV_BAD_LENGTH  0x8 /* prefix_len[i] outside [0, prefix_total] (clamped)       */
+
+/* Static, human-readable name of a status code (host pointer, never NULL). */
+const char *pulsar_status_string(int32_t status);
+
+/* Version of this ABI (bumped on any signature change). */
+int32_t pulsar_abi_version(void);
+
+/* ------------------------------------------------------------------------------------------
+ * Max-IDF summary selection (Section 3.1; Algorithm 1 lines 3 and 6; Appendix C.1, C.5).
+ *
+ * The L context tokens form B = L / block_size logical blocks.  df(t) = number of blocks in
+ * which token t occurs; IDF(t) = ln(B / max(df(t),1)) (Eq. 3); each block is cut into
+ * C = block_size / chunk chunks scored by the largest IDF among their tokens (Eq. 2); the k
+ * best chunks of a block, equal scores going to the lower chunk index, listed in positional
+ * order, are its summary Sigma_b.  The prefix list is [0..sink-1 | Sigma_0 | ... | Sigma_{B-2}]
+ * as global token positions; block i attends to its first prefix_len[i] entries, with
+ * prefix_len[0] = 0 and prefix_len[i] = sink + i*k*chunk (Eq. 4, Eq. 14).  Ranking is done on
+ * the integer df (IDF is strictly decreasing in df), so the result is exact.
+ *
+ *   token_ids   in  [L] uint32, each < vocab_size
+ *   sel_chunks  out [B*k] int32: chunk indices within the block, ascending, for every block
+ *   prefix_idx  out [sink + (B-1)*k*chunk] int32
+ *   prefix_len  out [B] int32
+ *   df_out      out [vocab_size] uint32, or NULL
+ *   idf_out     out [vocab_size] float32 (natural log), or NULL
+ *
+ * Requirements (else PULSAR_ERR_SHAPE): L % block_size == 0, block_size % chunk == 0,
+ * 0 <= k <= C, 0 <= sink <= block_size, B <= 65535, vocab_size <= 1,800,000 (one block's
+ * presence bitmap must fit in shared memory), C <= 32768.
+ * ------------------------------------------------------------------------------------------ */
+size_t pulsar_maxidf_select_workspace_bytes(int64_t L, int32_t vocab_size, int32_t block_size,
+                                            int32_t chunk, int32_t k, int32_t sink);
+
+int32_t pulsar_maxidf_select(const uint32_t *token_ids, int64_t L, int32_t vocab_size,
+                             int32_t block_size, int32_t chunk, int32_t k, int32_t sink,
+                             int32_t *sel_chunks, int32_t *prefix_idx, int32_t *prefix_len,
+                             uint32_t *df_out, float *idf_out,
+                             void *workspace, size_t workspace_bytes,
+                             int32_t *device_status, void *stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Phase-1 prefix-block attention (Eq. 1 over the assembled input of Eq. 4; Alg. 1 l.7-8).
+ *
+ * For block i, row r (global position p = i*block_size + r) and query head h, the keys are
+ * rows prefix_idx[0 .. prefix_len[i]) followed by rows i*block_size .. p of K (KV head
+ * h / (Hq/Hkv)); the prefix is fully visible, the block causal; a row listed twice counts
+ * twice.  O = softmax(q.k * scale) V, LSE = ln sum exp(q.k * scale).  Only block rows are
+ * computed; the keys and values of the prefix are read from the given K and V, never
+ * produced, so the retained KV of block i (Alg. 1 l.8, Appendix F) is rows
+ * [i*block_size, (i+1)*block_size) of K and V themselves; K_ret/V_ret optionally receive a copy.
+ * A Star-Attention-style anchor is the same call with prefix_idx = 0..block_size-1 and
+ * prefix_len = {0, block_size, block_size, ...}.
+ *
+ *   Q           in  [L, Hq, d] bf16         K, V   in [L, Hkv, d] bf16
+ *   prefix_idx  in  [prefix_total] int32    prefix_len in [B] int32, B = L / block_size
+ *   softmax_scale   <= 0 selects 1/sqrt(d)
+ *   O           out [L, Hq, d] bf16         LSE    out [L, Hq] float32 (natural log) or NULL
+ *   K_ret,V_ret out [L, Hkv, d] bf16 (= [B, block_size, Hkv, d]) or NULL
+ *
+ * Requirements (else PULSAR_ERR_SHAPE): d in {64, 128}; Hq % Hkv == 0; L % block_size == 0;
+ * prefix_total >= 0; L < 2^31.  Arithmetic: bf16 operands, fp32 accumulation on the tensor
+ * cores, probabilities rounded to bf16 before the PV product, bf16 output.
+ * ------------------------------------------------------------------------------------------ */
+size_t pulsar_phase1_workspace_bytes(int64_t L, int32_t Hq, int32_t Hkv, int32_t d,
+                                     int32_t block_size, int32_t prefix_total);
+
+int32_t pulsar_phase1_attn(const uint16_t *Q, const uint16_t *K, const uint16_t *V,
+                           int64_t L, int32_t Hq, int32_t Hkv, int32_t d, int32_t block_size,
+                           const int32_t *prefix_idx, const int32_t *prefix_len,
+                           int32_t prefix_total, float softmax_scale,
+                           uint16_t *O, float *LSE, uint16_t *K_ret, uint16_t *V_ret,
+                           void *workspace, size_t workspace_bytes,
+                           int32_t *device_status, void *stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Phase-2 query attention over the retained KV of all blocks, merged exactly (Section 3.2;
+ * Algorithm 1 lines 12-13; Appendix H).
+ *
+ * Every query row attends, without mask, to all B*block_size retained keys of its KV head.
+ * The KV range is cut into n_splits contiguous parts (each "host" of the paper is a part on
+ * this GPU); a split-KV kernel produces per part the normalised output A_j and l_j = ln sum
+ * exp(q.k*scale) in fp32, and a merge kernel combines them: l = ln sum_j e^{l_j},
+ * O = sum_j e^{l_j - l} A_j, which equals one softmax over the concatenated keys.
+ *
+ *   Qq          in  [nq, Hq, d] bf16 (a batch of queries is flattened into nq rows)
+ *   Kblocks, Vblocks in [B, block_size, Hkv, d] bf16 (the retained rows, i.e. [L, Hkv, d])
+ *   n_splits    number of KV parts: 0 = let the library choose; otherwise 1 <= n_splits,
+ *               and (B*block_size) % n_splits == 0.  n_splits == B gives the per-block
+ *               (A_h, l_h) of Algorithm 1 line 12.
+ *   O           out [nq, Hq, d] bf16        LSE out [nq, Hq] float32 (natural log), or NULL
+ *   part_O      out [n_splits, nq, Hq, d] float32 or NULL (requires n_splits > 0)
+ *   part_LSE    out [n_splits, nq, Hq]    float32 or NULL (both or neither)
+ *
+ * Requirements (else PULSAR_ERR_SHAPE): d in {64,128}; Hq % Hkv == 0; Hq/Hkv in {1,2,4,8,16};
+ * nq >= 1.  pulsar_phase2_choose_splits returns the value used for n_splits == 0.
+ * ------------------------------------------------------------------------------------------ */
+int32_t pulsar_phase2_choose_splits(int32_t nq, int32_t B, int32_t block_size,
+                                    int32_t Hq, int32_t Hkv, int32_t d);
+
+size_t pulsar_phase2_workspace_bytes(int32_t nq, int32_t B, int32_t block_size,
+                                     int32_t Hq, int32_t Hkv, int32_t d, int32_t n_splits);
+
+int32_t pulsar_phase2_attn(const uint16_t *Qq, int32_t nq,
+                           const uint16_t *Kblocks, const uint16_t *Vblocks,
+                           int32_t B, int32_t block_size, int32_t Hq, int32_t Hkv, int32_t d,
+                           float softmax_scale, int32_t n_splits,
+                           uint16_t *O, float *LSE, float *part_O, float *part_LSE,
+                           void *workspace, size_t workspace_bytes,
+                           int32_t *device_status, void *stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Online-softmax merge (Appendix H, Eq. 12-13), in its order-free closed form:
+ *   l = m + ln sum_j e^{l_j - m} (m = max_j l_j),  O = sum_j e^{l_j - l} A_j.
+ * A part with l_j = -inf has weight 0.  Also the entry point for merging partials gathered
+ * from several GPUs.
+ *
+ *   part_O   in  [n_parts, rows, d] float32     part_LSE in [n_parts, rows] float32
+ *   O        out [rows, d] bf16                 LSE      out [rows] float32, or NULL
+ * Requirements: n_parts >= 1, rows >= 0, d % 4 == 0, d <= 1024.
+ * ------------------------------------------------------------------------------------------ */
+int32_t pulsar_lse_merge(const float *part_O, const float *part_LSE, int32_t n_parts,
+                         int64_t rows, int32_t d, uint16_t *O, float *LSE, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PULSAR_H_ */

@@ -1,0 +1,225 @@
+"""ctypes binding of the Pulsar CUDA library (``include/pulsar.h``).
+
+Argument marshalling only: tensors in, device pointers and sizes through the C
+ABI, tensors out.  Every step of the path runs in the library's kernels.  torch
+provides device memory and the stream; nothing here computes.  The library is
+required: if it is missing the first call raises, there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import _build
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_lib = None
+
+STATUS_NAMES = {
+    0: "PULSAR_OK", 1: "PULSAR_ERR_INVALID_ARG", 2: "PULSAR_ERR_SHAPE", 3: "PULSAR_ERR_ALIGNMENT",
+    4: "PULSAR_ERR_WORKSPACE", 5: "PULSAR_ERR_UNSUPPORTED_DEVICE", 6: "PULSAR_ERR_CUDA",
+    7: "PULSAR_ERR_TIMEOUT", 8: "PULSAR_ERR_DEVICE_CHECK",
+}
+DEV_BAD_TOKEN, DEV_BAD_PREFIX, DEV_TIMEOUT, DEV_BAD_LENGTH = 0x1, 0x2, 0x4, 0x8
+
+EXPORTS = (
+    "pulsar_status_string", "pulsar_abi_version",
+    "pulsar_maxidf_select_workspace_bytes", "pulsar_maxidf_select",
+    "pulsar_phase1_workspace_bytes", "pulsar_phase1_attn",
+    "pulsar_phase2_choose_splits", "pulsar_phase2_workspace_bytes", "pulsar_phase2_attn",
+    "pulsar_lse_merge",
+)
+
+
+class PulsarError(RuntimeError):
+    def __init__(self, call: str, status: int):
+        self.status = status
+        super().__init__(f"{call} failed: {STATUS_NAMES.get(status, status)}")
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def load_library(build_if_missing: bool = False):
+    """Load ``libpulsar.so`` (built in-tree).  Raises if it does not exist."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = library_path()
+    if not os.path.exists(path):
+        if build_if_missing:
+            _build.build()
+        else:
+            raise FileNotFoundError(
+                f"{path} is missing: build it with `python -m paper_2607_20457_b200._build` "
+                "(the CUDA library is the only implementation; there is no CPU path)")
+    lib = ctypes.CDLL(path)
+    i32, i64, vp, sz, f32 = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_float
+    lib.pulsar_status_string.argtypes = [i32]
+    lib.pulsar_status_string.restype = ctypes.c_char_p
+    lib.pulsar_abi_version.argtypes = []
+    lib.pulsar_abi_version.restype = i32
+    lib.pulsar_maxidf_select_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, i32]
+    lib.pulsar_maxidf_select_workspace_bytes.restype = sz
+    lib.pulsar_maxidf_select.argtypes = [vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+    lib.pulsar_maxidf_select.restype = i32
+    lib.pulsar_phase1_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, i32]
+    lib.pulsar_phase1_workspace_bytes.restype = sz
+    lib.pulsar_phase1_attn.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, vp, vp, i32, f32,
+                                       vp, vp, vp, vp, vp, sz, vp, vp]
+    lib.pulsar_phase1_attn.restype = i32
+    lib.pulsar_phase2_choose_splits.argtypes = [i32, i32, i32, i32, i32, i32]
+    lib.pulsar_phase2_choose_splits.restype = i32
+    lib.pulsar_phase2_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, i32, i32]
+    lib.pulsar_phase2_workspace_bytes.restype = sz
+    lib.pulsar_phase2_attn.argtypes = [vp, i32, vp, vp, i32, i32, i32, i32, i32, f32, i32,
+                                       vp, vp, vp, vp, vp, sz, vp, vp]
+    lib.pulsar_phase2_attn.restype = i32
+    lib.pulsar_lse_merge.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp]
+    lib.pulsar_lse_merge.restype = i32
+    _lib = lib
+    return lib
+
+
+def _p(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(call: str, rc: int):
+    if rc != 0:
+        raise PulsarError(call, rc)
+
+
+def _need(t: torch.Tensor, dtype, name: str):
+    if not (t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError(f"{name}: expected a contiguous CUDA tensor of {dtype}, got {t.dtype} on {t.device}")
+
+
+def _workspace(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def new_status(device) -> torch.Tensor:
+    """A zeroed device status word for the kernels' data-dependent checks."""
+    return torch.zeros(1, dtype=torch.int32, device=device)
+
+
+def maxidf_select_workspace_bytes(L, vocab_size, block_size, chunk, k, sink) -> int:
+    return load_library().pulsar_maxidf_select_workspace_bytes(L, vocab_size, block_size, chunk, k, sink)
+
+
+def pulsar_maxidf_select(token_ids: torch.Tensor, vocab_size: int, block_size: int, chunk: int, k: int,
+                         sink: int, want_df: bool = False, want_idf: bool = False, workspace=None,
+                         status=None):
+    """Max-IDF summary selection.  ``token_ids``: CUDA int32 [L] holding the uint32 ids.
+    Returns a dict of CUDA tensors: sel_chunks [B,k], prefix_idx, prefix_len [B] (+ df, idf)."""
+    lib = load_library()
+    _need(token_ids, torch.int32, "token_ids")
+    L = token_ids.numel()
+    dev = token_ids.device
+    B = L // block_size if block_size > 0 else 0
+    sel = torch.empty((max(B, 0), max(k, 0)), dtype=torch.int32, device=dev)
+    pidx = torch.empty(max(sink, 0) + max(B - 1, 0) * max(k, 0) * max(chunk, 0) + 4, dtype=torch.int32, device=dev)
+    plen = torch.empty(max(B, 1), dtype=torch.int32, device=dev)
+    df = torch.empty(vocab_size, dtype=torch.int32, device=dev) if want_df else None
+    idf = torch.empty(vocab_size, dtype=torch.float32, device=dev) if want_idf else None
+    if workspace is None:
+        workspace = _workspace(maxidf_select_workspace_bytes(L, vocab_size, block_size, chunk, k, sink), dev)
+    rc = lib.pulsar_maxidf_select(_p(token_ids), L, vocab_size, block_size, chunk, k, sink, _p(sel), _p(pidx),
+                                  _p(plen), _p(df), _p(idf), _p(workspace), workspace.numel(), _p(status),
+                                  _stream())
+    _check("pulsar_maxidf_select", rc)
+    n_pref = sink + max(B - 1, 0) * k * chunk
+    out = dict(sel_chunks=sel, prefix_idx=pidx[:n_pref], prefix_len=plen[:B])
+    if want_df:
+        out["df"] = df
+    if want_idf:
+        out["idf"] = idf
+    return out
+
+
+def phase1_workspace_bytes(L, Hq, Hkv, d, block_size, prefix_total) -> int:
+    return load_library().pulsar_phase1_workspace_bytes(L, Hq, Hkv, d, block_size, prefix_total)
+
+
+def pulsar_phase1_attn(Q, K, V, block_size: int, prefix_idx, prefix_len, softmax_scale: float = 0.0,
+                       want_lse: bool = True, retain_copy: bool = False, out=None, workspace=None, status=None):
+    """Phase-1 prefix-block attention.  Q [L,Hq,d], K,V [L,Hkv,d] CUDA bf16; prefix_idx,
+    prefix_len CUDA int32.  Returns (O bf16 [L,Hq,d], LSE f32 [L,Hq] or None, K_ret, V_ret)."""
+    lib = load_library()
+    for t, n in ((Q, "Q"), (K, "K"), (V, "V")):
+        _need(t, torch.bfloat16, n)
+    _need(prefix_len, torch.int32, "prefix_len")
+    _need(prefix_idx, torch.int32, "prefix_idx")
+    L, Hq, d = Q.shape
+    Hkv = K.shape[1]
+    dev = Q.device
+    prefix_total = prefix_idx.numel()
+    O = torch.empty_like(Q) if out is None else out
+    LSE = torch.empty((L, Hq), dtype=torch.float32, device=dev) if want_lse else None
+    K_ret = torch.empty_like(K) if retain_copy else None
+    V_ret = torch.empty_like(V) if retain_copy else None
+    if workspace is None:
+        workspace = _workspace(phase1_workspace_bytes(L, Hq, Hkv, d, block_size, prefix_total), dev)
+    rc = lib.pulsar_phase1_attn(_p(Q), _p(K), _p(V), L, Hq, Hkv, d, block_size,
+                                _p(prefix_idx) if prefix_total > 0 else None, _p(prefix_len), prefix_total,
+                                float(softmax_scale), _p(O), _p(LSE), _p(K_ret), _p(V_ret),
+                                _p(workspace), workspace.numel(), _p(status), _stream())
+    _check("pulsar_phase1_attn", rc)
+    if not retain_copy:
+        K_ret, V_ret = K, V          # the retained KV is the block's own rows of K and V
+    return O, LSE, K_ret, V_ret
+
+
+def phase2_choose_splits(nq, B, block_size, Hq, Hkv, d) -> int:
+    return load_library().pulsar_phase2_choose_splits(nq, B, block_size, Hq, Hkv, d)
+
+
+def phase2_workspace_bytes(nq, B, block_size, Hq, Hkv, d, n_splits=0) -> int:
+    return load_library().pulsar_phase2_workspace_bytes(nq, B, block_size, Hq, Hkv, d, n_splits)
+
+
+def pulsar_phase2_attn(Qq, Kblocks, Vblocks, n_blocks: int, block_size: int, softmax_scale: float = 0.0,
+                       n_splits: int = 0, want_partials: bool = False, out=None, workspace=None, status=None):
+    """Phase-2 query attention with exact LSE merge.  Qq [nq,Hq,d], K/V [n_blocks*block_size,Hkv,d]
+    CUDA bf16.  Returns (O bf16 [nq,Hq,d], LSE f32 [nq,Hq]) and, with ``want_partials``
+    (needs n_splits > 0), also (part_O f32 [J,nq,Hq,d], part_LSE f32 [J,nq,Hq])."""
+    lib = load_library()
+    for t, n in ((Qq, "Qq"), (Kblocks, "Kblocks"), (Vblocks, "Vblocks")):
+        _need(t, torch.bfloat16, n)
+    nq, Hq, d = Qq.shape
+    Hkv = Kblocks.shape[-2]
+    dev = Qq.device
+    O = torch.empty_like(Qq) if out is None else out
+    LSE = torch.empty((nq, Hq), dtype=torch.float32, device=dev)
+    pO = pL = None
+    if want_partials:
+        pO = torch.empty((n_splits, nq, Hq, d), dtype=torch.float32, device=dev)
+        pL = torch.empty((n_splits, nq, Hq), dtype=torch.float32, device=dev)
+    if workspace is None:
+        workspace = _workspace(phase2_workspace_bytes(nq, n_blocks, block_size, Hq, Hkv, d, n_splits), dev)
+    rc = lib.pulsar_phase2_attn(_p(Qq), nq, _p(Kblocks), _p(Vblocks), n_blocks, block_size, Hq, Hkv, d,
+                                float(softmax_scale), n_splits, _p(O), _p(LSE), _p(pO), _p(pL),
+                                _p(workspace), workspace.numel(), _p(status), _stream())
+    _check("pulsar_phase2_attn", rc)
+    return (O, LSE, pO, pL) if want_partials else (O, LSE)
+
+
+def pulsar_lse_merge(part_O, part_LSE, want_lse: bool = True):
+    """Merge partials: part_O f32 [J,rows,d], part_LSE f32 [J,rows] -> (O bf16 [rows,d], LSE f32 [rows])."""
+    lib = load_library()
+    _need(part_O, torch.float32, "part_O")
+    _need(part_LSE, torch.float32, "part_LSE")
+    J, rows, d = part_O.shape
+    O = torch.empty((rows, d), dtype=torch.bfloat16, device=part_O.device)
+    LSE = torch.empty(rows, dtype=torch.float32, device=part_O.device) if want_lse else None
+    rc = lib.pulsar_lse_merge(_p(part_O), _p(part_LSE), J, rows, d, _p(O), _p(LSE), _stream())
+    _check("pulsar_lse_merge", rc)
+    return O, LSE

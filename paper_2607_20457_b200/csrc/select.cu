@@ -1,0 +1,232 @@
+// Max-IDF summary selection (Section 3.1, Eq. 2-4; Algorithm 1 lines 3 and 6).
+//
+// Three launches on one stream, no host synchronisation:
+//   presence_kernel   one CTA per block: a V-bit presence set of the block's token ids, built
+//                     with shared-memory atomicOr and written to the workspace
+//   df_idf_kernel     one thread per vocabulary entry: df(t) = number of blocks whose set holds
+//                     t, IDF(t) = ln(B / max(df, 1))   (Eq. 3)
+//   topk_kernel       one CTA per block: per chunk the minimum df of its tokens (the chunk with
+//                     the largest IDF is the one with the smallest df, Eq. 2), a counting
+//                     select of the k best chunks with ties to the lower index, then the
+//                     block's part of the prefix list (Eq. 4)
+// Ranking uses the integer df only, so the selection is exact.
+#include "common.cuh"
+
+namespace pulsar {
+namespace {
+
+constexpr int kPresenceThreads = 1024;
+constexpr int kTopkThreads = 256;
+constexpr size_t kMaxDynSmem = 227 * 1024;
+
+__global__ void __launch_bounds__(kPresenceThreads)
+presence_kernel(const uint32_t* __restrict__ ids, int block_size, int vocab_size, int words,
+                uint32_t* __restrict__ bitmaps, int32_t* status) {
+    extern __shared__ uint32_t bits[];
+    const int b = blockIdx.x;
+    for (int w = threadIdx.x; w < words; w += blockDim.x) bits[w] = 0u;
+    __syncthreads();
+    const uint32_t* blk = ids + static_cast<size_t>(b) * block_size;
+    for (int i = threadIdx.x; i < block_size; i += blockDim.x) {
+        const uint32_t t = blk[i];
+        if (t < static_cast<uint32_t>(vocab_size)) atomicOr(&bits[t >> 5], 1u << (t & 31));
+        else report(status, PULSAR_DEV_BAD_TOKEN);
+    }
+    __syncthreads();
+    uint32_t* out = bitmaps + static_cast<size_t>(b) * words;
+    for (int w = threadIdx.x; w < words; w += blockDim.x) out[w] = bits[w];
+}
+
+__global__ void df_idf_kernel(const uint32_t* __restrict__ bitmaps, int n_blocks, int words, int vocab_size,
+                              uint16_t* __restrict__ df_table, uint32_t* __restrict__ df_out,
+                              float* __restrict__ idf_out) {
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= vocab_size) return;
+    const int w = t >> 5, bit = t & 31;
+    uint32_t df = 0;
+    for (int b = 0; b < n_blocks; ++b) df += (bitmaps[static_cast<size_t>(b) * words + w] >> bit) & 1u;
+    df_table[t] = static_cast<uint16_t>(df);
+    if (df_out) df_out[t] = df;
+    if (idf_out) idf_out[t] = logf(static_cast<float>(n_blocks) / static_cast<float>(df > 0 ? df : 1));
+}
+
+// Exclusive block-wide prefix sum of one int per thread; returns the thread's offset and the
+// block total through `total`.  warp_sums: kTopkThreads/32 ints of shared scratch.
+__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int n = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += n;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    int base = 0;
+    total = 0;
+    for (int i = 0; i < kTopkThreads / 32; ++i) {
+        int s = warp_sums[i];
+        if (i < warp) base += s;
+        total += s;
+    }
+    __syncthreads();
+    return base + incl - v;
+}
+
+__global__ void __launch_bounds__(kTopkThreads)
+topk_kernel(const uint32_t* __restrict__ ids, const uint16_t* __restrict__ df_table, int n_blocks,
+            int block_size, int chunk, int k, int sink, int vocab_size,
+            int32_t* __restrict__ sel_chunks, int32_t* __restrict__ prefix_idx, int32_t* __restrict__ prefix_len) {
+    extern __shared__ int smem[];
+    const int C = block_size / chunk;
+    int* level = smem;                       // [C]   min df of the chunk
+    int* hist = level + C;                   // [n_blocks + 2]
+    int* chosen = hist + n_blocks + 2;       // [k]   selected chunk ids, ascending
+    __shared__ int warp_sums[kTopkThreads / 32];
+    __shared__ int s_threshold, s_need;
+
+    const int b = blockIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t* blk = ids + static_cast<size_t>(b) * block_size;
+
+    for (int i = threadIdx.x; i < n_blocks + 2; i += blockDim.x) hist[i] = 0;
+    __syncthreads();
+
+    // chunk score: one warp per chunk, lanes stride over its tokens
+    for (int c = warp; c < C; c += kTopkThreads / 32) {
+        int mn = n_blocks + 1;               // ids outside the vocabulary rank last
+        for (int p = lane; p < chunk; p += 32) {
+            const uint32_t t = blk[c * chunk + p];
+            if (t < static_cast<uint32_t>(vocab_size)) mn = min(mn, static_cast<int>(df_table[t]));
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        if (lane == 0) {
+            level[c] = mn;
+            atomicAdd(&hist[mn], 1);
+        }
+    }
+    __syncthreads();
+
+    // threshold level T: all chunks below T are taken, `need` more at T (lowest indices first)
+    if (threadIdx.x == 0) {
+        int cum = 0, T = 0;
+        for (; T <= n_blocks + 1; ++T) {
+            if (cum + hist[T] >= k) break;
+            cum += hist[T];
+        }
+        s_threshold = T;
+        s_need = k - cum;
+    }
+    __syncthreads();
+    const int T = s_threshold, need = s_need;
+
+    // ordered compaction over the chunks, a tile of blockDim chunks at a time
+    int at_T_before = 0, taken_before = 0;
+    for (int c0 = 0; c0 < C; c0 += kTopkThreads) {
+        const int c = c0 + threadIdx.x;
+        const int lv = c < C ? level[c] : n_blocks + 2;
+        const int is_T = (lv == T) ? 1 : 0;
+        int tot_T;
+        const int rank_T = at_T_before + block_exclusive_scan(is_T, warp_sums, tot_T);
+        const int take = (lv < T || (is_T && rank_T < need)) ? 1 : 0;
+        int tot_take;
+        const int pos = taken_before + block_exclusive_scan(take, warp_sums, tot_take);
+        if (take && pos < k) {
+            chosen[pos] = c;
+            sel_chunks[static_cast<size_t>(b) * k + pos] = c;
+        }
+        at_T_before += tot_T;
+        taken_before += tot_take;
+    }
+    __syncthreads();
+
+    const int sigma = k * chunk;
+    if (b < n_blocks - 1) {
+        int32_t* dst = prefix_idx + sink + static_cast<size_t>(b) * sigma;
+        for (int i = threadIdx.x; i < sigma; i += blockDim.x) {
+            const int j = i / chunk, p = i - j * chunk;
+            dst[i] = b * block_size + chosen[j] * chunk + p;
+        }
+    }
+    if (b == 0)
+        for (int i = threadIdx.x; i < sink; i += blockDim.x) prefix_idx[i] = i;
+    if (threadIdx.x == 0) prefix_len[b] = b == 0 ? 0 : sink + b * sigma;
+}
+
+struct SelectPlan {
+    int n_blocks, words, C;
+    size_t bitmap_bytes, df_bytes, total;
+    size_t presence_smem, topk_smem;
+};
+
+int32_t plan_select(int64_t L, int32_t vocab_size, int32_t block_size, int32_t chunk, int32_t k, int32_t sink,
+                    SelectPlan& p) {
+    if (L <= 0 || vocab_size <= 0 || block_size <= 0 || chunk <= 0 || k < 0 || sink < 0) return PULSAR_ERR_INVALID_ARG;
+    if (L % block_size != 0 || block_size % chunk != 0) return PULSAR_ERR_SHAPE;
+    if (L >= (1ll << 31)) return PULSAR_ERR_SHAPE;
+    const int64_t B = L / block_size;
+    p.C = block_size / chunk;
+    if (B > 65535 || k > p.C || sink > block_size || p.C > 32768) return PULSAR_ERR_SHAPE;
+    p.n_blocks = static_cast<int>(B);
+    p.words = (vocab_size + 31) / 32;
+    p.presence_smem = static_cast<size_t>(p.words) * 4;
+    p.topk_smem = (static_cast<size_t>(p.C) + p.n_blocks + 2 + k) * 4;
+    if (p.presence_smem > kMaxDynSmem || p.topk_smem > kMaxDynSmem) return PULSAR_ERR_SHAPE;
+    p.bitmap_bytes = round_up(static_cast<size_t>(p.n_blocks) * p.words * 4, 256);
+    p.df_bytes = round_up(static_cast<size_t>(vocab_size) * 2, 256);
+    p.total = p.bitmap_bytes + p.df_bytes;
+    return PULSAR_OK;
+}
+
+}  // namespace
+}  // namespace pulsar
+
+using namespace pulsar;
+
+extern "C" size_t pulsar_maxidf_select_workspace_bytes(int64_t L, int32_t vocab_size, int32_t block_size,
+                                                       int32_t chunk, int32_t k, int32_t sink) {
+    SelectPlan p;
+    if (plan_select(L, vocab_size, block_size, chunk, k, sink, p) != PULSAR_OK) return 0;
+    return p.total;
+}
+
+extern "C" int32_t pulsar_maxidf_select(const uint32_t* token_ids, int64_t L, int32_t vocab_size,
+                                        int32_t block_size, int32_t chunk, int32_t k, int32_t sink,
+                                        int32_t* sel_chunks, int32_t* prefix_idx, int32_t* prefix_len,
+                                        uint32_t* df_out, float* idf_out, void* workspace,
+                                        size_t workspace_bytes, int32_t* device_status, void* stream_) {
+    SelectPlan p;
+    int32_t rc = plan_select(L, vocab_size, block_size, chunk, k, sink, p);
+    if (rc != PULSAR_OK) return rc;
+    if (!token_ids || !sel_chunks || !prefix_idx || !prefix_len || !workspace) return PULSAR_ERR_INVALID_ARG;
+    if (!aligned(token_ids, 16) || !aligned(sel_chunks, 16) || !aligned(prefix_idx, 16) || !aligned(prefix_len, 16) ||
+        (df_out && !aligned(df_out, 16)) || (idf_out && !aligned(idf_out, 16)) || !aligned(workspace, 256))
+        return PULSAR_ERR_ALIGNMENT;
+    if (workspace_bytes < p.total) return PULSAR_ERR_WORKSPACE;
+    rc = check_device();
+    if (rc != PULSAR_OK) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+
+    uint32_t* bitmaps = static_cast<uint32_t*>(workspace);
+    uint16_t* df_table = reinterpret_cast<uint16_t*>(static_cast<char*>(workspace) + p.bitmap_bytes);
+
+    if (p.presence_smem > 48 * 1024)
+        PULSAR_CUDA_OK(cudaFuncSetAttribute(presence_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            static_cast<int>(p.presence_smem)));
+    if (p.topk_smem > 48 * 1024)
+        PULSAR_CUDA_OK(cudaFuncSetAttribute(topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            static_cast<int>(p.topk_smem)));
+
+    presence_kernel<<<p.n_blocks, kPresenceThreads, p.presence_smem, stream>>>(
+        token_ids, block_size, vocab_size, p.words, bitmaps, device_status);
+    PULSAR_CUDA_OK(cudaGetLastError());
+    df_idf_kernel<<<(vocab_size + 255) / 256, 256, 0, stream>>>(bitmaps, p.n_blocks, p.words, vocab_size, df_table,
+                                                                df_out, idf_out);
+    PULSAR_CUDA_OK(cudaGetLastError());
+    topk_kernel<<<p.n_blocks, kTopkThreads, p.topk_smem, stream>>>(token_ids, df_table, p.n_blocks, block_size, chunk,
+                                                                   k, sink, vocab_size, sel_chunks, prefix_idx,
+                                                                   prefix_len);
+    PULSAR_CUDA_OK(cudaGetLastError());
+    return PULSAR_OK;
+}

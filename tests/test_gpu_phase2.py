@@ -1,0 +1,98 @@
+"""GPU parity: Phase-2 split-KV attention and the LSE merge against the oracle (Section 3.2, App. H)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import check_attention, TOL_LSE_ABS
+from paper_2607_20457_b200 import binding, workloads as W
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def run_phase2(w, Qq, K, V, n_splits=0, what="", scale=0.0):
+    status = binding.new_status(DEV)
+    O, LSE = binding.pulsar_phase2_attn(Qq.to(DEV), K.to(DEV), V.to(DEV), w.n_blocks, w.block_size,
+                                        softmax_scale=scale, n_splits=n_splits, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    Oref, Lref = oracle.phase2_attn(Qq, K, V, w.n_blocks, w.block_size, scale=scale)
+    return check_attention(O, LSE, Oref, Lref, what)
+
+
+@pytest.mark.parametrize("n_splits", [0, 1, 4, 32])
+def test_tiny_config(n_splits):
+    w = W.CONFIGS["tiny"]
+    _, K, V = W.qkv(w)
+    print(run_phase2(w, W.phase2_query(w), K, V, n_splits, what=f"tiny J={n_splits}"))
+
+
+def test_tiny_peaked():
+    w = W.CONFIGS["tiny"]
+    _, K, V = W.qkv(w)
+    print(run_phase2(w, W.phase2_query(w, q_scale=6.0), K, V, 4, what="tiny peaked"))
+
+
+@pytest.mark.parametrize("shape", [
+    dict(L=1000, block_size=250, Hq=4, Hkv=2, d=128, nq=1),       # decode shape, ragged keys
+    dict(L=768, block_size=192, Hq=8, Hkv=1, d=64, nq=17),        # g = 8, ragged rows
+    dict(L=512, block_size=128, Hq=2, Hkv=2, d=128, nq=130),      # g = 1, more than one row tile
+    dict(L=640, block_size=320, Hq=16, Hkv=1, d=64, nq=9),        # g = 16
+])
+@pytest.mark.parametrize("n_splits", [1, 2])
+def test_small_shapes(shape, n_splits):
+    w = W.shrink(W.CONFIGS["tiny"], **shape)
+    _, K, V = W.qkv(w)
+    print(run_phase2(w, W.phase2_query(w, q_scale=2.0), K, V, n_splits, what=f"{shape} J={n_splits}", scale=0.2))
+
+
+def test_per_block_partials_match_oracle_partials():
+    w = W.CONFIGS["tiny"]
+    _, K, V = W.qkv(w)
+    Qq = W.phase2_query(w)
+    O, LSE, pO, pL = binding.pulsar_phase2_attn(Qq.to(DEV), K.to(DEV), V.to(DEV), w.n_blocks, w.block_size,
+                                                n_splits=w.n_blocks, want_partials=True)
+    Oref, Lref, pOref, pLref = oracle.phase2_attn(Qq, K, V, w.n_blocks, w.block_size, partials=True)
+    for b in range(w.n_blocks):
+        check_attention(pO[b], pL[b], pOref[b], pLref[b], f"block {b} partial")
+    check_attention(O, LSE, Oref, Lref, "merged")
+
+
+@pytest.mark.parametrize("name,nq", [("16k", None), ("128k", 64), ("128k", 1)])
+def test_full_size_kv(name, nq):
+    w = W.CONFIGS[name]
+    _, K, V = W.qkv(w)
+    Qq = W.phase2_query(w, nq=nq)
+    print(run_phase2(w, Qq, K, V, 0, what=f"{name} nq={Qq.shape[0]}"))
+
+
+def test_merge_entry_point_against_oracle_merge():
+    rng = np.random.default_rng(0)
+    J, rows, d = 5, 333, 128
+    pO = rng.standard_normal((J, rows, d))
+    pL = rng.standard_normal((J, rows)) * 4
+    pL[2, :7] = -np.inf                                   # an empty part has weight zero
+    Oref, Lref = oracle.lse_merge(pO.astype(np.float32).astype(np.float64),
+                                  np.where(np.isinf(pL), -1e30, pL.astype(np.float32).astype(np.float64)))
+    O, LSE = binding.pulsar_lse_merge(torch.from_numpy(pO.astype(np.float32)).to(DEV),
+                                      torch.from_numpy(pL.astype(np.float32)).to(DEV))
+    torch.cuda.synchronize()
+    assert np.abs(O.float().cpu().numpy() - Oref).max() <= 1e-2
+    assert np.abs(LSE.cpu().numpy() - Lref).max() <= TOL_LSE_ABS
+    # one part: identity up to the bf16 rounding of the output
+    O1, L1 = binding.pulsar_lse_merge(torch.from_numpy(pO[:1].astype(np.float32)).to(DEV),
+                                      torch.from_numpy(pL[:1].astype(np.float32)).to(DEV))
+    assert torch.equal(O1, torch.from_numpy(pO[0].astype(np.float32)).to(DEV).to(torch.bfloat16))
+
+
+def test_phase1_then_phase2_chain_on_retained_kv():
+    w = W.CONFIGS["tiny"]
+    Q, K, V = W.qkv(w)
+    pidx, plen = W.first_k_prefix(w)
+    _, _, Kr, Vr = binding.pulsar_phase1_attn(Q.to(DEV), K.to(DEV), V.to(DEV), w.block_size,
+                                              torch.from_numpy(pidx).to(DEV), torch.from_numpy(plen).to(DEV))
+    Qq = W.phase2_query(w)
+    O, LSE = binding.pulsar_phase2_attn(Qq.to(DEV), Kr, Vr, w.n_blocks, w.block_size)
+    Oref, Lref = oracle.phase2_attn(Qq, K, V, w.n_blocks, w.block_size)
+    check_attention(O, LSE, Oref, Lref, "chain")
