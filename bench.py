@@ -1,0 +1,382 @@
+#!/usr/bin/env python
+"""Benchmark of the Pulsar context-encoding hot path on B200.
+
+A step is one pass of the whole path -- Max-IDF selection, Phase-1 prefix-block
+attention, Phase-2 query attention with LSE merge -- over one synthetic 128K-token
+sequence with Llama-3.1-8B attention shapes (one layer).  The metric is context
+tokens per second per layer.  One process per GPU; with N > 1 every rank encodes
+its own sequence (independent problems, no data-path collective: weak scaling).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 128k] [--impl reference]
+
+Prints one JSON line on rank 0.  ``--impl reference`` times the float64 CPU oracle
+on a bounded sample of the same workload instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2607_20457_b200 import cost_model as cm
+from paper_2607_20457_b200 import workloads as W
+
+METRIC = "context_tokens_per_s_per_layer"
+UNIT = "tokens/s"
+LAUNCHES_PER_STEP = None   # measured from the library's own launch counter
+
+
+# --------------------------------------------------------------------------------------------
+# helpers
+# --------------------------------------------------------------------------------------------
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_burst=p["bf16_tflops"], bf16_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.proc = None
+        try:
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["unsampled"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["unsampled"])
+        return dict(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), power_w_max=max(power), samples=len(sm),
+                    reasons=sorted(reasons))
+
+
+def dist_setup(n_gpus: int):
+    """Returns (rank, world, local_rank).  Initialises NCCL only when launched with N > 1."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    return rank, world, local
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def max_over_ranks(value: float, world: int, device) -> float:
+    """The slowest rank's figure (what a whole job waits for)."""
+    if world <= 1:
+        return value
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+# --------------------------------------------------------------------------------------------
+# CPU oracle on a bounded sample (cpu_baseline leg and --impl reference)
+# --------------------------------------------------------------------------------------------
+def oracle_sample(w, ids, Q, K, V, Qq, rows_per_block=12, p2_rows=6):
+    """Times the float64 oracle, as it stands, on a bounded sample of the workload and scales
+    the three parts to one full step by exact work counts.  Returns a dict."""
+    import oracle
+    t0 = time.perf_counter()
+    sel = oracle.maxidf_select(ids, w.vocab_size, w.block_size, w.chunk, w.k, w.sink)
+    t_sel = time.perf_counter() - t0
+    pidx, plen = sel["prefix_idx"], sel["prefix_len"]
+    rows = W.sample_rows(w, per_block=rows_per_block)
+    t0 = time.perf_counter()
+    oracle.phase1_attn(Q, K, V, w.block_size, pidx, plen, rows=rows)
+    t_p1 = time.perf_counter() - t0
+    sample_pairs = int(sum(int(plen[r // w.block_size]) + (r % w.block_size) + 1 for r in rows))
+    total_pairs = cm.phase1_pairs(w.block_size, plen)
+    n2 = min(p2_rows, w.nq)
+    t0 = time.perf_counter()
+    oracle.phase2_attn(Qq[:n2], K, V, w.n_blocks, w.block_size)
+    t_p2 = time.perf_counter() - t0
+    est_step = t_sel + t_p1 * total_pairs / sample_pairs + t_p2 * w.nq / n2
+    return dict(
+        value=w.L / est_step, seconds_measured=t_sel + t_p1 + t_p2, est_step_seconds=est_step,
+        cores=oracle.num_threads(),
+        sample=(f"selection in full ({t_sel:.3f}s); Phase 1 on {len(rows)} sampled query positions x all heads "
+                f"({sample_pairs} of {total_pairs} (q,k) pairs per head, {t_p1:.2f}s); Phase 2 on {n2} of {w.nq} "
+                f"query rows ({t_p2:.2f}s); each part scaled to the full step by its exact work count"))
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    ids = W.token_ids(w)
+    Q, K, V = W.qkv(w)
+    Qq = W.phase2_query(w)
+    import oracle
+    oracle.build()
+    times, last = [], None
+    for i in range(args.warmup + args.steps):
+        last = oracle_sample(w, ids, Q, K, V, Qq, rows_per_block=2, p2_rows=1)
+        if i >= args.warmup:
+            times.append(last["est_step_seconds"])
+    est = statistics.mean(times)
+    value = w.L / est
+    line = dict(
+        impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+        warmup=args.warmup, ms_per_step=est * 1e3, higher_is_better=True, scaling="weak", vs_baseline=None,
+        dtype="f64", data="synthetic",
+        config=dict(workload=w.name, L=w.L, blocks=w.n_blocks, block_size=w.block_size, chunk=w.chunk, k=w.k,
+                    sink=w.sink, Hq=w.Hq, Hkv=w.Hkv, d=w.d, phase2_query_rows=w.nq),
+        cpu_baseline=dict(value=value, unit=UNIT, cores=last["cores"], kind="oracle", sample=last["sample"]),
+        e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+        gpu_launches=0,
+        note="float64 CPU oracle; each step is a bounded sample scaled to a full step by exact work counts")
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------------
+# GPU arm
+# --------------------------------------------------------------------------------------------
+def time_calls(fn, iters, warmup=3):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
+    for a, b in evs:
+        a.record(); fn(); b.record()
+    torch.cuda.synchronize()
+    ts = sorted(a.elapsed_time(b) for a, b in evs)
+    return dict(median_ms=ts[len(ts) // 2], min_ms=ts[0])
+
+
+def run_gpu(args, w):
+    from paper_2607_20457_b200 import binding
+    from paper_2607_20457_b200.pipeline import ContextEncoder
+
+    rank, world, local = dist_setup(args.gpus)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (B200); there is no CPU path")
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    binding.load_library()
+    peaks = load_peaks()
+
+    # every rank encodes its own sequence
+    wl = W.shrink(w, ids_seed=w.ids_seed + 17 * rank)
+    ids = W.token_ids(wl)
+    Q, K, V = W.qkv(wl, seed=1 + 100 * rank)
+    Qq = W.phase2_query(wl, seed=2 + 100 * rank)
+    enc = ContextEncoder(wl, dev)
+    h = enc.host_buffers()
+    h["ids"].copy_(torch.from_numpy(ids.view(np.int32)))
+    h["Q"].copy_(Q); h["K"].copy_(K); h["V"].copy_(V); h["Qq"].copy_(Qq)
+    ids_d, Q_d, K_d, V_d, Qq_d = (h[n].to(dev) for n in ("ids", "Q", "K", "V", "Qq"))
+
+    # ---- device-resident steps -----------------------------------------------------------
+    for _ in range(args.warmup):
+        enc.step_device(ids_d, Q_d, K_d, V_d, Qq_d)
+    torch.cuda.synchronize()
+    marks = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local) if rank == 0 else None
+    launches0 = binding.launch_count()
+    barrier(world); torch.cuda.synchronize()
+    start.record()
+    for i in range(args.steps):
+        enc.step_device(ids_d, Q_d, K_d, V_d, Qq_d, record=marks[i])
+    stop.record()
+    torch.cuda.synchronize(); barrier(world)
+    launches = binding.launch_count() - launches0
+    clocks = sampler.stop() if sampler else None
+    dev_ms = max_over_ranks(start.elapsed_time(stop), world, dev)
+    status = int(enc.status.item())
+    sel_ms = statistics.mean(m[0].elapsed_time(m[1]) for m in marks)
+    p1_ms = statistics.mean(m[1].elapsed_time(m[2]) for m in marks)
+    p2_ms = statistics.mean(m[2].elapsed_time(m[3]) for m in marks)
+
+    # ---- end to end from pinned host buffers ---------------------------------------------
+    e2e_steps = max(2, min(args.steps, 5))
+    h2d = d2h = 0
+    for _ in range(2):
+        enc.step_host(h)
+    torch.cuda.synchronize(); barrier(world)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        h2d, d2h = enc.step_host(h)
+    e1.record()
+    torch.cuda.synchronize(); barrier(world)
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, dev) / e2e_steps
+
+    if rank != 0:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+        return
+
+    ms_per_step = dev_ms / args.steps
+    value = world * wl.L / (ms_per_step * 1e-3)
+    plen = cm.prefix_lens(wl.n_blocks, wl.sink, wl.sigma)
+    p1_flops = cm.phase1_flops(wl.block_size, plen, wl.Hq, wl.d)
+    achieved_tf = p1_flops / (p1_ms * 1e-3) / 1e12
+    p2_flops = cm.phase2_flops(wl.nq, wl.L, wl.Hq, wl.d)
+    p2_bytes = cm.phase2_hbm_bytes(wl.nq, wl.L, wl.Hq, wl.Hkv, wl.d, enc.n_splits if enc.n_splits > 1 else 0)
+
+    extras = {}
+    if args.extras:
+        extras = run_extras(binding, wl, dev, K_d, V_d, peaks)
+
+    cpu = oracle_sample(wl, ids, Q, K, V, Qq) if args.cpu_baseline else None
+
+    line = dict(
+        metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+        ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
+        dtype="bf16", data="synthetic",
+        config=dict(workload=wl.name, L=wl.L, blocks=wl.n_blocks, block_size=wl.block_size, chunk=wl.chunk, k=wl.k,
+                    sink=wl.sink, vocab=wl.vocab_size, Hq=wl.Hq, Hkv=wl.Hkv, d=wl.d, phase2_query_rows=wl.nq,
+                    phase2_splits=enc.n_splits, ids="zipf(1.1)", qkv="N(0,1) bf16",
+                    cache="inputs (2.5 GiB) larger than the 126 MB L2; no flush needed",
+                    sequences_per_gpu=1),
+        parts=dict(select_us=sel_ms * 1e3, phase1_ms=p1_ms, phase2_ms=p2_ms,
+                   phase1_tokens_per_s=wl.L / (p1_ms * 1e-3),
+                   phase1_tflops=achieved_tf, phase1_frac_of_spec_2250=achieved_tf / 2250.0,
+                   phase1_frac_of_measured_burst=achieved_tf / peaks["bf16_burst"],
+                   phase2_tflops=p2_flops / (p2_ms * 1e-3) / 1e12,
+                   phase2_gbs=p2_bytes / (p2_ms * 1e-3) / 1e9,
+                   phase2_bound="tensor (2048 query rows share every KV row)"),
+        roofline=dict(bound="tensor", kernel="attn_kernel<128> (Phase 1)", achieved=achieved_tf,
+                      peak=peaks["bf16_sustained"], unit="TFLOP/s", frac=achieved_tf / peaks["bf16_sustained"],
+                      peak_source=f"{peaks['source']} sustained bf16 (kernel timed inside a long step)",
+                      algorithmic_flops_per_launch=p1_flops, traffic=args.traffic_bytes,
+                      timed="CUDA events around pulsar_phase1_attn (prefix gather + attention kernel)"),
+        e2e=dict(value=world * wl.L / (e2e_ms * 1e-3), unit=UNIT, ms_per_step=e2e_ms,
+                 h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h, steps=e2e_steps),
+        gpu_launches=launches, device_status=status, clocks=clocks,
+        paper_context=("paper reports up to 3.3x fewer Phase-1 FLOPs per GPU than Star Attention "
+                       "(analytical, B=4, 64K, 4xA100-80GB); no absolute throughput published"),
+    )
+    if cpu is not None:
+        line["cpu_baseline"] = dict(value=cpu["value"], unit=UNIT, cores=cpu["cores"], kind="oracle",
+                                    sample=cpu["sample"], seconds_measured=cpu["seconds_measured"])
+    if extras:
+        line["extras"] = extras
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def run_extras(binding, w, dev, K_d, V_d, peaks):
+    """Context measurements beside the headline: decode-shaped Phase 2 (HBM-bound) and the
+    Star-anchor prefix against the Pulsar prefix through the same Phase-1 kernel (64K config)."""
+    out = {}
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    for name, nq in (("phase2_decode_8x1", 8), ("phase2_decode_1x1", 1)):
+        Qd = W.phase2_query(w, nq=nq).to(dev)
+        J = binding.phase2_choose_splits(nq, w.n_blocks, w.block_size, w.Hq, w.Hkv, w.d)
+        ws = binding._workspace(binding.phase2_workspace_bytes(nq, w.n_blocks, w.block_size, w.Hq, w.Hkv, w.d, J), dev)
+        O = torch.empty_like(Qd)
+
+        def call():
+            flush.zero_()
+            binding.pulsar_phase2_attn(Qd, K_d, V_d, w.n_blocks, w.block_size, n_splits=J, out=O, workspace=ws)
+        both = time_calls(call, 10)
+        only_flush = time_calls(lambda: flush.zero_(), 10)
+        ms = both["median_ms"] - only_flush["median_ms"]
+        nbytes = cm.phase2_hbm_bytes(nq, w.L, w.Hq, w.Hkv, w.d, J if J > 1 else 0)
+        out[name] = dict(ms=ms, splits=J, gbs=nbytes / (ms * 1e-3) / 1e9,
+                         frac_of_measured_hbm=nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                         l2="flushed by a 512 MiB memset before every call (its time subtracted)")
+    del flush
+    w4 = W.CONFIGS["64k"]
+    Q, K, V = (t.to(dev) for t in W.qkv(w4))
+    ws = binding._workspace(binding.phase1_workspace_bytes(w4.L, w4.Hq, w4.Hkv, w4.d, w4.block_size, w4.block_size), dev)
+    O = torch.empty_like(Q)
+    res = {}
+    for tag, (pidx, plen) in (("pulsar", W.first_k_prefix(w4)), ("star_anchor", W.star_anchor_prefix(w4))):
+        pi, pl = torch.from_numpy(pidx).to(dev), torch.from_numpy(plen).to(dev)
+        t = time_calls(lambda: binding.pulsar_phase1_attn(Q, K, V, w4.block_size, pi, pl, out=O, workspace=ws), 5)
+        fl = cm.phase1_flops(w4.block_size, plen, w4.Hq, w4.d)
+        res[tag] = dict(ms=t["median_ms"], tflop=fl / 1e12, tflops=fl / (t["median_ms"] * 1e-3) / 1e12)
+    res["flop_ratio_star_over_pulsar"] = res["star_anchor"]["tflop"] / res["pulsar"]["tflop"]
+    res["time_ratio_star_over_pulsar"] = res["star_anchor"]["ms"] / res["pulsar"]["ms"]
+    out["phase1_64k_prefix_comparison"] = res
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="128k", choices=list(W.CONFIGS))
+    ap.add_argument("--impl", default="pulsar", choices=["pulsar", "reference"])
+    ap.add_argument("--no-extras", dest="extras", action="store_false")
+    ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--traffic-bytes", type=float, default=None,
+                    help="DRAM bytes per Phase-1 launch from an ncu capture (reported as roofline.traffic)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "pulsar" else args.warmup
+    w = W.CONFIGS[args.workload]
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+    if world > 1:
+        args.extras = False
+        args.cpu_baseline = False
+    run_gpu(args, w)
+
+
+if __name__ == "__main__":
+    main()

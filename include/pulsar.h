@@ -64,6 +64,10 @@ const char *pulsar_status_string(int32_t status);
 /* Version of this ABI (bumped on any signature change). */
 int32_t pulsar_abi_version(void);
 
+/* Number of kernels this library has launched in this process so far (all entry points, all
+ * threads).  Bookkeeping for benchmarks; the paper has no counterpart. */
+uint64_t pulsar_launch_count(void);
+
 /* ------------------------------------------------------------------------------------------
  * Max-IDF summary selection (Section 3.1; Algorithm 1 lines 3 and 6; Appendix C.1, C.5).
  *

@@ -25,7 +25,7 @@ STATUS_NAMES = {
 DEV_BAD_TOKEN, DEV_BAD_PREFIX, DEV_TIMEOUT, DEV_BAD_LENGTH = 0x1, 0x2, 0x4, 0x8
 
 EXPORTS = (
-    "pulsar_status_string", "pulsar_abi_version",
+    "pulsar_status_string", "pulsar_abi_version", "pulsar_launch_count",
     "pulsar_maxidf_select_workspace_bytes", "pulsar_maxidf_select",
     "pulsar_phase1_workspace_bytes", "pulsar_phase1_attn",
     "pulsar_phase2_choose_splits", "pulsar_phase2_workspace_bytes", "pulsar_phase2_attn",
@@ -62,6 +62,8 @@ def load_library(build_if_missing: bool = False):
     lib.pulsar_status_string.restype = ctypes.c_char_p
     lib.pulsar_abi_version.argtypes = []
     lib.pulsar_abi_version.restype = i32
+    lib.pulsar_launch_count.argtypes = []
+    lib.pulsar_launch_count.restype = ctypes.c_uint64
     lib.pulsar_maxidf_select_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, i32]
     lib.pulsar_maxidf_select_workspace_bytes.restype = sz
     lib.pulsar_maxidf_select.argtypes = [vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp, vp]
@@ -106,6 +108,11 @@ def _workspace(nbytes: int, device) -> torch.Tensor:
     return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
 
 
+def launch_count() -> int:
+    """Kernels launched by the library in this process so far."""
+    return int(load_library().pulsar_launch_count())
+
+
 def new_status(device) -> torch.Tensor:
     """A zeroed device status word for the kernels' data-dependent checks."""
     return torch.zeros(1, dtype=torch.int32, device=device)
@@ -125,18 +132,19 @@ def pulsar_maxidf_select(token_ids: torch.Tensor, vocab_size: int, block_size: i
     L = token_ids.numel()
     dev = token_ids.device
     B = L // block_size if block_size > 0 else 0
-    sel = torch.empty((max(B, 0), max(k, 0)), dtype=torch.int32, device=dev)
+    sel_buf = torch.empty(max(B, 0) * max(k, 0) + 4, dtype=torch.int32, device=dev)
     pidx = torch.empty(max(sink, 0) + max(B - 1, 0) * max(k, 0) * max(chunk, 0) + 4, dtype=torch.int32, device=dev)
     plen = torch.empty(max(B, 1), dtype=torch.int32, device=dev)
     df = torch.empty(vocab_size, dtype=torch.int32, device=dev) if want_df else None
     idf = torch.empty(vocab_size, dtype=torch.float32, device=dev) if want_idf else None
     if workspace is None:
         workspace = _workspace(maxidf_select_workspace_bytes(L, vocab_size, block_size, chunk, k, sink), dev)
-    rc = lib.pulsar_maxidf_select(_p(token_ids), L, vocab_size, block_size, chunk, k, sink, _p(sel), _p(pidx),
+    rc = lib.pulsar_maxidf_select(_p(token_ids), L, vocab_size, block_size, chunk, k, sink, _p(sel_buf), _p(pidx),
                                   _p(plen), _p(df), _p(idf), _p(workspace), workspace.numel(), _p(status),
                                   _stream())
     _check("pulsar_maxidf_select", rc)
     n_pref = sink + max(B - 1, 0) * k * chunk
+    sel = sel_buf[: B * k].view(B, k)
     out = dict(sel_chunks=sel, prefix_idx=pidx[:n_pref], prefix_len=plen[:B])
     if want_df:
         out["df"] = df

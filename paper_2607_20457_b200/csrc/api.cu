@@ -1,4 +1,6 @@
 // Status strings, ABI version and the device gate shared by all entry points.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace pulsar {
@@ -31,6 +33,9 @@ int sm_count() {
     return cached;
 }
 
+static std::atomic<uint64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(static_cast<uint64_t>(n), std::memory_order_relaxed); }
+
 }  // namespace pulsar
 
 extern "C" const char* pulsar_status_string(int32_t status) {
@@ -49,3 +54,5 @@ extern "C" const char* pulsar_status_string(int32_t status) {
 }
 
 extern "C" int32_t pulsar_abi_version(void) { return 1; }
+
+extern "C" uint64_t pulsar_launch_count(void) { return pulsar::g_launches.load(std::memory_order_relaxed); }

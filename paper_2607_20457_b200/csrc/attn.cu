@@ -405,6 +405,7 @@ int32_t launch_attn(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMa
     }
     attn_kernel<D><<<grid, 128, smem, stream>>>(q, k, v, kp, vp, a);
     PULSAR_CUDA_OK(cudaGetLastError());
+    count_launch();
     return PULSAR_OK;
 }
 
@@ -493,6 +494,8 @@ extern "C" int32_t pulsar_phase1_attn(const uint16_t* Q, const uint16_t* K, cons
             block_size, L, Hkv * d * 2 / 16, reinterpret_cast<uint4*>(Kp), reinterpret_cast<uint4*>(Vp),
             device_status);
         PULSAR_CUDA_OK(cudaGetLastError());
+        count_launch();
+    count_launch();
     }
 
     AttnArgs a{};

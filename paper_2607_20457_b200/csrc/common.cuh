@@ -15,6 +15,7 @@ namespace pulsar {
 // ---------------------------------------------------------------------------------------
 int32_t check_device();                       // PULSAR_OK iff the current device is sm_100
 int     sm_count();                           // SMs of the current device (cached)
+void    count_launch(int n = 1);              // adds to the process-wide kernel launch counter
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

@@ -45,6 +45,7 @@ int32_t launch_lse_merge(const float* part_O, const float* part_LSE, int32_t n_p
     if (blocks > 0x7fffffffll) return PULSAR_ERR_SHAPE;
     lse_merge_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(part_O, part_LSE, n_parts, rows, d, O, LSE);
     PULSAR_CUDA_OK(cudaGetLastError());
+    count_launch();
     return PULSAR_OK;
 }
 

@@ -221,12 +221,15 @@ extern "C" int32_t pulsar_maxidf_select(const uint32_t* token_ids, int64_t L, in
     presence_kernel<<<p.n_blocks, kPresenceThreads, p.presence_smem, stream>>>(
         token_ids, block_size, vocab_size, p.words, bitmaps, device_status);
     PULSAR_CUDA_OK(cudaGetLastError());
+    count_launch();
     df_idf_kernel<<<(vocab_size + 255) / 256, 256, 0, stream>>>(bitmaps, p.n_blocks, p.words, vocab_size, df_table,
                                                                 df_out, idf_out);
     PULSAR_CUDA_OK(cudaGetLastError());
+    count_launch();
     topk_kernel<<<p.n_blocks, kTopkThreads, p.topk_smem, stream>>>(token_ids, df_table, p.n_blocks, block_size, chunk,
                                                                    k, sink, vocab_size, sel_chunks, prefix_idx,
                                                                    prefix_len);
     PULSAR_CUDA_OK(cudaGetLastError());
+    count_launch();
     return PULSAR_OK;
 }
