@@ -495,7 +495,6 @@ extern "C" int32_t pulsar_phase1_attn(const uint16_t* Q, const uint16_t* K, cons
             device_status);
         PULSAR_CUDA_OK(cudaGetLastError());
         count_launch();
-    count_launch();
     }
 
     AttnArgs a{};
