@@ -38,6 +38,10 @@ struct AttnArgs {
     int prefix_total;      // phase 1: rows in the gathered prefix buffers
     const int32_t* prefix_len;
     int split_len;         // phase 2: keys per KV part
+    int Hkv;
+    int pairs;             // phase 1: query-tile pairs per block; phase 2: query-tile pairs per KV head
+    int n_items;           // work items in total
+    const int32_t* order;  // phase 1: (block, pair) combos, costliest first
     float scale_log2;      // softmax scale * log2(e)
     uint16_t* O;           // bf16 [tokens, Hq, d]   (final output mode)
     float* LSE;            // f32  [tokens, Hq] or null
@@ -76,31 +80,133 @@ gather_prefix_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V, c
 }
 
 // ---------------------------------------------------------------------------------------------
-// Attention kernel
+// Phase-1 work order: one entry per (block, pair of query tiles), costliest first, so that a
+// static round-robin over the persistent CTAs ends level (longest-processing-time-first).
+// Cost in key tiles: 2 * prefix tiles + block tiles of both query tiles.  Single CTA.
 // ---------------------------------------------------------------------------------------------
+constexpr int kPlanBins = 4096;
+
+__global__ void __launch_bounds__(256)
+phase1_plan_kernel(const int32_t* __restrict__ prefix_len, int n_blocks, int pairs_per_block, int prefix_total,
+                   int32_t* __restrict__ order, int32_t* status) {
+    __shared__ int bins[kPlanBins];
+    const int n_combos = n_blocks * pairs_per_block;
+    for (int i = threadIdx.x; i < kPlanBins; i += blockDim.x) bins[i] = 0;
+    __syncthreads();
+    auto bin_of = [&](int c) {
+        const int blk = c / pairs_per_block, pair = c - blk * pairs_per_block;
+        int pl = prefix_len[blk];
+        if (pl < 0 || pl > prefix_total) {
+            report(status, PULSAR_DEV_BAD_LENGTH);
+            pl = max(0, min(pl, prefix_total));
+        }
+        const int cost = 2 * ((pl + 127) / 128) + 4 * pair + 3;
+        return kPlanBins - 1 - min(cost, kPlanBins - 1);        // costliest first
+    };
+    for (int c = threadIdx.x; c < n_combos; c += blockDim.x) atomicAdd(&bins[bin_of(c)], 1);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int run = 0;
+        for (int i = 0; i < kPlanBins; ++i) { const int n = bins[i]; bins[i] = run; run += n; }
+    }
+    __syncthreads();
+    for (int c = threadIdx.x; c < n_combos; c += blockDim.x) order[atomicAdd(&bins[bin_of(c)], 1)] = c;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Attention kernel: persistent, warp-specialised.
+//
+//   warps 0-3   softmax of query tile 0 (one thread per query row, TMEM lane = row)
+//   warps 4-7   softmax of query tile 1
+//   warp  8     MMA issuer (one elected lane): S_s = Q_s K^T, O_s += P_s V
+//   warp  9     TMA loader (one elected lane): Q tiles and the K/V ring
+//
+// A work item is two 128-row query tiles sharing one list of 128-key tiles.  The two tiles
+// ping-pong on the tensor pipe: while the softmax warpgroup of one tile works on S, the pipe
+// runs the other tile's PV and next S.  TMEM: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512);
+// P_s (bf16 pairs) overwrites the first 64 columns of S_s.  The running maximum is only moved
+// when it grows by more than 2^8 (the stale maximum is used consistently for P, O and the row
+// sum, so the result is unchanged); the rare rescale of O is done by the softmax warpgroup.
+// ---------------------------------------------------------------------------------------------
+constexpr int kStages = 5;
+constexpr int kAttnThreads = 320;
+constexpr int kMmaWarp = 8;
+constexpr int kLoadWarp = 9;
+constexpr float kRescaleThreshold = 8.0f;      // in log2 units
+
 template <int D>
 struct SmemLayout {
     static constexpr int kPanels = D / 64;
     static constexpr int kTileBytes = kPanels * kPanelBytes;
-    static constexpr int kQ = 0;
-    static constexpr int kK = kTileBytes;
-    static constexpr int kV = 2 * kTileBytes;
-    static constexpr int kBars = 3 * kTileBytes;      // 4 mbarriers
-    static constexpr int kTmemPtr = kBars + 4 * 8;
+    static constexpr int kQ = 0;                                   // 2 query tiles
+    static constexpr int kKV = 2 * kTileBytes;                     // kStages key/value tiles
+    static constexpr int kBars = kKV + kStages * kTileBytes;
+    // barrier indices
+    static constexpr int bQFull = 0, bQEmpty = 2, bSFull = 4, bPFull = 6, bOFull = 8, bOEmpty = 10;
+    static constexpr int bKvFull = 12, bKvEmpty = 12 + kStages, kNumBars = 12 + 2 * kStages;
+    static constexpr int kTmemPtr = kBars + kNumBars * 8;
     static constexpr int kAbort = kTmemPtr + 4;
     static constexpr int kTotal = kAbort + 4;
-    static constexpr int kDynBytes = kTotal + 1024;   // room to align the base to 1024 bytes
+    static constexpr int kDynBytes = kTotal + 1024;                // room to align the base to 1024 bytes
 };
 
-struct KvTile {
-    int from_prefix;   // 1: gathered prefix buffer, 0: K/V themselves
-    int row0;          // first key row of the tile in that tensor
-    int valid;         // keys of the tile that exist for this work item (<= 128)
-    int causal_base;   // >= 0: key c is visible to row r iff causal_base + c <= r_in_block; < 0: no causal mask
+// What one work item covers; every role decodes it the same way.
+struct Item {
+    int token0_a, token0_b;      // first token of each query tile
+    int head0, kvh, part;
+    int has1;                    // second query tile exists
+    int n_tiles_a, n_tiles_b;    // key tiles each query tile walks
+    int n_load;                  // key tiles to stage = max of the two
+    int n_pref_tiles, pref_len;
+    int main_row0, main_len;
+    int row0_a, row0_b;          // first row of each query tile within its block (phase 1)
 };
+
+__device__ __forceinline__ void decode_item(const AttnArgs& a, int idx, Item& it) {
+    if (a.mode == kModePhase1) {
+        const int combo = a.order[idx / a.Hq];
+        it.head0 = idx - (idx / a.Hq) * a.Hq;
+        it.kvh = it.head0 / a.g;
+        it.part = 0;
+        const int blk = combo / a.pairs, pair = combo - blk * a.pairs;
+        const int qt0 = 2 * pair;
+        it.has1 = (qt0 + 1 < a.tiles_per_block) ? 1 : 0;
+        it.row0_a = qt0 * kTileM;
+        it.row0_b = (qt0 + 1) * kTileM;
+        it.token0_a = blk * a.block_size + it.row0_a;
+        it.token0_b = blk * a.block_size + it.row0_b;
+        int pl = a.prefix_len[blk];
+        pl = max(0, min(pl, a.prefix_total));
+        it.pref_len = pl;
+        it.n_pref_tiles = (pl + kTileN - 1) / kTileN;
+        it.main_row0 = blk * a.block_size;
+        it.main_len = a.block_size;
+        it.n_tiles_a = it.n_pref_tiles + qt0 + 1;
+        it.n_tiles_b = it.has1 ? it.n_pref_tiles + qt0 + 2 : 0;
+    } else {
+        const int rp = idx % a.pairs;
+        const int rest = idx / a.pairs;
+        it.kvh = rest % a.Hkv;
+        it.part = rest / a.Hkv;
+        it.head0 = it.kvh * a.g;
+        const int tokens_per_tile = kTileM / a.pack;
+        it.token0_a = (2 * rp) * tokens_per_tile;
+        it.token0_b = (2 * rp + 1) * tokens_per_tile;
+        it.has1 = (it.token0_b < a.n_tokens) ? 1 : 0;
+        it.row0_a = it.row0_b = 0;
+        it.pref_len = 0;
+        it.n_pref_tiles = 0;
+        it.main_row0 = it.part * a.split_len;
+        it.main_len = a.split_len;
+        const int n = (a.split_len + kTileN - 1) / kTileN;
+        it.n_tiles_a = n;
+        it.n_tiles_b = it.has1 ? n : 0;
+    }
+    it.n_load = max(it.n_tiles_a, it.n_tiles_b);
+}
 
 template <int D>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(kAttnThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
             const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmKp,
             const __grid_constant__ CUtensorMap tmVp, const AttnArgs a) {
@@ -108,242 +214,349 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sQ = smem + SL::kQ;
-    uint8_t* sK = smem + SL::kK;
-    uint8_t* sV = smem + SL::kV;
+    uint8_t* sKV = smem + SL::kKV;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::kBars);
-    uint64_t* bar_q = bars + 0;
-    uint64_t* bar_kv = bars + 1;
-    uint64_t* bar_s = bars + 2;
-    uint64_t* bar_o = bars + 3;
     uint32_t* tmem_ptr = reinterpret_cast<uint32_t*>(smem + SL::kTmemPtr);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SL::kAbort);
 
-    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    // ---- work item ---------------------------------------------------------------------
-    int token0, head0, kvh, part = 0;
-    int n_pref_tiles = 0, pref_len = 0, n_main_tiles, main_row0, main_len, row0_in_block = 0;
-    if (a.mode == kModePhase1) {
-        const int blk = blockIdx.x / a.tiles_per_block, qt = blockIdx.x - blk * a.tiles_per_block;
-        row0_in_block = qt * kTileM;
-        token0 = blk * a.block_size + row0_in_block;
-        head0 = blockIdx.y;
-        kvh = head0 / a.g;
-        pref_len = a.prefix_len[blk];
-        if (pref_len < 0 || pref_len > a.prefix_total) {
-            if (tid == 0) report(a.status, PULSAR_DEV_BAD_LENGTH);
-            pref_len = max(0, min(pref_len, a.prefix_total));
-        }
-        n_pref_tiles = (pref_len + kTileN - 1) / kTileN;
-        n_main_tiles = qt + 1;
-        main_row0 = blk * a.block_size;
-        main_len = a.block_size;
-    } else {
-        token0 = blockIdx.x * (kTileM / a.pack);
-        kvh = blockIdx.y;
-        head0 = kvh * a.g;
-        part = blockIdx.z;
-        main_row0 = part * a.split_len;
-        main_len = a.split_len;
-        n_main_tiles = (a.split_len + kTileN - 1) / kTileN;
-    }
-    const int n_tiles = n_pref_tiles + n_main_tiles;
-
-    // ---- set-up --------------------------------------------------------------------------
     if (tid == 0) {
         *abort_flag = 0;
-        mbar_init(bar_q, 1);
-        mbar_init(bar_kv, 1);
-        mbar_init(bar_s, 1);
-        mbar_init(bar_o, 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bars + SL::bQFull + s, 1);
+            mbar_init(bars + SL::bQEmpty + s, 1);
+            mbar_init(bars + SL::bSFull + s, 1);
+            mbar_init(bars + SL::bPFull + s, 4);
+            mbar_init(bars + SL::bOFull + s, 1);
+            mbar_init(bars + SL::bOEmpty + s, 4);
+        }
+        for (int i = 0; i < kStages; ++i) {
+            mbar_init(bars + SL::bKvFull + i, 1);
+            mbar_init(bars + SL::bKvEmpty + i, 1);
+        }
         mbar_fence_init();
+    }
+    if (warp == kLoadWarp && lane == 0) {
         tma_prefetch_desc(&tmQ);
         tma_prefetch_desc(&tmK);
         tma_prefetch_desc(&tmV);
+        tma_prefetch_desc(&tmKp);
+        tma_prefetch_desc(&tmVp);
     }
-    if (warp == 0) {
-        tmem_alloc(tmem_ptr, 256);
+    if (warp == kMmaWarp) {
+        tmem_alloc(tmem_ptr, 512);
         tmem_relinquish();
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr;
-    const uint32_t tS = tmem_base;              // S: columns [0,128); P (bf16 pairs) reuses [0,64)
-    const uint32_t tO = tmem_base + 128;        // O: columns [128, 128+D)
-    const uint32_t lane_sel = static_cast<uint32_t>(warp * 32) << 16;
 
-    constexpr uint32_t kIdescQK = umma_idesc_bf16(kTileM, kTileN, false, false);
-    constexpr uint32_t kIdescPV = umma_idesc_bf16(kTileM, D, false, true);
-
-    if (tid == 0) {
-        mbar_expect_tx(bar_q, SL::kTileBytes);
-        for (int p = 0; p < SL::kPanels; ++p)
-            tma_load_3d(sQ + p * kPanelBytes, &tmQ, bar_q, p * 64, head0, token0);
-    }
-
-    float m_run = -INFINITY, l_run = 0.f;
-    const int my_row_in_block = row0_in_block + tid;    // phase 1 only
-    bool ok = true;
-
-    for (int t = 0; t < n_tiles; ++t) {
-        // ---- which keys ----------------------------------------------------------------
-        KvTile kt;
-        if (t < n_pref_tiles) {
-            kt.from_prefix = 1;
-            kt.row0 = t * kTileN;
-            kt.valid = min(kTileN, pref_len - kt.row0);
-            kt.causal_base = -1;
-        } else {
-            const int j = t - n_pref_tiles;
-            kt.from_prefix = 0;
-            kt.row0 = main_row0 + j * kTileN;
-            kt.valid = min(kTileN, main_len - j * kTileN);
-            kt.causal_base = (a.mode == kModePhase1 && j == n_main_tiles - 1) ? j * kTileN : -1;
-        }
-
-        // ---- load K and V tiles ----------------------------------------------------------
-        if (tid == 0 && ok) {
-            mbar_expect_tx(bar_kv, 2 * SL::kTileBytes);
-            const CUtensorMap* mk = kt.from_prefix ? &tmKp : &tmK;
-            const CUtensorMap* mv = kt.from_prefix ? &tmVp : &tmV;
-            for (int p = 0; p < SL::kPanels; ++p) {
-                tma_load_2d(sK + p * kPanelBytes, mk, bar_kv, kvh * D + p * 64, kt.row0);
-                tma_load_2d(sV + p * kPanelBytes, mv, bar_kv, kvh * D + p * 64, kt.row0);
-            }
-        }
-        if (t == 0) ok = ok && mbar_wait(bar_q, 0, abort_flag, a.status);
-        ok = ok && mbar_wait(bar_kv, t & 1, abort_flag, a.status);
-
-        // ---- S = Q K^T --------------------------------------------------------------------
-        if (tid == 0 && ok) {
-            tc_fence_after();
+    if (warp == kLoadWarp) {
+        // =============================== TMA loader ===============================
+        if (lane == 0) {
+            uint32_t ring = 0;                 // key/value tiles staged so far (ring position)
+            uint32_t q_use[2] = {0, 0};
+            bool ok = true;
+            auto stage_kv = [&](const CUtensorMap* tm, int x, int y) {
+                const uint32_t slot = ring % kStages, par = (ring / kStages) & 1;
+                ok = ok && mbar_wait(bars + SL::bKvEmpty + slot, par ^ 1, abort_flag, a.status);
+                if (!ok) return;
+                uint64_t* full = bars + SL::bKvFull + slot;
+                mbar_expect_tx(full, SL::kTileBytes);
+                uint8_t* dst = sKV + slot * SL::kTileBytes;
 #pragma unroll
-            for (int kk = 0; kk < D / 16; ++kk) {
-                const uint32_t off = (kk >> 2) * kPanelBytes + (kk & 3) * 32;
-                const uint64_t da = umma_smem_desc_sw128(smem_u32(sQ) + off, 16, 1024);
-                const uint64_t db = umma_smem_desc_sw128(smem_u32(sK) + off, 16, 1024);
-                umma_ss(tS, da, db, kIdescQK, kk > 0 ? 1u : 0u);
-            }
-            umma_commit(bar_s);
-        }
-        ok = ok && mbar_wait(bar_s, t & 1, abort_flag, a.status);
-        tc_fence_after();
-
-        // ---- softmax on this thread's row -------------------------------------------------
-        // visible key columns of the tile for this row: [0, n_vis)
-        int n_vis = kt.valid;
-        if (kt.causal_base >= 0) n_vis = min(n_vis, my_row_in_block - kt.causal_base + 1);
-
-        float m_tile = -INFINITY;
+                for (int p = 0; p < SL::kPanels; ++p) tma_load_2d(dst + p * kPanelBytes, tm, full, x + p * 64, y);
+                ++ring;
+            };
+            auto stage_q = [&](int s, const Item& it) {
+                ok = ok && mbar_wait(bars + SL::bQEmpty + s, (q_use[s] & 1) ^ 1, abort_flag, a.status);
+                if (!ok) return;
+                uint64_t* full = bars + SL::bQFull + s;
+                mbar_expect_tx(full, SL::kTileBytes);
+                uint8_t* dst = sQ + s * SL::kTileBytes;
 #pragma unroll
-        for (int c0 = 0; c0 < kTileN; c0 += 32) {
-            uint32_t r[32];
-            tmem_ld32(tS + lane_sel + c0, r);
-            tmem_wait_ld();
-#pragma unroll
-            for (int c = 0; c < 32; ++c)
-                if (c0 + c < n_vis) m_tile = fmaxf(m_tile, __uint_as_float(r[c]));
-        }
-        const float m_new = fmaxf(m_run, m_tile * a.scale_log2);
-        const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-        const float alpha = ex2(m_run - m_use);          // 0 on the first tile (m_run = -inf)
-        float l_tile = 0.f;
-#pragma unroll
-        for (int c0 = 0; c0 < kTileN; c0 += 32) {
-            uint32_t r[32];
-            tmem_ld32(tS + lane_sel + c0, r);
-            tmem_wait_ld();
-            uint32_t pk[16];
-#pragma unroll
-            for (int c = 0; c < 32; c += 2) {
-                float p0 = (c0 + c < n_vis) ? ex2(fmaf(__uint_as_float(r[c]), a.scale_log2, -m_use)) : 0.f;
-                float p1 = (c0 + c + 1 < n_vis) ? ex2(fmaf(__uint_as_float(r[c + 1]), a.scale_log2, -m_use)) : 0.f;
-                l_tile += p0 + p1;
-                pk[c >> 1] = pack_bf16x2(p0, p1);
-            }
-            tmem_st16(tS + lane_sel + (c0 >> 1), pk);     // P column c/2 holds keys c, c+1
-        }
-        l_run = l_run * alpha + l_tile;
-        m_run = m_new;
-
-        // ---- rescale the running output ------------------------------------------------------
-        if (t > 0) {
-#pragma unroll
-            for (int c0 = 0; c0 < D; c0 += 32) {
-                uint32_t r[32];
-                tmem_ld32(tO + lane_sel + c0, r);
-                tmem_wait_ld();
-#pragma unroll
-                for (int c = 0; c < 32; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * alpha);
-                tmem_st32(tO + lane_sel + c0, r);
-            }
-        }
-        tmem_wait_st();
-        tc_fence_before();
-        __syncthreads();
-        ok = ok && (*abort_flag == 0);
-
-        // ---- O += P V -----------------------------------------------------------------------
-        if (tid == 0 && ok) {
-            tc_fence_after();
-#pragma unroll
-            for (int kk = 0; kk < kTileN / 16; ++kk) {
-                const uint64_t db = umma_smem_desc_sw128(smem_u32(sV) + kk * 2048, kPanelBytes, 1024);
-                umma_ts(tO, tS + kk * 8, db, kIdescPV, (t > 0 || kk > 0) ? 1u : 0u);
-            }
-            umma_commit(bar_o);
-        }
-        ok = ok && mbar_wait(bar_o, t & 1, abort_flag, a.status);
-        tc_fence_after();
-        // After a failed wait the loop keeps its shape (barriers and warp-collective TMEM
-        // accesses stay convergent) but issues no further copies or MMAs and stores nothing.
-    }
-
-    // ---- epilogue: normalise and store this thread's row ---------------------------------------
-    {
-        const int token = token0 + tid / a.pack;
-        const int head = head0 + tid % a.pack;
-        bool store = ok && token < a.n_tokens;
-        if (a.mode == kModePhase1) store = store && my_row_in_block < a.block_size;
-        const float inv_l = l_run > 0.f ? 1.f / l_run : 0.f;
-        const float lse = (l_run > 0.f) ? (m_run + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
-        const size_t row = static_cast<size_t>(token) * a.Hq + head;
-#pragma unroll
-        for (int c0 = 0; c0 < D; c0 += 32) {
-            uint32_t r[32];
-            tmem_ld32(tO + lane_sel + c0, r);      // every thread of the warp takes part in the load
-            tmem_wait_ld();
-            if (!store) continue;
-            if (a.part_O != nullptr) {
-                float4* dst = reinterpret_cast<float4*>(
-                    a.part_O + (static_cast<size_t>(part) * a.n_tokens * a.Hq + row) * D + c0);
-#pragma unroll
-                for (int c = 0; c < 32; c += 4)
-                    dst[c >> 2] = make_float4(__uint_as_float(r[c]) * inv_l, __uint_as_float(r[c + 1]) * inv_l,
-                                              __uint_as_float(r[c + 2]) * inv_l, __uint_as_float(r[c + 3]) * inv_l);
-            } else {
-                uint4* dst = reinterpret_cast<uint4*>(a.O + row * D + c0);
-#pragma unroll
-                for (int c = 0; c < 32; c += 8) {
-                    uint4 v;
-                    v.x = pack_bf16x2(__uint_as_float(r[c]) * inv_l, __uint_as_float(r[c + 1]) * inv_l);
-                    v.y = pack_bf16x2(__uint_as_float(r[c + 2]) * inv_l, __uint_as_float(r[c + 3]) * inv_l);
-                    v.z = pack_bf16x2(__uint_as_float(r[c + 4]) * inv_l, __uint_as_float(r[c + 5]) * inv_l);
-                    v.w = pack_bf16x2(__uint_as_float(r[c + 6]) * inv_l, __uint_as_float(r[c + 7]) * inv_l);
-                    dst[c >> 3] = v;
+                for (int p = 0; p < SL::kPanels; ++p)
+                    tma_load_3d(dst + p * kPanelBytes, &tmQ, full, p * 64, it.head0, s ? it.token0_b : it.token0_a);
+                ++q_use[s];
+            };
+            for (int idx = blockIdx.x; idx < a.n_items && ok; idx += gridDim.x) {
+                Item it;
+                decode_item(a, idx, it);
+                stage_q(0, it);
+                for (int t = 0; t < it.n_load && ok; ++t) {
+                    const bool pref = t < it.n_pref_tiles;
+                    const int row = pref ? t * kTileN : it.main_row0 + (t - it.n_pref_tiles) * kTileN;
+                    stage_kv(pref ? &tmKp : &tmK, it.kvh * D, row);
+                    if (t == 0 && it.has1) stage_q(1, it);
+                    stage_kv(pref ? &tmVp : &tmV, it.kvh * D, row);
                 }
             }
         }
-        if (store) {
-            if (a.part_O != nullptr) a.part_LSE[static_cast<size_t>(part) * a.n_tokens * a.Hq + row] = lse;
-            else if (a.LSE != nullptr) a.LSE[row] = lse;
+        __syncwarp();
+    } else if (warp == kMmaWarp) {
+        // =============================== MMA issuer ===============================
+        if (lane == 0) {
+            constexpr uint32_t kIdescQK = umma_idesc_bf16(kTileM, kTileN, false, false);
+            constexpr uint32_t kIdescPV = umma_idesc_bf16(kTileM, D, false, true);
+            uint32_t ring = 0;
+            uint32_t q_use[2] = {0, 0}, p_cnt[2] = {0, 0}, o_use[2] = {0, 0};
+            bool ok = true;
+            auto wait_kv = [&](uint32_t n) {
+                ok = ok && mbar_wait(bars + SL::bKvFull + n % kStages, (n / kStages) & 1, abort_flag, a.status);
+                tc_fence_after();
+            };
+            auto release_kv = [&](uint32_t n) { umma_commit(bars + SL::bKvEmpty + n % kStages); };
+            auto issue_s = [&](int s, uint32_t n) {           // S_s = Q_s K^T, K in ring position n
+                const uint32_t qa = smem_u32(sQ + s * SL::kTileBytes);
+                const uint32_t ka = smem_u32(sKV + (n % kStages) * SL::kTileBytes);
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk >> 2) * kPanelBytes + (kk & 3) * 32;
+                    umma_ss(tmem_base + s * 128, umma_smem_desc_sw128(qa + off, 16, 1024),
+                            umma_smem_desc_sw128(ka + off, 16, 1024), kIdescQK, kk > 0 ? 1u : 0u);
+                }
+                umma_commit(bars + SL::bSFull + s);
+            };
+            auto issue_pv = [&](int s, uint32_t n, bool accumulate) {   // O_s (+)= P_s V, V in ring position n
+                const uint32_t va = smem_u32(sKV + (n % kStages) * SL::kTileBytes);
+#pragma unroll
+                for (int kk = 0; kk < kTileN / 16; ++kk)
+                    umma_ts(tmem_base + 256 + s * 128, tmem_base + s * 128 + kk * 8,
+                            umma_smem_desc_sw128(va + kk * 2048, kPanelBytes, 1024), kIdescPV,
+                            (accumulate || kk > 0) ? 1u : 0u);
+            };
+            auto wait_p = [&](int s) {
+                ok = ok && mbar_wait(bars + SL::bPFull + s, p_cnt[s] & 1, abort_flag, a.status);
+                ++p_cnt[s];
+                tc_fence_after();
+            };
+            for (int idx = blockIdx.x; idx < a.n_items && ok; idx += gridDim.x) {
+                Item it;
+                decode_item(a, idx, it);
+                const int n0 = it.n_tiles_a, n1 = it.n_tiles_b;
+                const uint32_t base = ring;                   // K_t at base + 2t, V_t at base + 2t + 1
+                ok = ok && mbar_wait(bars + SL::bQFull + 0, q_use[0] & 1, abort_flag, a.status);
+                ++q_use[0];
+                wait_kv(base);
+                if (!ok) break;
+                issue_s(0, base);
+                if (it.has1) {
+                    ok = ok && mbar_wait(bars + SL::bQFull + 1, q_use[1] & 1, abort_flag, a.status);
+                    ++q_use[1];
+                    tc_fence_after();
+                    if (!ok) break;
+                    issue_s(1, base);
+                }
+                release_kv(base);
+                for (int t = 0; t < it.n_load && ok; ++t) {
+                    const uint32_t nv = base + 2 * t + 1, nk = base + 2 * t + 2;
+                    wait_kv(nv);
+                    if (t < n0) {
+                        if (t == 0) {
+                            ok = ok && mbar_wait(bars + SL::bOEmpty + 0, (o_use[0] & 1) ^ 1, abort_flag, a.status);
+                            ++o_use[0];
+                        }
+                        wait_p(0);
+                        if (!ok) break;
+                        issue_pv(0, nv, t > 0);
+                        if (t == n0 - 1) {
+                            umma_commit(bars + SL::bOFull + 0);
+                            umma_commit(bars + SL::bQEmpty + 0);
+                        }
+                    }
+                    const bool more = t + 1 < it.n_load;
+                    if (more) wait_kv(nk);
+                    if (!ok) break;
+                    if (t + 1 < n0) issue_s(0, nk);
+                    if (t < n1) {
+                        if (t == 0) {
+                            ok = ok && mbar_wait(bars + SL::bOEmpty + 1, (o_use[1] & 1) ^ 1, abort_flag, a.status);
+                            ++o_use[1];
+                        }
+                        wait_p(1);
+                        if (!ok) break;
+                        issue_pv(1, nv, t > 0);
+                        if (t == n1 - 1) {
+                            umma_commit(bars + SL::bOFull + 1);
+                            umma_commit(bars + SL::bQEmpty + 1);
+                        }
+                    }
+                    release_kv(nv);
+                    if (more) {
+                        if (t + 1 < n1) issue_s(1, nk);
+                        release_kv(nk);
+                    }
+                }
+                ring = base + 2 * it.n_load;
+            }
+        }
+        __syncwarp();
+    } else {
+        // =============================== softmax warpgroups ===============================
+        const int s = warp >> 2;                               // query tile of this warpgroup
+        const int row = (warp & 3) * 32 + lane;                // row of the tile = TMEM lane
+        const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem_base + s * 128 + lane_sel;
+        const uint32_t tO = tmem_base + 256 + s * 128 + lane_sel;
+        uint64_t* bar_s = bars + SL::bSFull + s;
+        uint64_t* bar_p = bars + SL::bPFull + s;
+        uint64_t* bar_of = bars + SL::bOFull + s;
+        uint64_t* bar_oe = bars + SL::bOEmpty + s;
+        uint32_t s_cnt = 0, o_cnt = 0;
+        bool ok = true;
+
+        for (int idx = blockIdx.x; idx < a.n_items && ok; idx += gridDim.x) {
+            Item it;
+            decode_item(a, idx, it);
+            const int n = s ? it.n_tiles_b : it.n_tiles_a;
+            if (n == 0) continue;
+            float m_used = -INFINITY, l_run = 0.f;
+            const int my_row_in_block = (s ? it.row0_b : it.row0_a) + row;
+
+            for (int t = 0; t < n; ++t) {
+                // visible key columns of this tile for this row: [0, n_vis)
+                int n_vis = kTileN;
+                bool masked = false;
+                if (t < it.n_pref_tiles) {
+                    const int valid = it.pref_len - t * kTileN;
+                    if (valid < kTileN) { n_vis = valid; masked = true; }
+                } else {
+                    const int j = t - it.n_pref_tiles;
+                    const int valid = it.main_len - j * kTileN;
+                    if (valid < kTileN) { n_vis = valid; masked = true; }
+                    if (a.mode == kModePhase1 && t == n - 1) {
+                        n_vis = min(n_vis, my_row_in_block - j * kTileN + 1);
+                        masked = true;
+                    }
+                }
+
+                ok = __all_sync(0xffffffffu, ok && mbar_wait(bar_s, s_cnt & 1, abort_flag, a.status));
+                ++s_cnt;
+                if (!ok) break;
+                tc_fence_after();
+
+                uint32_t r[kTileN];
+#pragma unroll
+                for (int c0 = 0; c0 < kTileN; c0 += 32) tmem_ld32(tS + c0, *reinterpret_cast<uint32_t(*)[32]>(&r[c0]));
+                tmem_wait_ld();
+
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+                if (masked) {
+#pragma unroll
+                    for (int c = 0; c < kTileN; ++c)
+                        if (c >= n_vis) r[c] = 0xff800000u;          // -inf
+                }
+#pragma unroll
+                for (int c = 0; c < kTileN; c += 4) {
+                    mx0 = fmaxf(mx0, __uint_as_float(r[c]));
+                    mx1 = fmaxf(mx1, __uint_as_float(r[c + 1]));
+                    mx2 = fmaxf(mx2, __uint_as_float(r[c + 2]));
+                    mx3 = fmaxf(mx3, __uint_as_float(r[c + 3]));
+                }
+                const float m_tile = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * a.scale_log2;
+
+                const bool need = m_tile > m_used + kRescaleThreshold;   // always true on the first tile
+                if (__any_sync(0xffffffffu, need)) {
+                    const float m_new = need ? m_tile : m_used;
+                    const float alpha = (m_new == -INFINITY) ? 1.f : ex2(m_used - m_new);
+                    l_run *= alpha;
+                    m_used = m_new;
+                    if (t > 0) {
+#pragma unroll
+                        for (int c0 = 0; c0 < D; c0 += 32) {
+                            uint32_t o[32];
+                            tmem_ld32(tO + c0, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                            tmem_st32(tO + c0, o);
+                        }
+                    }
+                }
+                const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
+
+                float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+#pragma unroll
+                for (int c0 = 0; c0 < kTileN; c0 += 32) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int c = 0; c < 32; c += 4) {
+                        const float p0 = ex2(fmaf(__uint_as_float(r[c0 + c]), a.scale_log2, neg_m));
+                        const float p1 = ex2(fmaf(__uint_as_float(r[c0 + c + 1]), a.scale_log2, neg_m));
+                        const float p2 = ex2(fmaf(__uint_as_float(r[c0 + c + 2]), a.scale_log2, neg_m));
+                        const float p3 = ex2(fmaf(__uint_as_float(r[c0 + c + 3]), a.scale_log2, neg_m));
+                        l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+                        pk[c >> 1] = pack_bf16x2(p0, p1);
+                        pk[(c >> 1) + 1] = pack_bf16x2(p2, p3);
+                    }
+                    tmem_st16(tS + (c0 >> 1), pk);                   // P column c/2 holds keys c, c+1
+                }
+                l_run += (l0 + l1) + (l2 + l3);
+
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_p);
+            }
+            if (!ok) break;
+
+            // ---- epilogue: normalise and store this thread's row ----
+            ok = __all_sync(0xffffffffu, ok && mbar_wait(bar_of, o_cnt & 1, abort_flag, a.status));
+            ++o_cnt;
+            if (!ok) break;
+            tc_fence_after();
+            {
+                const int token = (s ? it.token0_b : it.token0_a) + row / a.pack;
+                const int head = it.head0 + row % a.pack;
+                bool store = token < a.n_tokens;
+                if (a.mode == kModePhase1) store = store && my_row_in_block < a.block_size;
+                const float inv_l = l_run > 0.f ? 1.f / l_run : 0.f;
+                const float lse = (l_run > 0.f) ? (m_used + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+                const size_t orow = static_cast<size_t>(token) * a.Hq + head;
+#pragma unroll
+                for (int c0 = 0; c0 < D; c0 += 32) {
+                    uint32_t o[32];
+                    tmem_ld32(tO + c0, o);
+                    tmem_wait_ld();
+                    if (!store) continue;
+                    if (a.part_O != nullptr) {
+                        float4* dst = reinterpret_cast<float4*>(
+                            a.part_O + (static_cast<size_t>(it.part) * a.n_tokens * a.Hq + orow) * D + c0);
+#pragma unroll
+                        for (int c = 0; c < 32; c += 4)
+                            dst[c >> 2] = make_float4(__uint_as_float(o[c]) * inv_l, __uint_as_float(o[c + 1]) * inv_l,
+                                                      __uint_as_float(o[c + 2]) * inv_l, __uint_as_float(o[c + 3]) * inv_l);
+                    } else {
+                        uint4* dst = reinterpret_cast<uint4*>(a.O + orow * D + c0);
+#pragma unroll
+                        for (int c = 0; c < 32; c += 8) {
+                            uint4 v;
+                            v.x = pack_bf16x2(__uint_as_float(o[c]) * inv_l, __uint_as_float(o[c + 1]) * inv_l);
+                            v.y = pack_bf16x2(__uint_as_float(o[c + 2]) * inv_l, __uint_as_float(o[c + 3]) * inv_l);
+                            v.z = pack_bf16x2(__uint_as_float(o[c + 4]) * inv_l, __uint_as_float(o[c + 5]) * inv_l);
+                            v.w = pack_bf16x2(__uint_as_float(o[c + 6]) * inv_l, __uint_as_float(o[c + 7]) * inv_l);
+                            dst[c >> 3] = v;
+                        }
+                    }
+                }
+                if (store) {
+                    if (a.part_O != nullptr)
+                        a.part_LSE[static_cast<size_t>(it.part) * a.n_tokens * a.Hq + orow] = lse;
+                    else if (a.LSE != nullptr)
+                        a.LSE[orow] = lse;
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_oe);
         }
     }
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem_base, 256);
+    if (warp == kMmaWarp) tmem_dealloc(tmem_base, 512);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -396,22 +609,24 @@ bool make_map_2d(CUtensorMap* m, const void* base, int64_t rows, int64_t width) 
 
 template <int D>
 int32_t launch_attn(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& v, const CUtensorMap& kp,
-                    const CUtensorMap& vp, const AttnArgs& a, dim3 grid, cudaStream_t stream) {
+                    const CUtensorMap& vp, const AttnArgs& a, cudaStream_t stream) {
     constexpr int smem = SmemLayout<D>::kDynBytes;
     static bool configured = false;
     if (!configured) {
         PULSAR_CUDA_OK(cudaFuncSetAttribute(attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         configured = true;
     }
-    attn_kernel<D><<<grid, 128, smem, stream>>>(q, k, v, kp, vp, a);
+    const int grid = a.n_items < sm_count() ? a.n_items : sm_count();     // one persistent CTA per SM
+    if (grid <= 0) return PULSAR_OK;
+    attn_kernel<D><<<grid, kAttnThreads, smem, stream>>>(q, k, v, kp, vp, a);
     PULSAR_CUDA_OK(cudaGetLastError());
     count_launch();
     return PULSAR_OK;
 }
 
 struct Phase1Plan {
-    int n_blocks, tiles_per_block;
-    size_t pref_rows, pref_bytes, total;
+    int n_blocks, tiles_per_block, pairs_per_block;
+    size_t pref_rows, pref_bytes, order_bytes, total;
 };
 
 int32_t plan_phase1(int64_t L, int32_t Hq, int32_t Hkv, int32_t d, int32_t block_size, int32_t prefix_total,
@@ -419,18 +634,22 @@ int32_t plan_phase1(int64_t L, int32_t Hq, int32_t Hkv, int32_t d, int32_t block
     if (L <= 0 || Hq <= 0 || Hkv <= 0 || block_size <= 0 || prefix_total < 0) return PULSAR_ERR_INVALID_ARG;
     if ((d != 64 && d != 128) || Hq % Hkv != 0 || L % block_size != 0 || L >= (1ll << 31)) return PULSAR_ERR_SHAPE;
     if (L / block_size > 65535 || Hq > 65535) return PULSAR_ERR_SHAPE;
+    if (prefix_total > (1 << 30)) return PULSAR_ERR_SHAPE;
     p.n_blocks = static_cast<int>(L / block_size);
     p.tiles_per_block = (block_size + kTileM - 1) / kTileM;
     p.pref_rows = static_cast<size_t>(prefix_total > 0 ? prefix_total : 1);
+    p.pairs_per_block = (p.tiles_per_block + 1) / 2;
     p.pref_bytes = round_up(p.pref_rows * Hkv * d * 2, 256);
-    p.total = 2 * p.pref_bytes;
+    p.order_bytes = round_up(static_cast<size_t>(p.n_blocks) * p.pairs_per_block * 4, 256);
+    p.total = 2 * p.pref_bytes + p.order_bytes;
+    if (static_cast<int64_t>(p.n_blocks) * p.pairs_per_block * Hq >= (1ll << 31)) return PULSAR_ERR_SHAPE;
     return PULSAR_OK;
 }
 
 int32_t choose_splits(int32_t nq, int64_t L, int32_t Hq, int32_t Hkv) {
     const int g = Hq / Hkv;
     const int64_t row_tiles = (static_cast<int64_t>(nq) * g + kTileM - 1) / kTileM;
-    const int64_t items = row_tiles * Hkv;
+    const int64_t items = (row_tiles + 1) / 2 * Hkv;               // a work item is a pair of row tiles
     const int64_t want = 2ll * sm_count();
     if (L % kTileN != 0) return 1;
     const int64_t kv_tiles = L / kTileN;
@@ -480,6 +699,7 @@ extern "C" int32_t pulsar_phase1_attn(const uint16_t* Q, const uint16_t* K, cons
 
     uint16_t* Kp = static_cast<uint16_t*>(workspace);
     uint16_t* Vp = reinterpret_cast<uint16_t*>(static_cast<char*>(workspace) + p.pref_bytes);
+    int32_t* order = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + 2 * p.pref_bytes);
 
     CUtensorMap tmQ, tmK, tmV, tmKp, tmVp;
     if (!make_map_3d(&tmQ, Q, L, Hq, d, 1, kTileM) || !make_map_2d(&tmK, K, L, static_cast<int64_t>(Hkv) * d) ||
@@ -497,8 +717,17 @@ extern "C" int32_t pulsar_phase1_attn(const uint16_t* Q, const uint16_t* K, cons
         count_launch();
     }
 
+    phase1_plan_kernel<<<1, 256, 0, stream>>>(prefix_len, p.n_blocks, p.pairs_per_block, prefix_total, order,
+                                              device_status);
+    PULSAR_CUDA_OK(cudaGetLastError());
+    count_launch();
+
     AttnArgs a{};
     a.mode = kModePhase1;
+    a.Hkv = Hkv;
+    a.pairs = p.pairs_per_block;
+    a.n_items = p.n_blocks * p.pairs_per_block * Hq;
+    a.order = order;
     a.n_tokens = static_cast<int>(L);
     a.Hq = Hq;
     a.g = Hq / Hkv;
@@ -511,9 +740,8 @@ extern "C" int32_t pulsar_phase1_attn(const uint16_t* Q, const uint16_t* K, cons
     a.O = O;
     a.LSE = LSE;
     a.status = device_status;
-    dim3 grid(static_cast<unsigned>(p.tiles_per_block) * p.n_blocks, Hq, 1);
-    rc = d == 128 ? launch_attn<128>(tmQ, tmK, tmV, tmKp, tmVp, a, grid, stream)
-                  : launch_attn<64>(tmQ, tmK, tmV, tmKp, tmVp, a, grid, stream);
+    rc = d == 128 ? launch_attn<128>(tmQ, tmK, tmV, tmKp, tmVp, a, stream)
+                  : launch_attn<64>(tmQ, tmK, tmV, tmKp, tmVp, a, stream);
     if (rc != PULSAR_OK) return rc;
 
     if (K_ret) {
@@ -607,9 +835,12 @@ extern "C" int32_t pulsar_phase2_attn(const uint16_t* Qq, int32_t nq, const uint
     a.part_LSE = partial_out ? pL : nullptr;
     a.status = device_status;
     const int tokens_per_tile = kTileM / g;
-    dim3 grid((nq + tokens_per_tile - 1) / tokens_per_tile, Hkv, n_splits);
-    rc = d == 128 ? launch_attn<128>(tmQ, tmK, tmV, tmK, tmV, a, grid, stream)
-                  : launch_attn<64>(tmQ, tmK, tmV, tmK, tmV, a, grid, stream);
+    const int row_tiles = (nq + tokens_per_tile - 1) / tokens_per_tile;
+    a.Hkv = Hkv;
+    a.pairs = (row_tiles + 1) / 2;
+    a.n_items = a.pairs * Hkv * n_splits;
+    rc = d == 128 ? launch_attn<128>(tmQ, tmK, tmV, tmK, tmV, a, stream)
+                  : launch_attn<64>(tmQ, tmK, tmV, tmK, tmV, a, stream);
     if (rc != PULSAR_OK) return rc;
     if (partial_out)
         return launch_lse_merge(pO, pL, n_splits, static_cast<int64_t>(nq) * Hq, d, O, LSE, stream);
