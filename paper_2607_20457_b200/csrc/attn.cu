@@ -129,10 +129,16 @@ phase1_plan_kernel(const int32_t* __restrict__ prefix_len, int n_blocks, int pai
 // sum, so the result is unchanged); the rare rescale of O is done by the softmax warpgroup.
 // ---------------------------------------------------------------------------------------------
 constexpr int kStages = 5;
-constexpr int kAttnThreads = 320;
+constexpr int kAttnThreads = 384;             // warps 10 and 11 only take part in register hand-back
 constexpr int kMmaWarp = 8;
 constexpr int kLoadWarp = 9;
 constexpr float kRescaleThreshold = 8.0f;      // in log2 units
+// Registers per thread: the kernel is compiled for 168 (twelve warps).  setmaxnreg moves
+// registers inside the CTA's own pool of 12 * 168 per lane slot and acts on whole warpgroups:
+// warpgroup 2 (MMA issuer, TMA loader and two spare warps) hands back all but kRegsIssuer,
+// the eight softmax warps grow to kRegsSoftmax:  4 * 88 + 8 * 208 = 2016 = 12 * 168.
+constexpr int kRegsIssuer = 88;
+constexpr int kRegsSoftmax = 208;
 
 template <int D>
 struct SmemLayout {
@@ -253,6 +259,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr;
 
+    if (warp >= 8) reg_dealloc<kRegsIssuer>();
     if (warp == kLoadWarp) {
         // =============================== TMA loader ===============================
         if (lane == 0) {
@@ -393,8 +400,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             }
         }
         __syncwarp();
-    } else {
+    } else if (warp < 8) {
         // =============================== softmax warpgroups ===============================
+        reg_alloc<kRegsSoftmax>();
         const int s = warp >> 2;                               // query tile of this warpgroup
         const int row = (warp & 3) * 32 + lane;                // row of the tile = TMEM lane
         const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
@@ -438,8 +446,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 tc_fence_after();
 
                 uint32_t r[kTileN];
-#pragma unroll
-                for (int c0 = 0; c0 < kTileN; c0 += 32) tmem_ld32(tS + c0, *reinterpret_cast<uint32_t(*)[32]>(&r[c0]));
+                PULSAR_TMEM_LD32_AT(tS + 0, r, 0);
+                PULSAR_TMEM_LD32_AT(tS + 32, r, 32);
+                PULSAR_TMEM_LD32_AT(tS + 64, r, 64);
+                PULSAR_TMEM_LD32_AT(tS + 96, r, 96);
                 tmem_wait_ld();
 
                 float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;

@@ -258,6 +258,27 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         : "memory");
 }
 
+// Warp-level register reallocation (all lanes of the warp execute it; N a multiple of 8).
+template <int N>
+__device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N>
+__device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+
+// 32 consecutive columns into r[base .. base+32) of a larger register array.
+#define PULSAR_TMEM_LD32_AT(taddr, r, b)                                                                     \
+    asm volatile(                                                                                            \
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "                                                            \
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "                            \
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"            \
+        : "=r"(r[b + 0]), "=r"(r[b + 1]), "=r"(r[b + 2]), "=r"(r[b + 3]), "=r"(r[b + 4]), "=r"(r[b + 5]),    \
+          "=r"(r[b + 6]), "=r"(r[b + 7]), "=r"(r[b + 8]), "=r"(r[b + 9]), "=r"(r[b + 10]), "=r"(r[b + 11]),  \
+          "=r"(r[b + 12]), "=r"(r[b + 13]), "=r"(r[b + 14]), "=r"(r[b + 15]), "=r"(r[b + 16]),               \
+          "=r"(r[b + 17]), "=r"(r[b + 18]), "=r"(r[b + 19]), "=r"(r[b + 20]), "=r"(r[b + 21]),               \
+          "=r"(r[b + 22]), "=r"(r[b + 23]), "=r"(r[b + 24]), "=r"(r[b + 25]), "=r"(r[b + 26]),               \
+          "=r"(r[b + 27]), "=r"(r[b + 28]), "=r"(r[b + 29]), "=r"(r[b + 30]), "=r"(r[b + 31])                \
+        : "r"(taddr)                                                                                         \
+        : "memory")
+
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
