@@ -40,7 +40,8 @@ class PulsarError(RuntimeError):
 
 
 def library_path() -> str:
-    return _build.LIB
+    """Path of the CUDA library: the in-tree build, or $PULSAR_LIBRARY if set (a custom build)."""
+    return os.environ.get("PULSAR_LIBRARY") or _build.LIB
 
 
 def load_library(build_if_missing: bool = False):

@@ -118,8 +118,9 @@ phase1_plan_kernel(const int32_t* __restrict__ prefix_len, int n_blocks, int pai
 //
 //   warps 0-3   softmax of query tile 0 (one thread per query row, TMEM lane = row)
 //   warps 4-7   softmax of query tile 1
-//   warp  8     MMA issuer (one elected lane): S_s = Q_s K^T, O_s += P_s V
-//   warp  9     TMA loader (one elected lane): Q tiles and the K/V ring
+//   warp  8     MMA issuer of tile 0 (one lane): S_0 = Q_0 K^T, O_0 += P_0 V
+//   warp  9     TMA loader (one lane): Q tiles and the K/V ring
+//   warp  10    MMA issuer of tile 1
 //
 // A work item is two 128-row query tiles sharing one list of 128-key tiles.  The two tiles
 // ping-pong on the tensor pipe: while the softmax warpgroup of one tile works on S, the pipe
@@ -129,13 +130,23 @@ phase1_plan_kernel(const int32_t* __restrict__ prefix_len, int n_blocks, int pai
 // sum, so the result is unchanged); the rare rescale of O is done by the softmax warpgroup.
 // ---------------------------------------------------------------------------------------------
 constexpr int kStages = 5;
-constexpr int kAttnThreads = 384;             // warps 10 and 11 only take part in register hand-back
-constexpr int kMmaWarp = 8;
+constexpr int kAttnThreads = 384;             // warp 11 only takes part in the register hand-back
+constexpr int kMmaWarp = 8;    // issuer of query tile 0 (also owns the TMEM allocation)
 constexpr int kLoadWarp = 9;
+constexpr int kMmaWarp1 = 10;  // issuer of query tile 1
 constexpr float kRescaleThreshold = 8.0f;      // in log2 units
+// Tuning knobs (overridable at build time with -D).
+#ifndef PULSAR_POLY_PAIRS
+#define PULSAR_POLY_PAIRS 0
+#endif
+#ifndef PULSAR_SPECULATE
+#define PULSAR_SPECULATE 0
+#endif
+constexpr int kPolyPairs = PULSAR_POLY_PAIRS;  // of every four column pairs, how many use the polynomial exp2
+constexpr bool kSpeculate = PULSAR_SPECULATE;  // form P with the maximum in use while the tile maximum is computed
 // Registers per thread: the kernel is compiled for 168 (twelve warps).  setmaxnreg moves
 // registers inside the CTA's own pool of 12 * 168 per lane slot and acts on whole warpgroups:
-// warpgroup 2 (MMA issuer, TMA loader and two spare warps) hands back all but kRegsIssuer,
+// warpgroup 2 (the two MMA issuers, the TMA loader and a spare warp) hands back all but kRegsIssuer,
 // the eight softmax warps grow to kRegsSoftmax:  4 * 88 + 8 * 208 = 2016 = 12 * 168.
 constexpr int kRegsIssuer = 88;
 constexpr int kRegsSoftmax = 208;
@@ -211,6 +222,50 @@ __device__ __forceinline__ void decode_item(const AttnArgs& a, int idx, Item& it
     it.n_load = max(it.n_tiles_a, it.n_tiles_b);
 }
 
+// Row maximum of 128 raw logits (3-input max, four independent chains).
+__device__ __forceinline__ float row_max128(const uint32_t (&r)[kTileN]) {
+    float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < kTileN; c += 8) {
+        m0 = max3(m0, __uint_as_float(r[c]), __uint_as_float(r[c + 1]));
+        m1 = max3(m1, __uint_as_float(r[c + 2]), __uint_as_float(r[c + 3]));
+        m2 = max3(m2, __uint_as_float(r[c + 4]), __uint_as_float(r[c + 5]));
+        m3 = max3(m3, __uint_as_float(r[c + 6]), __uint_as_float(r[c + 7]));
+    }
+    return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+}
+
+// p_c = 2^(s_c * scale + neg_m) for the 128 logits of a row, rounded to bf16 pairs and written
+// to TMEM as the A operand of the PV product; returns the fp32 row sum.  kPoly of every four
+// column pairs take the polynomial exp2 (FMA pipe) instead of MUFU.  kPoly must be 0 when
+// logits may be -inf (masked tiles).
+template <int kPoly>
+__device__ __forceinline__ float exp_row128(const uint32_t (&r)[kTileN], float scale, float neg_m, uint32_t tP) {
+    float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+    const float2 sc = make_float2(scale, scale), nm = make_float2(neg_m, neg_m);
+#pragma unroll
+    for (int c0 = 0; c0 < kTileN; c0 += 32) {
+        uint32_t pk[16];
+#pragma unroll
+        for (int c = 0; c < 32; c += 2) {
+            const float2 x =
+                __ffma2_rn(make_float2(__uint_as_float(r[c0 + c]), __uint_as_float(r[c0 + c + 1])), sc, nm);
+            float2 pv;
+            if (((c >> 1) & 3) >= 4 - kPoly) {
+                pv = ex2_poly2(x);
+            } else {
+                pv.x = ex2(x.x);
+                pv.y = ex2(x.y);
+            }
+            if ((c >> 1) & 1) acc1 = __fadd2_rn(acc1, pv);
+            else acc0 = __fadd2_rn(acc0, pv);
+            pk[c >> 1] = pack_bf16x2(pv.x, pv.y);
+        }
+        tmem_st16(tP + (c0 >> 1), pk);                           // P column c/2 holds keys c, c+1
+    }
+    return (acc0.x + acc0.y) + (acc1.x + acc1.y);
+}
+
 template <int D>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -239,7 +294,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         }
         for (int i = 0; i < kStages; ++i) {
             mbar_init(bars + SL::bKvFull + i, 1);
-            mbar_init(bars + SL::bKvEmpty + i, 1);
+            mbar_init(bars + SL::bKvEmpty + i, 2);          // one arrival from each MMA issuer
         }
         mbar_fence_init();
     }
@@ -260,143 +315,182 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     const uint32_t tmem_base = *tmem_ptr;
 
     if (warp >= 8) reg_dealloc<kRegsIssuer>();
+    // Ring bookkeeping shared by the two issuer roles: `stage` walks 0..kStages-1, `phase`
+    // flips at every wrap.  Barrier i lives at bar0 + 8 * i.
+    const uint32_t bar0 = smem_u32(bars);
+#define PULSAR_RING_NEXT(stage, phase) \
+    do { if (++(stage) == kStages) { (stage) = 0; (phase) ^= 1u; } } while (0)
+
     if (warp == kLoadWarp) {
         // =============================== TMA loader ===============================
-        if (lane == 0) {
-            uint32_t ring = 0;                 // key/value tiles staged so far (ring position)
-            uint32_t q_use[2] = {0, 0};
+        // The whole warp walks the loops so that addresses, coordinates and barrier numbers stay
+        // warp-uniform (the copy and barrier instructions take uniform operands); one elected
+        // lane issues.
+        {
+            const bool leader = elect_one();
+            const uint32_t q_smem = smem_u32(sQ), kv_smem = smem_u32(sKV);
+            uint32_t stage = 0, phase = 0;           // next ring slot to fill
+            uint32_t q_use0 = 0, q_use1 = 0;
             bool ok = true;
-            auto stage_kv = [&](const CUtensorMap* tm, int x, int y) {
-                const uint32_t slot = ring % kStages, par = (ring / kStages) & 1;
-                ok = ok && mbar_wait(bars + SL::bKvEmpty + slot, par ^ 1, abort_flag, a.status);
-                if (!ok) return;
-                uint64_t* full = bars + SL::bKvFull + slot;
-                mbar_expect_tx(full, SL::kTileBytes);
-                uint8_t* dst = sKV + slot * SL::kTileBytes;
-#pragma unroll
-                for (int p = 0; p < SL::kPanels; ++p) tma_load_2d(dst + p * kPanelBytes, tm, full, x + p * 64, y);
-                ++ring;
-            };
-            auto stage_q = [&](int s, const Item& it) {
-                ok = ok && mbar_wait(bars + SL::bQEmpty + s, (q_use[s] & 1) ^ 1, abort_flag, a.status);
-                if (!ok) return;
-                uint64_t* full = bars + SL::bQFull + s;
-                mbar_expect_tx(full, SL::kTileBytes);
-                uint8_t* dst = sQ + s * SL::kTileBytes;
-#pragma unroll
-                for (int p = 0; p < SL::kPanels; ++p)
-                    tma_load_3d(dst + p * kPanelBytes, &tmQ, full, p * 64, it.head0, s ? it.token0_b : it.token0_a);
-                ++q_use[s];
-            };
             for (int idx = blockIdx.x; idx < a.n_items && ok; idx += gridDim.x) {
                 Item it;
                 decode_item(a, idx, it);
-                stage_q(0, it);
+                const int x = it.kvh * D;
+                // query tile 0
+                ok = mbar_wait_a(bar0 + 8 * (SL::bQEmpty + 0), (q_use0 & 1) ^ 1, abort_flag, a.status);
+                ++q_use0;
+                if (!ok) break;
+                if (leader) mbar_expect_tx_a(bar0 + 8 * (SL::bQFull + 0), SL::kTileBytes);
+#pragma unroll
+                for (int p = 0; p < SL::kPanels; ++p)
+                    if (leader) tma_load_3d_a(q_smem + p * kPanelBytes, &tmQ, bar0 + 8 * (SL::bQFull + 0), p * 64, it.head0,
+                                  it.token0_a);
                 for (int t = 0; t < it.n_load && ok; ++t) {
                     const bool pref = t < it.n_pref_tiles;
                     const int row = pref ? t * kTileN : it.main_row0 + (t - it.n_pref_tiles) * kTileN;
-                    stage_kv(pref ? &tmKp : &tmK, it.kvh * D, row);
-                    if (t == 0 && it.has1) stage_q(1, it);
-                    stage_kv(pref ? &tmVp : &tmV, it.kvh * D, row);
+                    // K_t
+                    ok = mbar_wait_a(bar0 + 8 * (SL::bKvEmpty + stage), phase ^ 1, abort_flag, a.status);
+                    if (!ok) break;
+                    {
+                        const uint32_t full = bar0 + 8 * (SL::bKvFull + stage), dst = kv_smem + stage * SL::kTileBytes;
+                        if (leader) mbar_expect_tx_a(full, SL::kTileBytes);
+#pragma unroll
+                        for (int p = 0; p < SL::kPanels; ++p)
+                            if (leader) tma_load_2d_a(dst + p * kPanelBytes, pref ? &tmKp : &tmK, full, x + p * 64, row);
+                    }
+                    PULSAR_RING_NEXT(stage, phase);
+                    if (t == 0 && it.has1) {
+                        ok = mbar_wait_a(bar0 + 8 * (SL::bQEmpty + 1), (q_use1 & 1) ^ 1, abort_flag, a.status);
+                        ++q_use1;
+                        if (!ok) break;
+                        if (leader) mbar_expect_tx_a(bar0 + 8 * (SL::bQFull + 1), SL::kTileBytes);
+#pragma unroll
+                        for (int p = 0; p < SL::kPanels; ++p)
+                            if (leader) tma_load_3d_a(q_smem + SL::kTileBytes + p * kPanelBytes, &tmQ, bar0 + 8 * (SL::bQFull + 1),
+                                          p * 64, it.head0, it.token0_b);
+                    }
+                    // V_t
+                    ok = mbar_wait_a(bar0 + 8 * (SL::bKvEmpty + stage), phase ^ 1, abort_flag, a.status);
+                    if (!ok) break;
+                    {
+                        const uint32_t full = bar0 + 8 * (SL::bKvFull + stage), dst = kv_smem + stage * SL::kTileBytes;
+                        if (leader) mbar_expect_tx_a(full, SL::kTileBytes);
+#pragma unroll
+                        for (int p = 0; p < SL::kPanels; ++p)
+                            if (leader) tma_load_2d_a(dst + p * kPanelBytes, pref ? &tmVp : &tmV, full, x + p * 64, row);
+                    }
+                    PULSAR_RING_NEXT(stage, phase);
                 }
             }
         }
         __syncwarp();
-    } else if (warp == kMmaWarp) {
-        // =============================== MMA issuer ===============================
-        if (lane == 0) {
+    } else if (warp == kMmaWarp || warp == kMmaWarp1) {
+        // =============================== MMA issuers ===============================
+        // One issuer per query tile (warp 8: tile 0, warp 10: tile 1).  Each runs its tile's chain
+        // S(0), then per key tile: PV(t), S(t+1).  An issuing lane is blocked while it polls a
+        // barrier and while the pipe works off its previous instruction, so two independent
+        // issuers keep the tensor pipe fed where one would leave gaps.  Both walk the whole
+        // K/V ring; a slot the tile does not use is still acknowledged so that the slot's
+        // "empty" barrier always collects one arrival from each issuer.
+        // Warp-uniform control flow, one elected lane issues (descriptors, TMEM addresses and
+        // barrier numbers then live in uniform registers, which the MMA instructions read).
+        {
+            const bool leader = elect_one();
+            const int s = (warp == kMmaWarp) ? 0 : 1;
             constexpr uint32_t kIdescQK = umma_idesc_bf16(kTileM, kTileN, false, false);
             constexpr uint32_t kIdescPV = umma_idesc_bf16(kTileM, D, false, true);
-            uint32_t ring = 0;
-            uint32_t q_use[2] = {0, 0}, p_cnt[2] = {0, 0}, o_use[2] = {0, 0};
+            constexpr uint32_t kStageStep = SL::kTileBytes >> 4;         // descriptor address units (16 bytes)
+            // Descriptors of stage 0; other stages add a multiple of kStageStep to the address
+            // field (shared memory is below 256 KB, so the 14-bit field never carries).
+            const uint64_t descQ = umma_smem_desc_sw128(smem_u32(sQ) + s * SL::kTileBytes, 16, 1024);
+            const uint64_t descK = umma_smem_desc_sw128(smem_u32(sKV), 16, 1024);
+            const uint64_t descV = umma_smem_desc_sw128(smem_u32(sKV), kPanelBytes, 1024);
+            const uint32_t tS = tmem_base + s * 128, tO = tmem_base + 256 + s * 128;
+            const uint32_t bQF = bar0 + 8 * (SL::bQFull + s), bQE = bar0 + 8 * (SL::bQEmpty + s);
+            const uint32_t bSF = bar0 + 8 * (SL::bSFull + s), bPF = bar0 + 8 * (SL::bPFull + s);
+            const uint32_t bOF = bar0 + 8 * (SL::bOFull + s), bOE = bar0 + 8 * (SL::bOEmpty + s);
+            uint32_t stage = 0, phase = 0;           // next ring slot to consume
+            uint32_t q_use = 0, p_cnt = 0, o_use = 0;
             bool ok = true;
-            auto wait_kv = [&](uint32_t n) {
-                ok = ok && mbar_wait(bars + SL::bKvFull + n % kStages, (n / kStages) & 1, abort_flag, a.status);
-                tc_fence_after();
-            };
-            auto release_kv = [&](uint32_t n) { umma_commit(bars + SL::bKvEmpty + n % kStages); };
-            auto issue_s = [&](int s, uint32_t n) {           // S_s = Q_s K^T, K in ring position n
-                const uint32_t qa = smem_u32(sQ + s * SL::kTileBytes);
-                const uint32_t ka = smem_u32(sKV + (n % kStages) * SL::kTileBytes);
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * kPanelBytes + (kk & 3) * 32;
-                    umma_ss(tmem_base + s * 128, umma_smem_desc_sw128(qa + off, 16, 1024),
-                            umma_smem_desc_sw128(ka + off, 16, 1024), kIdescQK, kk > 0 ? 1u : 0u);
-                }
-                umma_commit(bars + SL::bSFull + s);
-            };
-            auto issue_pv = [&](int s, uint32_t n, bool accumulate) {   // O_s (+)= P_s V, V in ring position n
-                const uint32_t va = smem_u32(sKV + (n % kStages) * SL::kTileBytes);
-#pragma unroll
-                for (int kk = 0; kk < kTileN / 16; ++kk)
-                    umma_ts(tmem_base + 256 + s * 128, tmem_base + s * 128 + kk * 8,
-                            umma_smem_desc_sw128(va + kk * 2048, kPanelBytes, 1024), kIdescPV,
-                            (accumulate || kk > 0) ? 1u : 0u);
-            };
-            auto wait_p = [&](int s) {
-                ok = ok && mbar_wait(bars + SL::bPFull + s, p_cnt[s] & 1, abort_flag, a.status);
-                ++p_cnt[s];
-                tc_fence_after();
-            };
+
             for (int idx = blockIdx.x; idx < a.n_items && ok; idx += gridDim.x) {
                 Item it;
                 decode_item(a, idx, it);
-                const int n0 = it.n_tiles_a, n1 = it.n_tiles_b;
-                const uint32_t base = ring;                   // K_t at base + 2t, V_t at base + 2t + 1
-                ok = ok && mbar_wait(bars + SL::bQFull + 0, q_use[0] & 1, abort_flag, a.status);
-                ++q_use[0];
-                wait_kv(base);
+                const int n = s ? it.n_tiles_b : it.n_tiles_a;
+                // K_0
+                uint32_t ks = stage, kp = phase;
+                PULSAR_RING_NEXT(stage, phase);
+                if (n > 0) {
+                    ok = mbar_wait_a(bQF, q_use & 1, abort_flag, a.status);
+                    ++q_use;
+                }
+                ok = ok && mbar_wait_a(bar0 + 8 * (SL::bKvFull + ks), kp, abort_flag, a.status);
                 if (!ok) break;
-                issue_s(0, base);
-                if (it.has1) {
-                    ok = ok && mbar_wait(bars + SL::bQFull + 1, q_use[1] & 1, abort_flag, a.status);
-                    ++q_use[1];
+                if (n > 0) {
                     tc_fence_after();
-                    if (!ok) break;
-                    issue_s(1, base);
-                }
-                release_kv(base);
-                for (int t = 0; t < it.n_load && ok; ++t) {
-                    const uint32_t nv = base + 2 * t + 1, nk = base + 2 * t + 2;
-                    wait_kv(nv);
-                    if (t < n0) {
-                        if (t == 0) {
-                            ok = ok && mbar_wait(bars + SL::bOEmpty + 0, (o_use[0] & 1) ^ 1, abort_flag, a.status);
-                            ++o_use[0];
-                        }
-                        wait_p(0);
-                        if (!ok) break;
-                        issue_pv(0, nv, t > 0);
-                        if (t == n0 - 1) {
-                            umma_commit(bars + SL::bOFull + 0);
-                            umma_commit(bars + SL::bQEmpty + 0);
-                        }
+                    const uint64_t dk = descK + static_cast<uint64_t>(ks * kStageStep);
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint64_t off = static_cast<uint64_t>(((kk >> 2) * kPanelBytes + (kk & 3) * 32) >> 4);
+                        if (leader) umma_ss(tS, descQ + off, dk + off, kIdescQK, kk > 0 ? 1u : 0u);
                     }
+                    if (leader) umma_commit_a(bSF);
+                    if (leader) umma_commit_a(bar0 + 8 * (SL::bKvEmpty + ks));
+                } else {
+                    if (leader) mbar_arrive(bars + SL::bKvEmpty + ks);
+                }
+                for (int t = 0; t < it.n_load; ++t) {
+                    const uint32_t vs = stage, vp = phase;                 // V_t
+                    PULSAR_RING_NEXT(stage, phase);
                     const bool more = t + 1 < it.n_load;
-                    if (more) wait_kv(nk);
-                    if (!ok) break;
-                    if (t + 1 < n0) issue_s(0, nk);
-                    if (t < n1) {
-                        if (t == 0) {
-                            ok = ok && mbar_wait(bars + SL::bOEmpty + 1, (o_use[1] & 1) ^ 1, abort_flag, a.status);
-                            ++o_use[1];
-                        }
-                        wait_p(1);
-                        if (!ok) break;
-                        issue_pv(1, nv, t > 0);
-                        if (t == n1 - 1) {
-                            umma_commit(bars + SL::bOFull + 1);
-                            umma_commit(bars + SL::bQEmpty + 1);
-                        }
+                    if (more) {                                            // K_{t+1}
+                        ks = stage;
+                        kp = phase;
+                        PULSAR_RING_NEXT(stage, phase);
                     }
-                    release_kv(nv);
+                    ok = mbar_wait_a(bar0 + 8 * (SL::bKvFull + vs), vp, abort_flag, a.status);
+                    if (!ok) break;
+                    if (t < n) {
+                        if (t == 0) {
+                            ok = mbar_wait_a(bOE, (o_use & 1) ^ 1, abort_flag, a.status);
+                            ++o_use;
+                        }
+                        ok = ok && mbar_wait_a(bPF, p_cnt & 1, abort_flag, a.status);
+                        ++p_cnt;
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint64_t dv = descV + static_cast<uint64_t>(vs * kStageStep);
+#pragma unroll
+                        for (int kk = 0; kk < kTileN / 16; ++kk)
+                            if (leader) umma_ts(tO, tS + kk * 8, dv + static_cast<uint64_t>(kk * 128), kIdescPV,
+                                    (t > 0 || kk > 0) ? 1u : 0u);
+                        if (t == n - 1) {
+                            if (leader) umma_commit_a(bOF);
+                            if (leader) umma_commit_a(bQE);
+                        }
+                        if (leader) umma_commit_a(bar0 + 8 * (SL::bKvEmpty + vs));
+                    } else {
+                        if (leader) mbar_arrive(bars + SL::bKvEmpty + vs);
+                    }
                     if (more) {
-                        if (t + 1 < n1) issue_s(1, nk);
-                        release_kv(nk);
+                        ok = mbar_wait_a(bar0 + 8 * (SL::bKvFull + ks), kp, abort_flag, a.status);
+                        if (!ok) break;
+                        if (t + 1 < n) {
+                            tc_fence_after();
+                            const uint64_t dk = descK + static_cast<uint64_t>(ks * kStageStep);
+#pragma unroll
+                            for (int kk = 0; kk < D / 16; ++kk) {
+                                const uint64_t off =
+                                    static_cast<uint64_t>(((kk >> 2) * kPanelBytes + (kk & 3) * 32) >> 4);
+                                if (leader) umma_ss(tS, descQ + off, dk + off, kIdescQK, kk > 0 ? 1u : 0u);
+                            }
+                            if (leader) umma_commit_a(bSF);
+                            if (leader) umma_commit_a(bar0 + 8 * (SL::bKvEmpty + ks));
+                        } else {
+                            if (leader) mbar_arrive(bars + SL::bKvEmpty + ks);
+                        }
                     }
                 }
-                ring = base + 2 * it.n_load;
             }
         }
         __syncwarp();
@@ -452,58 +546,46 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 PULSAR_TMEM_LD32_AT(tS + 96, r, 96);
                 tmem_wait_ld();
 
-                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-                if (masked) {
-#pragma unroll
-                    for (int c = 0; c < kTileN; ++c)
-                        if (c >= n_vis) r[c] = 0xff800000u;          // -inf
+                // Fast path (unmasked tile, not the first): the probabilities are formed with the
+                // maximum already in use while the tile's own maximum is computed alongside; only
+                // if that maximum exceeds the one in use by more than the threshold (rare) is the
+                // tile redone on the exact path below.
+                bool exact = masked || t == 0 || !kSpeculate;
+                if (!exact) {
+                    const float l_tile = exp_row128<kPolyPairs>(r, a.scale_log2, -m_used, tS);
+                    const float m_tile = row_max128(r) * a.scale_log2;
+                    if (__any_sync(0xffffffffu, m_tile > m_used + kRescaleThreshold)) exact = true;
+                    else l_run += l_tile;
                 }
+                if (exact) {
+                    if (masked) {
 #pragma unroll
-                for (int c = 0; c < kTileN; c += 4) {
-                    mx0 = fmaxf(mx0, __uint_as_float(r[c]));
-                    mx1 = fmaxf(mx1, __uint_as_float(r[c + 1]));
-                    mx2 = fmaxf(mx2, __uint_as_float(r[c + 2]));
-                    mx3 = fmaxf(mx3, __uint_as_float(r[c + 3]));
-                }
-                const float m_tile = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * a.scale_log2;
-
-                const bool need = m_tile > m_used + kRescaleThreshold;   // always true on the first tile
-                if (__any_sync(0xffffffffu, need)) {
-                    const float m_new = need ? m_tile : m_used;
-                    const float alpha = (m_new == -INFINITY) ? 1.f : ex2(m_used - m_new);
-                    l_run *= alpha;
-                    m_used = m_new;
-                    if (t > 0) {
+                        for (int c = 0; c < kTileN; ++c)
+                            if (c >= n_vis) r[c] = 0xff800000u;          // -inf
+                    }
+                    const float m_tile = row_max128(r) * a.scale_log2;
+                    const bool need = m_tile > m_used + kRescaleThreshold;   // always true on the first tile
+                    if (__any_sync(0xffffffffu, need)) {
+                        const float m_new = need ? m_tile : m_used;
+                        const float alpha = (m_new == -INFINITY) ? 1.f : ex2(m_used - m_new);
+                        l_run *= alpha;
+                        m_used = m_new;
+                        if (t > 0) {
 #pragma unroll
-                        for (int c0 = 0; c0 < D; c0 += 32) {
-                            uint32_t o[32];
-                            tmem_ld32(tO + c0, o);
-                            tmem_wait_ld();
+                            for (int c0 = 0; c0 < D; c0 += 32) {
+                                uint32_t o[32];
+                                tmem_ld32(tO + c0, o);
+                                tmem_wait_ld();
 #pragma unroll
-                            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-                            tmem_st32(tO + c0, o);
+                                for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                                tmem_st32(tO + c0, o);
+                            }
                         }
                     }
+                    const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
+                    if (masked) l_run += exp_row128<0>(r, a.scale_log2, neg_m, tS);
+                    else l_run += exp_row128<kSpeculate ? 0 : kPolyPairs>(r, a.scale_log2, neg_m, tS);
                 }
-                const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
-
-                float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
-#pragma unroll
-                for (int c0 = 0; c0 < kTileN; c0 += 32) {
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int c = 0; c < 32; c += 4) {
-                        const float p0 = ex2(fmaf(__uint_as_float(r[c0 + c]), a.scale_log2, neg_m));
-                        const float p1 = ex2(fmaf(__uint_as_float(r[c0 + c + 1]), a.scale_log2, neg_m));
-                        const float p2 = ex2(fmaf(__uint_as_float(r[c0 + c + 2]), a.scale_log2, neg_m));
-                        const float p3 = ex2(fmaf(__uint_as_float(r[c0 + c + 3]), a.scale_log2, neg_m));
-                        l0 += p0; l1 += p1; l2 += p2; l3 += p3;
-                        pk[c >> 1] = pack_bf16x2(p0, p1);
-                        pk[(c >> 1) + 1] = pack_bf16x2(p2, p3);
-                    }
-                    tmem_st16(tS + (c0 >> 1), pk);                   // P column c/2 holds keys c, c+1
-                }
-                l_run += (l0 + l1) + (l2 + l3);
 
                 tmem_wait_st();
                 tc_fence_before();
