@@ -118,9 +118,8 @@ phase1_plan_kernel(const int32_t* __restrict__ prefix_len, int n_blocks, int pai
 //
 //   warps 0-3   softmax of query tile 0 (one thread per query row, TMEM lane = row)
 //   warps 4-7   softmax of query tile 1
-//   warp  8     MMA issuer of tile 0 (one lane): S_0 = Q_0 K^T, O_0 += P_0 V
-//   warp  9     TMA loader (one lane): Q tiles and the K/V ring
-//   warp  10    MMA issuer of tile 1
+//   warp  8     MMA issuer (one elected lane): S_s = Q_s K^T, O_s += P_s V
+//   warp  9     TMA loader (one elected lane): Q tiles and the K/V ring
 //
 // A work item is two 128-row query tiles sharing one list of 128-key tiles.  The two tiles
 // ping-pong on the tensor pipe: while the softmax warpgroup of one tile works on S, the pipe
@@ -130,10 +129,9 @@ phase1_plan_kernel(const int32_t* __restrict__ prefix_len, int n_blocks, int pai
 // sum, so the result is unchanged); the rare rescale of O is done by the softmax warpgroup.
 // ---------------------------------------------------------------------------------------------
 constexpr int kStages = 5;
-constexpr int kAttnThreads = 384;             // warp 11 only takes part in the register hand-back
-constexpr int kMmaWarp = 8;    // issuer of query tile 0 (also owns the TMEM allocation)
+constexpr int kAttnThreads = 384;             // warps 10 and 11 only take part in the register hand-back
+constexpr int kMmaWarp = 8;
 constexpr int kLoadWarp = 9;
-constexpr int kMmaWarp1 = 10;  // issuer of query tile 1
 constexpr float kRescaleThreshold = 8.0f;      // in log2 units
 // Tuning knobs (overridable at build time with -D).
 #ifndef PULSAR_POLY_PAIRS
@@ -146,7 +144,7 @@ constexpr int kPolyPairs = PULSAR_POLY_PAIRS;  // of every four column pairs, ho
 constexpr bool kSpeculate = PULSAR_SPECULATE;  // form P with the maximum in use while the tile maximum is computed
 // Registers per thread: the kernel is compiled for 168 (twelve warps).  setmaxnreg moves
 // registers inside the CTA's own pool of 12 * 168 per lane slot and acts on whole warpgroups:
-// warpgroup 2 (the two MMA issuers, the TMA loader and a spare warp) hands back all but kRegsIssuer,
+// warpgroup 2 (MMA issuer, TMA loader and two spare warps) hands back all but kRegsIssuer,
 // the eight softmax warps grow to kRegsSoftmax:  4 * 88 + 8 * 208 = 2016 = 12 * 168.
 constexpr int kRegsIssuer = 88;
 constexpr int kRegsSoftmax = 208;
@@ -159,8 +157,8 @@ struct SmemLayout {
     static constexpr int kKV = 2 * kTileBytes;                     // kStages key/value tiles
     static constexpr int kBars = kKV + kStages * kTileBytes;
     // barrier indices
-    static constexpr int bQFull = 0, bQEmpty = 2, bSFull = 4, bPFull = 6, bOFull = 8, bOEmpty = 10;
-    static constexpr int bKvFull = 12, bKvEmpty = 12 + kStages, kNumBars = 12 + 2 * kStages;
+    static constexpr int bQFull = 0, bQEmpty = 2, bSFull = 4, bPFull = 6, bOFull = 8, bOEmpty = 10, bPFull2 = 12;
+    static constexpr int bKvFull = 14, bKvEmpty = 14 + kStages, kNumBars = 14 + 2 * kStages;
     static constexpr int kTmemPtr = kBars + kNumBars * 8;
     static constexpr int kAbort = kTmemPtr + 4;
     static constexpr int kTotal = kAbort + 4;
@@ -235,16 +233,16 @@ __device__ __forceinline__ float row_max128(const uint32_t (&r)[kTileN]) {
     return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
 }
 
-// p_c = 2^(s_c * scale + neg_m) for the 128 logits of a row, rounded to bf16 pairs and written
+// p_c = 2^(s_c * scale + neg_m) for logits [kBegin, kEnd) of a row, rounded to bf16 pairs and written
 // to TMEM as the A operand of the PV product; returns the fp32 row sum.  kPoly of every four
 // column pairs take the polynomial exp2 (FMA pipe) instead of MUFU.  kPoly must be 0 when
 // logits may be -inf (masked tiles).
-template <int kPoly>
+template <int kPoly, int kBegin = 0, int kEnd = kTileN>
 __device__ __forceinline__ float exp_row128(const uint32_t (&r)[kTileN], float scale, float neg_m, uint32_t tP) {
     float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
     const float2 sc = make_float2(scale, scale), nm = make_float2(neg_m, neg_m);
 #pragma unroll
-    for (int c0 = 0; c0 < kTileN; c0 += 32) {
+    for (int c0 = kBegin; c0 < kEnd; c0 += 32) {
         uint32_t pk[16];
 #pragma unroll
         for (int c = 0; c < 32; c += 2) {
@@ -288,13 +286,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             mbar_init(bars + SL::bQFull + s, 1);
             mbar_init(bars + SL::bQEmpty + s, 1);
             mbar_init(bars + SL::bSFull + s, 1);
-            mbar_init(bars + SL::bPFull + s, 4);
+            mbar_init(bars + SL::bPFull + s, 4);        // first half of P: one arrival per softmax warp
+            mbar_init(bars + SL::bPFull2 + s, 4);       // second half of P
             mbar_init(bars + SL::bOFull + s, 1);
             mbar_init(bars + SL::bOEmpty + s, 4);
         }
         for (int i = 0; i < kStages; ++i) {
             mbar_init(bars + SL::bKvFull + i, 1);
-            mbar_init(bars + SL::bKvEmpty + i, 2);          // one arrival from each MMA issuer
+            mbar_init(bars + SL::bKvEmpty + i, 1);
         }
         mbar_fence_init();
     }
@@ -384,61 +383,72 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             }
         }
         __syncwarp();
-    } else if (warp == kMmaWarp || warp == kMmaWarp1) {
-        // =============================== MMA issuers ===============================
-        // One issuer per query tile (warp 8: tile 0, warp 10: tile 1).  Each runs its tile's chain
-        // S(0), then per key tile: PV(t), S(t+1).  An issuing lane is blocked while it polls a
-        // barrier and while the pipe works off its previous instruction, so two independent
-        // issuers keep the tensor pipe fed where one would leave gaps.  Both walk the whole
-        // K/V ring; a slot the tile does not use is still acknowledged so that the slot's
-        // "empty" barrier always collects one arrival from each issuer.
-        // Warp-uniform control flow, one elected lane issues (descriptors, TMEM addresses and
-        // barrier numbers then live in uniform registers, which the MMA instructions read).
+    } else if (warp == kMmaWarp) {
+        // =============================== MMA issuer ===============================
+        // Per key tile t the issue order is PV_0(t), S_0(t+1), PV_1(t), S_1(t+1): tile 0 gets its
+        // next S about one PV + S ahead of tile 1, which keeps the two softmax warpgroups half a
+        // period apart (one exponentiates while the tensor pipe works for the other).
+        // Warp-uniform control flow, one elected lane issues: descriptors, TMEM addresses and
+        // barrier numbers then live in uniform registers, which the MMA instructions read.
         {
             const bool leader = elect_one();
-            const int s = (warp == kMmaWarp) ? 0 : 1;
             constexpr uint32_t kIdescQK = umma_idesc_bf16(kTileM, kTileN, false, false);
             constexpr uint32_t kIdescPV = umma_idesc_bf16(kTileM, D, false, true);
             constexpr uint32_t kStageStep = SL::kTileBytes >> 4;         // descriptor address units (16 bytes)
-            // Descriptors of stage 0; other stages add a multiple of kStageStep to the address
-            // field (shared memory is below 256 KB, so the 14-bit field never carries).
-            const uint64_t descQ = umma_smem_desc_sw128(smem_u32(sQ) + s * SL::kTileBytes, 16, 1024);
+            // Descriptors of stage 0 / query tile 0; other tiles add a multiple of kStageStep to the
+            // address field (shared memory is below 256 KB, so the 14-bit field never carries).
+            const uint64_t descQ0 = umma_smem_desc_sw128(smem_u32(sQ), 16, 1024);
+            const uint64_t descQ1 = descQ0 + kStageStep;
             const uint64_t descK = umma_smem_desc_sw128(smem_u32(sKV), 16, 1024);
             const uint64_t descV = umma_smem_desc_sw128(smem_u32(sKV), kPanelBytes, 1024);
-            const uint32_t tS = tmem_base + s * 128, tO = tmem_base + 256 + s * 128;
-            const uint32_t bQF = bar0 + 8 * (SL::bQFull + s), bQE = bar0 + 8 * (SL::bQEmpty + s);
-            const uint32_t bSF = bar0 + 8 * (SL::bSFull + s), bPF = bar0 + 8 * (SL::bPFull + s);
-            const uint32_t bOF = bar0 + 8 * (SL::bOFull + s), bOE = bar0 + 8 * (SL::bOEmpty + s);
+            const uint32_t tS0 = tmem_base, tS1 = tmem_base + 128, tO0 = tmem_base + 256, tO1 = tmem_base + 384;
             uint32_t stage = 0, phase = 0;           // next ring slot to consume
-            uint32_t q_use = 0, p_cnt = 0, o_use = 0;
+            uint32_t q_use0 = 0, q_use1 = 0, p_cnt0 = 0, p_cnt1 = 0, o_use0 = 0, o_use1 = 0;
             bool ok = true;
+
+#define PULSAR_ISSUE_S(tS, dq, dk, s_)                                                                    \
+    do {                                                                                                  \
+        _Pragma("unroll") for (int kk = 0; kk < D / 16; ++kk) {                                           \
+            const uint64_t off = static_cast<uint64_t>(((kk >> 2) * kPanelBytes + (kk & 3) * 32) >> 4);    \
+            if (leader) umma_ss(tS, (dq) + off, (dk) + off, kIdescQK, kk > 0 ? 1u : 0u);                  \
+        }                                                                                                 \
+        if (leader) umma_commit_a(bar0 + 8 * (SL::bSFull + (s_)));                                        \
+    } while (0)
+// P arrives in two halves of 64 keys, each with its own barrier.
+#define PULSAR_ISSUE_PV(tO, tP, dv, acc, s_, par)                                                         \
+    do {                                                                                                  \
+        _Pragma("unroll") for (int half = 0; half < 2; ++half) {                                          \
+            ok = ok && mbar_wait_a(bar0 + 8 * ((half ? SL::bPFull2 : SL::bPFull) + (s_)), par, abort_flag, \
+                                   a.status);                                                             \
+            tc_fence_after();                                                                             \
+            _Pragma("unroll") for (int kk = half * 4; kk < half * 4 + 4; ++kk)                            \
+                if (leader && ok)                                                                         \
+                    umma_ts(tO, (tP) + kk * 8, (dv) + static_cast<uint64_t>(kk * 128), kIdescPV,          \
+                            ((acc) || kk > 0) ? 1u : 0u);                                                 \
+        }                                                                                                 \
+    } while (0)
 
             for (int idx = blockIdx.x; idx < a.n_items && ok; idx += gridDim.x) {
                 Item it;
                 decode_item(a, idx, it);
-                const int n = s ? it.n_tiles_b : it.n_tiles_a;
+                const int n0 = it.n_tiles_a, n1 = it.n_tiles_b;
                 // K_0
                 uint32_t ks = stage, kp = phase;
                 PULSAR_RING_NEXT(stage, phase);
-                if (n > 0) {
-                    ok = mbar_wait_a(bQF, q_use & 1, abort_flag, a.status);
-                    ++q_use;
-                }
-                ok = ok && mbar_wait_a(bar0 + 8 * (SL::bKvFull + ks), kp, abort_flag, a.status);
+                ok = mbar_wait_a(bar0 + 8 * (SL::bQFull + 0), q_use0 & 1, abort_flag, a.status) &&
+                     mbar_wait_a(bar0 + 8 * (SL::bKvFull + ks), kp, abort_flag, a.status);
+                ++q_use0;
                 if (!ok) break;
-                if (n > 0) {
+                tc_fence_after();
+                PULSAR_ISSUE_S(tS0, descQ0, descK + static_cast<uint64_t>(ks * kStageStep), 0);
+                if (it.has1) {
+                    ok = mbar_wait_a(bar0 + 8 * (SL::bQFull + 1), q_use1 & 1, abort_flag, a.status);
+                    ++q_use1;
+                    if (!ok) break;
                     tc_fence_after();
-                    const uint64_t dk = descK + static_cast<uint64_t>(ks * kStageStep);
-#pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
-                        const uint64_t off = static_cast<uint64_t>(((kk >> 2) * kPanelBytes + (kk & 3) * 32) >> 4);
-                        if (leader) umma_ss(tS, descQ + off, dk + off, kIdescQK, kk > 0 ? 1u : 0u);
-                    }
-                    if (leader) umma_commit_a(bSF);
-                    if (leader) umma_commit_a(bar0 + 8 * (SL::bKvEmpty + ks));
-                } else {
-                    if (leader) mbar_arrive(bars + SL::bKvEmpty + ks);
+                    PULSAR_ISSUE_S(tS1, descQ1, descK + static_cast<uint64_t>(ks * kStageStep), 1);
                 }
+                if (leader) umma_commit_a(bar0 + 8 * (SL::bKvEmpty + ks));
                 for (int t = 0; t < it.n_load; ++t) {
                     const uint32_t vs = stage, vp = phase;                 // V_t
                     PULSAR_RING_NEXT(stage, phase);
@@ -448,50 +458,51 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                         kp = phase;
                         PULSAR_RING_NEXT(stage, phase);
                     }
+                    const uint64_t dv = descV + static_cast<uint64_t>(vs * kStageStep);
+                    const uint64_t dk = descK + static_cast<uint64_t>(ks * kStageStep);
                     ok = mbar_wait_a(bar0 + 8 * (SL::bKvFull + vs), vp, abort_flag, a.status);
                     if (!ok) break;
-                    if (t < n) {
+                    if (t < n0) {
                         if (t == 0) {
-                            ok = mbar_wait_a(bOE, (o_use & 1) ^ 1, abort_flag, a.status);
-                            ++o_use;
+                            ok = mbar_wait_a(bar0 + 8 * (SL::bOEmpty + 0), (o_use0 & 1) ^ 1, abort_flag, a.status);
+                            ++o_use0;
                         }
-                        ok = ok && mbar_wait_a(bPF, p_cnt & 1, abort_flag, a.status);
-                        ++p_cnt;
+                        PULSAR_ISSUE_PV(tO0, tS0, dv, t > 0, 0, p_cnt0 & 1);
+                        ++p_cnt0;
                         if (!ok) break;
-                        tc_fence_after();
-                        const uint64_t dv = descV + static_cast<uint64_t>(vs * kStageStep);
-#pragma unroll
-                        for (int kk = 0; kk < kTileN / 16; ++kk)
-                            if (leader) umma_ts(tO, tS + kk * 8, dv + static_cast<uint64_t>(kk * 128), kIdescPV,
-                                    (t > 0 || kk > 0) ? 1u : 0u);
-                        if (t == n - 1) {
-                            if (leader) umma_commit_a(bOF);
-                            if (leader) umma_commit_a(bQE);
+                        if (t == n0 - 1) {
+                            if (leader) umma_commit_a(bar0 + 8 * (SL::bOFull + 0));
+                            if (leader) umma_commit_a(bar0 + 8 * (SL::bQEmpty + 0));
                         }
-                        if (leader) umma_commit_a(bar0 + 8 * (SL::bKvEmpty + vs));
-                    } else {
-                        if (leader) mbar_arrive(bars + SL::bKvEmpty + vs);
                     }
                     if (more) {
                         ok = mbar_wait_a(bar0 + 8 * (SL::bKvFull + ks), kp, abort_flag, a.status);
                         if (!ok) break;
-                        if (t + 1 < n) {
-                            tc_fence_after();
-                            const uint64_t dk = descK + static_cast<uint64_t>(ks * kStageStep);
-#pragma unroll
-                            for (int kk = 0; kk < D / 16; ++kk) {
-                                const uint64_t off =
-                                    static_cast<uint64_t>(((kk >> 2) * kPanelBytes + (kk & 3) * 32) >> 4);
-                                if (leader) umma_ss(tS, descQ + off, dk + off, kIdescQK, kk > 0 ? 1u : 0u);
-                            }
-                            if (leader) umma_commit_a(bSF);
-                            if (leader) umma_commit_a(bar0 + 8 * (SL::bKvEmpty + ks));
-                        } else {
-                            if (leader) mbar_arrive(bars + SL::bKvEmpty + ks);
+                        tc_fence_after();
+                        if (t + 1 < n0) PULSAR_ISSUE_S(tS0, descQ0, dk, 0);
+                    }
+                    if (t < n1) {
+                        if (t == 0) {
+                            ok = mbar_wait_a(bar0 + 8 * (SL::bOEmpty + 1), (o_use1 & 1) ^ 1, abort_flag, a.status);
+                            ++o_use1;
                         }
+                        PULSAR_ISSUE_PV(tO1, tS1, dv, t > 0, 1, p_cnt1 & 1);
+                        ++p_cnt1;
+                        if (!ok) break;
+                        if (t == n1 - 1) {
+                            if (leader) umma_commit_a(bar0 + 8 * (SL::bOFull + 1));
+                            if (leader) umma_commit_a(bar0 + 8 * (SL::bQEmpty + 1));
+                        }
+                    }
+                    if (leader) umma_commit_a(bar0 + 8 * (SL::bKvEmpty + vs));
+                    if (more) {
+                        if (t + 1 < n1) PULSAR_ISSUE_S(tS1, descQ1, dk, 1);
+                        if (leader) umma_commit_a(bar0 + 8 * (SL::bKvEmpty + ks));
                     }
                 }
             }
+#undef PULSAR_ISSUE_S
+#undef PULSAR_ISSUE_PV
         }
         __syncwarp();
     } else if (warp < 8) {
@@ -504,6 +515,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         const uint32_t tO = tmem_base + 256 + s * 128 + lane_sel;
         uint64_t* bar_s = bars + SL::bSFull + s;
         uint64_t* bar_p = bars + SL::bPFull + s;
+        uint64_t* bar_p2 = bars + SL::bPFull2 + s;
         uint64_t* bar_of = bars + SL::bOFull + s;
         uint64_t* bar_oe = bars + SL::bOEmpty + s;
         uint32_t s_cnt = 0, o_cnt = 0;
@@ -583,14 +595,29 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                         }
                     }
                     const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
-                    if (masked) l_run += exp_row128<0>(r, a.scale_log2, neg_m, tS);
-                    else l_run += exp_row128<kSpeculate ? 0 : kPolyPairs>(r, a.scale_log2, neg_m, tS);
+                    // P goes to the MMA issuer in two halves of 64 keys, so that the first half
+                    // of the PV product runs while the second half of the row is exponentiated.
+                    // (The rescale above has stored its O columns before the first hand-over.)
+                    if (masked) l_run += exp_row128<0, 0, 64>(r, a.scale_log2, neg_m, tS);
+                    else l_run += exp_row128<kSpeculate ? 0 : kPolyPairs, 0, 64>(r, a.scale_log2, neg_m, tS);
+                    tmem_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_p);
+                    if (masked) l_run += exp_row128<0, 64, 128>(r, a.scale_log2, neg_m, tS);
+                    else l_run += exp_row128<kSpeculate ? 0 : kPolyPairs, 64, 128>(r, a.scale_log2, neg_m, tS);
+                } else {
+                    // speculative path: both halves were written above; first hand-over
+                    tmem_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_p);
                 }
 
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_p);
+                if (lane == 0) mbar_arrive(bar_p2);
             }
             if (!ok) break;
 
