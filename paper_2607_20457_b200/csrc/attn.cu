@@ -135,12 +135,16 @@ constexpr int kLoadWarp = 9;
 constexpr float kRescaleThreshold = 8.0f;      // in log2 units
 // Tuning knobs (overridable at build time with -D).
 #ifndef PULSAR_POLY_PAIRS
-#define PULSAR_POLY_PAIRS 0
+#define PULSAR_POLY_PAIRS 1
 #endif
 #ifndef PULSAR_SPECULATE
-#define PULSAR_SPECULATE 0
+#define PULSAR_SPECULATE 1
 #endif
 constexpr int kPolyPairs = PULSAR_POLY_PAIRS;  // of every four column pairs, how many use the polynomial exp2
+#ifndef PULSAR_SPLIT_FAST
+#define PULSAR_SPLIT_FAST 1
+#endif
+constexpr bool kSplitFast = PULSAR_SPLIT_FAST;   // fast path hands the first half of P over before forming the second
 constexpr bool kSpeculate = PULSAR_SPECULATE;  // form P with the maximum in use while the tile maximum is computed
 // Registers per thread: the kernel is compiled for 168 (twelve warps).  setmaxnreg moves
 // registers inside the CTA's own pool of 12 * 168 per lane slot and acts on whole warpgroups:
@@ -558,16 +562,30 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 PULSAR_TMEM_LD32_AT(tS + 96, r, 96);
                 tmem_wait_ld();
 
-                // Fast path (unmasked tile, not the first): the probabilities are formed with the
-                // maximum already in use while the tile's own maximum is computed alongside; only
-                // if that maximum exceeds the one in use by more than the threshold (rare) is the
-                // tile redone on the exact path below.
+                // Fast path (unmasked tile, not the first): the first half of the probabilities is
+                // formed with the maximum already in use while the tile's own maximum is computed
+                // alongside (independent instruction streams); only if that maximum exceeds the
+                // one in use by more than the threshold (rare) is the tile redone on the exact
+                // path below.  Either way P is handed over in two halves of 64 keys.
                 bool exact = masked || t == 0 || !kSpeculate;
                 if (!exact) {
-                    const float l_tile = exp_row128<kPolyPairs>(r, a.scale_log2, -m_used, tS);
+                    const float l_lo = exp_row128<kPolyPairs, 0, 64>(r, a.scale_log2, -m_used, tS);
                     const float m_tile = row_max128(r) * a.scale_log2;
-                    if (__any_sync(0xffffffffu, m_tile > m_used + kRescaleThreshold)) exact = true;
-                    else l_run += l_tile;
+                    if (__any_sync(0xffffffffu, m_tile > m_used + kRescaleThreshold)) {
+                        exact = true;
+                    } else if (kSplitFast) {
+                        tmem_wait_st();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_p);
+                        l_run += l_lo + exp_row128<kPolyPairs, 64, 128>(r, a.scale_log2, -m_used, tS);
+                    } else {
+                        l_run += l_lo + exp_row128<kPolyPairs, 64, 128>(r, a.scale_log2, -m_used, tS);
+                        tmem_wait_st();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_p);
+                    }
                 }
                 if (exact) {
                     if (masked) {
@@ -606,12 +624,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                     if (lane == 0) mbar_arrive(bar_p);
                     if (masked) l_run += exp_row128<0, 64, 128>(r, a.scale_log2, neg_m, tS);
                     else l_run += exp_row128<kSpeculate ? 0 : kPolyPairs, 64, 128>(r, a.scale_log2, neg_m, tS);
-                } else {
-                    // speculative path: both halves were written above; first hand-over
-                    tmem_wait_st();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_p);
                 }
 
                 tmem_wait_st();
