@@ -85,13 +85,15 @@ gather_prefix_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V, c
 // Cost in key tiles: 2 * prefix tiles + block tiles of both query tiles.  Single CTA.
 // ---------------------------------------------------------------------------------------------
 constexpr int kPlanBins = 4096;
+constexpr int kPlanThreads = 256;
 
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(kPlanThreads)
 phase1_plan_kernel(const int32_t* __restrict__ prefix_len, int n_blocks, int pairs_per_block, int prefix_total,
-                   int32_t* __restrict__ order, int32_t* status) {
+                   int n_bins, int32_t* __restrict__ order, int32_t* status) {
     __shared__ int bins[kPlanBins];
+    __shared__ int part[kPlanThreads];
     const int n_combos = n_blocks * pairs_per_block;
-    for (int i = threadIdx.x; i < kPlanBins; i += blockDim.x) bins[i] = 0;
+    for (int i = threadIdx.x; i < n_bins; i += blockDim.x) bins[i] = 0;
     __syncthreads();
     auto bin_of = [&](int c) {
         const int blk = c / pairs_per_block, pair = c - blk * pairs_per_block;
@@ -101,14 +103,34 @@ phase1_plan_kernel(const int32_t* __restrict__ prefix_len, int n_blocks, int pai
             pl = max(0, min(pl, prefix_total));
         }
         const int cost = 2 * ((pl + 127) / 128) + 4 * pair + 3;
-        return kPlanBins - 1 - min(cost, kPlanBins - 1);        // costliest first
+        return n_bins - 1 - min(cost, n_bins - 1);              // costliest first
     };
     for (int c = threadIdx.x; c < n_combos; c += blockDim.x) atomicAdd(&bins[bin_of(c)], 1);
     __syncthreads();
-    if (threadIdx.x == 0) {
-        int run = 0;
-        for (int i = 0; i < kPlanBins; ++i) { const int n = bins[i]; bins[i] = run; run += n; }
+    // exclusive prefix sum over the bins: each thread owns a run of consecutive bins
+    const int per = (n_bins + kPlanThreads - 1) / kPlanThreads;
+    const int lo = threadIdx.x * per, hi = min(lo + per, n_bins);
+    int sum = 0;
+    for (int i = lo; i < hi; ++i) sum += bins[i];
+    part[threadIdx.x] = sum;
+    __syncthreads();
+    if (threadIdx.x < 32) {                                     // scan of the 256 partial sums by one warp
+        int v[kPlanThreads / 32], tot = 0;
+#pragma unroll
+        for (int j = 0; j < kPlanThreads / 32; ++j) { v[j] = part[threadIdx.x * (kPlanThreads / 32) + j]; tot += v[j]; }
+        int incl = tot;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int nb = __shfl_up_sync(0xffffffffu, incl, o);
+            if (static_cast<int>(threadIdx.x) >= o) incl += nb;
+        }
+        int run = incl - tot;
+#pragma unroll
+        for (int j = 0; j < kPlanThreads / 32; ++j) { part[threadIdx.x * (kPlanThreads / 32) + j] = run; run += v[j]; }
     }
+    __syncthreads();
+    int run = part[threadIdx.x];
+    for (int i = lo; i < hi; ++i) { const int n = bins[i]; bins[i] = run; run += n; }
     __syncthreads();
     for (int c = threadIdx.x; c < n_combos; c += blockDim.x) order[atomicAdd(&bins[bin_of(c)], 1)] = c;
 }
@@ -848,8 +870,13 @@ extern "C" int32_t pulsar_phase1_attn(const uint16_t* Q, const uint16_t* K, cons
         count_launch();
     }
 
-    phase1_plan_kernel<<<1, 256, 0, stream>>>(prefix_len, p.n_blocks, p.pairs_per_block, prefix_total, order,
-                                              device_status);
+    {
+        // cost of an item in key tiles is at most 2 * prefix tiles + 4 * (pairs - 1) + 3
+        const int64_t max_cost = 2ll * ((prefix_total + 127) / 128) + 4ll * (p.pairs_per_block - 1) + 3;
+        const int n_bins = static_cast<int>(max_cost + 1 < kPlanBins ? max_cost + 1 : kPlanBins);
+        phase1_plan_kernel<<<1, kPlanThreads, 0, stream>>>(prefix_len, p.n_blocks, p.pairs_per_block, prefix_total,
+                                                           n_bins, order, device_status);
+    }
     PULSAR_CUDA_OK(cudaGetLastError());
     count_launch();
 

@@ -1,14 +1,14 @@
 // Max-IDF summary selection (Section 3.1, Eq. 2-4; Algorithm 1 lines 3 and 6).
 //
-// Three launches on one stream, no host synchronisation:
+// Four launches on one stream, no host synchronisation:
 //   presence_kernel   one CTA per block: a V-bit presence set of the block's token ids, built
 //                     with shared-memory atomicOr and written to the workspace
 //   df_idf_kernel     one thread per vocabulary entry: df(t) = number of blocks whose set holds
 //                     t, IDF(t) = ln(B / max(df, 1))   (Eq. 3)
-//   topk_kernel       one CTA per block: per chunk the minimum df of its tokens (the chunk with
-//                     the largest IDF is the one with the smallest df, Eq. 2), a counting
-//                     select of the k best chunks with ties to the lower index, then the
-//                     block's part of the prefix list (Eq. 4)
+//   chunk_level_kernel one warp per chunk: the minimum df of its tokens (the chunk with the largest
+//                     IDF is the one with the smallest df, Eq. 2)
+//   topk_kernel       one CTA per block: a counting select of the k best chunks with ties to the
+//                     lower index, then the block's part of the prefix list (Eq. 4)
 // Ranking uses the integer df only, so the selection is exact.
 #include "common.cuh"
 
@@ -73,9 +73,26 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int& 
     return base + incl - v;
 }
 
+// level[b*C + c] = min over the chunk's tokens of df (ids outside the vocabulary rank last).
+__global__ void __launch_bounds__(256)
+chunk_level_kernel(const uint32_t* __restrict__ ids, const uint16_t* __restrict__ df_table, int n_chunks_total,
+                   int chunk, int vocab_size, int worst, uint16_t* __restrict__ level) {
+    const int lane = threadIdx.x & 31;
+    const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (c >= n_chunks_total) return;
+    const uint32_t* tok = ids + static_cast<size_t>(c) * chunk;
+    int mn = worst;
+    for (int p = lane; p < chunk; p += 32) {
+        const uint32_t t = tok[p];
+        if (t < static_cast<uint32_t>(vocab_size)) mn = min(mn, static_cast<int>(df_table[t]));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+    if (lane == 0) level[c] = static_cast<uint16_t>(mn);
+}
+
 __global__ void __launch_bounds__(kTopkThreads)
-topk_kernel(const uint32_t* __restrict__ ids, const uint16_t* __restrict__ df_table, int n_blocks,
-            int block_size, int chunk, int k, int sink, int vocab_size,
+topk_kernel(const uint16_t* __restrict__ level_all, int n_blocks, int block_size, int chunk, int k, int sink,
             int32_t* __restrict__ sel_chunks, int32_t* __restrict__ prefix_idx, int32_t* __restrict__ prefix_len) {
     extern __shared__ int smem[];
     const int C = block_size / chunk;
@@ -86,25 +103,13 @@ topk_kernel(const uint32_t* __restrict__ ids, const uint16_t* __restrict__ df_ta
     __shared__ int s_threshold, s_need;
 
     const int b = blockIdx.x;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t* blk = ids + static_cast<size_t>(b) * block_size;
 
     for (int i = threadIdx.x; i < n_blocks + 2; i += blockDim.x) hist[i] = 0;
     __syncthreads();
-
-    // chunk score: one warp per chunk, lanes stride over its tokens
-    for (int c = warp; c < C; c += kTopkThreads / 32) {
-        int mn = n_blocks + 1;               // ids outside the vocabulary rank last
-        for (int p = lane; p < chunk; p += 32) {
-            const uint32_t t = blk[c * chunk + p];
-            if (t < static_cast<uint32_t>(vocab_size)) mn = min(mn, static_cast<int>(df_table[t]));
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, o));
-        if (lane == 0) {
-            level[c] = mn;
-            atomicAdd(&hist[mn], 1);
-        }
+    for (int c = threadIdx.x; c < C; c += blockDim.x) {
+        const int lv = level_all[static_cast<size_t>(b) * C + c];
+        level[c] = lv;
+        atomicAdd(&hist[lv], 1);
     }
     __syncthreads();
 
@@ -156,7 +161,7 @@ topk_kernel(const uint32_t* __restrict__ ids, const uint16_t* __restrict__ df_ta
 
 struct SelectPlan {
     int n_blocks, words, C;
-    size_t bitmap_bytes, df_bytes, total;
+    size_t bitmap_bytes, df_bytes, level_bytes, total;
     size_t presence_smem, topk_smem;
 };
 
@@ -175,7 +180,8 @@ int32_t plan_select(int64_t L, int32_t vocab_size, int32_t block_size, int32_t c
     if (p.presence_smem > kMaxDynSmem || p.topk_smem > kMaxDynSmem) return PULSAR_ERR_SHAPE;
     p.bitmap_bytes = round_up(static_cast<size_t>(p.n_blocks) * p.words * 4, 256);
     p.df_bytes = round_up(static_cast<size_t>(vocab_size) * 2, 256);
-    p.total = p.bitmap_bytes + p.df_bytes;
+    p.level_bytes = round_up(static_cast<size_t>(p.n_blocks) * p.C * 2, 256);
+    p.total = p.bitmap_bytes + p.df_bytes + p.level_bytes;
     return PULSAR_OK;
 }
 
@@ -210,6 +216,7 @@ extern "C" int32_t pulsar_maxidf_select(const uint32_t* token_ids, int64_t L, in
 
     uint32_t* bitmaps = static_cast<uint32_t*>(workspace);
     uint16_t* df_table = reinterpret_cast<uint16_t*>(static_cast<char*>(workspace) + p.bitmap_bytes);
+    uint16_t* level = reinterpret_cast<uint16_t*>(static_cast<char*>(workspace) + p.bitmap_bytes + p.df_bytes);
 
     if (p.presence_smem > 48 * 1024)
         PULSAR_CUDA_OK(cudaFuncSetAttribute(presence_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -226,9 +233,13 @@ extern "C" int32_t pulsar_maxidf_select(const uint32_t* token_ids, int64_t L, in
                                                                 df_out, idf_out);
     PULSAR_CUDA_OK(cudaGetLastError());
     count_launch();
-    topk_kernel<<<p.n_blocks, kTopkThreads, p.topk_smem, stream>>>(token_ids, df_table, p.n_blocks, block_size, chunk,
-                                                                   k, sink, vocab_size, sel_chunks, prefix_idx,
-                                                                   prefix_len);
+    const int n_chunks_total = p.n_blocks * p.C;
+    chunk_level_kernel<<<(n_chunks_total + 7) / 8, 256, 0, stream>>>(token_ids, df_table, n_chunks_total, chunk,
+                                                                     vocab_size, p.n_blocks + 1, level);
+    PULSAR_CUDA_OK(cudaGetLastError());
+    count_launch();
+    topk_kernel<<<p.n_blocks, kTopkThreads, p.topk_smem, stream>>>(level, p.n_blocks, block_size, chunk, k, sink,
+                                                                   sel_chunks, prefix_idx, prefix_len);
     PULSAR_CUDA_OK(cudaGetLastError());
     count_launch();
     return PULSAR_OK;

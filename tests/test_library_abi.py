@@ -35,9 +35,10 @@ def test_status_strings_and_version(lib):
 
 
 def test_workspace_sizes(lib):
-    # selection: B presence bitmaps of ceil(V/32) words + a uint16 df table, 256-byte rounded
+    # selection: B presence bitmaps of ceil(V/32) words + a uint16 df table + a uint16 level per
+    # chunk, each 256-byte rounded
     words = (128256 + 31) // 32
-    exp = -(-16 * words * 4 // 256) * 256 + -(-128256 * 2 // 256) * 256
+    exp = -(-16 * words * 4 // 256) * 256 + -(-128256 * 2 // 256) * 256 + 16 * 256 * 2
     assert binding.maxidf_select_workspace_bytes(131072, 128256, 8192, 32, 16, 64) == exp
     # phase 1: gathered prefix K and V + the work order (16 blocks x 32 tile pairs, int32)
     assert binding.phase1_workspace_bytes(131072, 32, 8, 128, 8192, 7744) == 2 * 7744 * 8 * 128 * 2 + 16 * 32 * 4
