@@ -115,6 +115,11 @@ def barrier(world):
         dist.barrier()
 
 
+def rank_workload(w, rank: int):
+    """The sequence a rank encodes: same shape for every rank, its own seed."""
+    return W.shrink(w, ids_seed=w.ids_seed + 17 * rank)
+
+
 def max_over_ranks(value: float, world: int, device) -> float:
     """The slowest rank's figure (what a whole job waits for)."""
     if world <= 1:
@@ -128,7 +133,7 @@ def max_over_ranks(value: float, world: int, device) -> float:
 # --------------------------------------------------------------------------------------------
 # CPU oracle on a bounded sample (cpu_baseline leg and --impl reference)
 # --------------------------------------------------------------------------------------------
-def oracle_sample(w, ids, Q, K, V, Qq, rows_per_block=12, p2_rows=6):
+def oracle_sample(w, ids, Q, K, V, Qq, rows_per_block=40, p2_rows=20):
     """Times the float64 oracle, as it stands, on a bounded sample of the workload and scales
     the three parts to one full step by exact work counts.  Returns a dict."""
     import oracle
@@ -203,16 +208,16 @@ def run_gpu(args, w):
     from paper_2607_20457_b200 import binding
     from paper_2607_20457_b200.pipeline import ContextEncoder
 
-    rank, world, local = dist_setup(args.gpus)
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (B200); there is no CPU path")
+    rank, world, local = dist_setup(args.gpus)
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
     binding.load_library()
     peaks = load_peaks()
 
     # every rank encodes its own sequence
-    wl = W.shrink(w, ids_seed=w.ids_seed + 17 * rank)
+    wl = rank_workload(w, rank)
     ids = W.token_ids(wl)
     Q, K, V = W.qkv(wl, seed=1 + 100 * rank)
     Qq = W.phase2_query(wl, seed=2 + 100 * rank)
