@@ -102,6 +102,42 @@ int32_t pulsar_maxidf_select(const uint32_t *token_ids, int64_t L, int32_t vocab
                              int32_t *device_status, void *stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Selection for callers that cannot allocate device memory (the paper has no counterpart; this
+ * is a packaging variant of pulsar_maxidf_select, same kernels, same results).
+ *
+ * Some hosts of this library may not call cudaMalloc at all once they are running: a serving
+ * process whose device memory is handed out in full to a pool at start-up, a plug-in loaded
+ * into an application that owns the GPU's memory budget, code that runs where the CUDA runtime
+ * forbids allocation.  Such a caller has nowhere to get the workspace pulsar_maxidf_select asks
+ * for.  This entry point takes no workspace: its scratch is a fixed array of
+ * pulsar_maxidf_select_noalloc_max_scratch() bytes (4 MiB) that is part of the library image,
+ * so every GPU that loads the library holds those bytes until the process exits.  The call
+ * itself allocates and frees nothing, on the device or through any library.
+ *
+ * Arguments, outputs, requirements and status codes are those of pulsar_maxidf_select, minus
+ * the workspace pair.  In addition:
+ *  - A problem whose workspace (pulsar_maxidf_select_workspace_bytes) exceeds the built-in
+ *    scratch is rejected with PULSAR_ERR_WORKSPACE and launches nothing.  The 128K
+ *    configuration needs about 0.5 MiB; roughly, B * vocab_size / 8 + 2 * vocab_size +
+ *    2 * L / chunk bytes must stay below 4 MiB.
+ *  - The first call on each device looks up the device address of the scratch array (one
+ *    cudaGetSymbolAddress with that device current).  Make that first call outside any stream
+ *    capture; later calls only enqueue kernels.
+ *  - All calls on a device share the one array.  Nothing in it has to be cleared between calls
+ *    (each region is written in full before it is read), but two calls whose kernels may run
+ *    at the same time (different streams without an ordering between them) race on it and
+ *    corrupt each other's results.  Order them, or use pulsar_maxidf_select with separate
+ *    workspaces.
+ * ------------------------------------------------------------------------------------------ */
+size_t pulsar_maxidf_select_noalloc_max_scratch(void);
+
+int32_t pulsar_maxidf_select_noalloc(const uint32_t *token_ids, int64_t L, int32_t vocab_size,
+                                     int32_t block_size, int32_t chunk, int32_t k, int32_t sink,
+                                     int32_t *sel_chunks, int32_t *prefix_idx, int32_t *prefix_len,
+                                     uint32_t *df_out, float *idf_out,
+                                     int32_t *device_status, void *stream);
+
+/* ------------------------------------------------------------------------------------------
  * Phase-1 prefix-block attention (Eq. 1 over the assembled input of Eq. 4; Alg. 1 l.7-8).
  *
  * For block i, row r (global position p = i*block_size + r) and query head h, the keys are

@@ -27,6 +27,7 @@ DEV_BAD_TOKEN, DEV_BAD_PREFIX, DEV_TIMEOUT, DEV_BAD_LENGTH = 0x1, 0x2, 0x4, 0x8
 EXPORTS = (
     "pulsar_status_string", "pulsar_abi_version", "pulsar_launch_count",
     "pulsar_maxidf_select_workspace_bytes", "pulsar_maxidf_select",
+    "pulsar_maxidf_select_noalloc_max_scratch", "pulsar_maxidf_select_noalloc",
     "pulsar_phase1_workspace_bytes", "pulsar_phase1_attn",
     "pulsar_phase2_choose_splits", "pulsar_phase2_workspace_bytes", "pulsar_phase2_attn",
     "pulsar_lse_merge",
@@ -69,6 +70,10 @@ def load_library(build_if_missing: bool = False):
     lib.pulsar_maxidf_select_workspace_bytes.restype = sz
     lib.pulsar_maxidf_select.argtypes = [vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp, vp]
     lib.pulsar_maxidf_select.restype = i32
+    lib.pulsar_maxidf_select_noalloc_max_scratch.argtypes = []
+    lib.pulsar_maxidf_select_noalloc_max_scratch.restype = sz
+    lib.pulsar_maxidf_select_noalloc.argtypes = [vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+    lib.pulsar_maxidf_select_noalloc.restype = i32
     lib.pulsar_phase1_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, i32]
     lib.pulsar_phase1_workspace_bytes.restype = sz
     lib.pulsar_phase1_attn.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, vp, vp, i32, f32,
@@ -152,6 +157,24 @@ def pulsar_maxidf_select(token_ids: torch.Tensor, vocab_size: int, block_size: i
     if want_idf:
         out["idf"] = idf
     return out
+
+
+def pulsar_maxidf_select_noalloc(token_ids: torch.Tensor, vocab_size: int, block_size: int, chunk: int, k: int,
+                                 sink: int, sel_chunks: torch.Tensor, prefix_idx: torch.Tensor,
+                                 prefix_len: torch.Tensor, status=None):
+    """Selection through the entry point that needs no workspace (its scratch is built into the
+    library, 4 MiB per GPU).  The caller passes every buffer: token_ids int32 [L] in, and the
+    outputs sel_chunks [B*k], prefix_idx [sink+(B-1)*k*chunk], prefix_len [B] (CUDA int32).
+    Raises PulsarError(PULSAR_ERR_WORKSPACE) if the problem does not fit the built-in scratch.
+    Calls that may overlap on the GPU share that scratch and must be ordered by the caller."""
+    lib = load_library()
+    for t, n in ((token_ids, "token_ids"), (sel_chunks, "sel_chunks"), (prefix_idx, "prefix_idx"),
+                 (prefix_len, "prefix_len")):
+        _need(t, torch.int32, n)
+    rc = lib.pulsar_maxidf_select_noalloc(_p(token_ids), token_ids.numel(), vocab_size, block_size, chunk, k, sink,
+                                          _p(sel_chunks), _p(prefix_idx), _p(prefix_len), None, None, _p(status),
+                                          _stream())
+    _check("pulsar_maxidf_select_noalloc", rc)
 
 
 def phase1_workspace_bytes(L, Hq, Hkv, d, block_size, prefix_total) -> int:

@@ -10,6 +10,8 @@
 //   topk_kernel       one CTA per block: a counting select of the k best chunks with ties to the
 //                     lower index, then the block's part of the prefix list (Eq. 4)
 // Ranking uses the integer df only, so the selection is exact.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace pulsar {
@@ -243,4 +245,64 @@ extern "C" int32_t pulsar_maxidf_select(const uint32_t* token_ids, int64_t L, in
     PULSAR_CUDA_OK(cudaGetLastError());
     count_launch();
     return PULSAR_OK;
+}
+
+// =============================================================================================
+// Selection without a caller workspace
+// =============================================================================================
+namespace {
+
+// Scratch shared by every pulsar_maxidf_select_noalloc call on a device.  It is part of the
+// library image: each GPU that loads the library holds these bytes until the process exits.
+constexpr size_t kStaticScratchBytes = 4u << 20;
+static __device__ __align__(256) unsigned char g_select_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_ptr[kMaxDevices] = {};
+
+// Device address of g_select_scratch on the current device.  In host code the symbol's name is
+// only a stand-in; the address a kernel can use comes from cudaGetSymbolAddress, looked up once
+// per device with that device current.
+int32_t static_scratch(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        (void)cudaGetLastError();
+        return PULSAR_ERR_CUDA;
+    }
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (g_scratch_ptr[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_select_scratch) != cudaSuccess || p == nullptr) {
+            (void)cudaGetLastError();
+            return PULSAR_ERR_CUDA;
+        }
+        g_scratch_ptr[dev] = p;
+    }
+    *out = g_scratch_ptr[dev];
+    return PULSAR_OK;
+}
+
+}  // namespace
+
+extern "C" size_t pulsar_maxidf_select_noalloc_max_scratch(void) { return kStaticScratchBytes; }
+
+extern "C" int32_t pulsar_maxidf_select_noalloc(const uint32_t* token_ids, int64_t L, int32_t vocab_size,
+                                                int32_t block_size, int32_t chunk, int32_t k, int32_t sink,
+                                                int32_t* sel_chunks, int32_t* prefix_idx, int32_t* prefix_len,
+                                                uint32_t* df_out, float* idf_out, int32_t* device_status,
+                                                void* stream) {
+    SelectPlan p;
+    int32_t rc = plan_select(L, vocab_size, block_size, chunk, k, sink, p);
+    if (rc != PULSAR_OK) return rc;
+    if (p.total > kStaticScratchBytes) return PULSAR_ERR_WORKSPACE;      // problem too large for the built-in scratch
+    rc = check_device();
+    if (rc != PULSAR_OK) return rc;
+    void* scratch = nullptr;
+    rc = static_scratch(&scratch);
+    if (rc != PULSAR_OK) return rc;
+    // Same kernels, same order as pulsar_maxidf_select; every scratch region is fully written
+    // before it is read, so nothing needs clearing between calls.
+    return pulsar_maxidf_select(token_ids, L, vocab_size, block_size, chunk, k, sink, sel_chunks, prefix_idx,
+                                prefix_len, df_out, idf_out, scratch, kStaticScratchBytes, device_status, stream);
 }
