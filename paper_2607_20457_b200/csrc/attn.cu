@@ -203,6 +203,14 @@ struct Item {
     int row0_a, row0_b;          // first row of each query tile within its block (phase 1)
 };
 
+// Work item of this CTA in a given round.  Items are sorted costliest first; rounds alternate
+// direction (boustrophedon) so that no CTA always draws the costlier end of a round.  -1: none.
+__device__ __forceinline__ int item_of_round(int round, int n_items) {
+    const int G = static_cast<int>(gridDim.x), c = static_cast<int>(blockIdx.x);
+    const int idx = round * G + ((round & 1) ? G - 1 - c : c);
+    return idx < n_items ? idx : -1;
+}
+
 __device__ __forceinline__ void decode_item(const AttnArgs& a, int idx, Item& it) {
     if (a.mode == kModePhase1) {
         const int combo = a.order[idx / a.Hq];
@@ -357,7 +365,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             uint32_t stage = 0, phase = 0;           // next ring slot to fill
             uint32_t q_use0 = 0, q_use1 = 0;
             bool ok = true;
-            for (int idx = blockIdx.x; idx < a.n_items && ok; idx += gridDim.x) {
+            for (int round = 0; round * static_cast<int>(gridDim.x) < a.n_items && ok; ++round) {
+                const int idx = item_of_round(round, a.n_items);
+                if (idx < 0) continue;
                 Item it;
                 decode_item(a, idx, it);
                 const int x = it.kvh * D;
@@ -454,7 +464,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         }                                                                                                 \
     } while (0)
 
-            for (int idx = blockIdx.x; idx < a.n_items && ok; idx += gridDim.x) {
+            for (int round = 0; round * static_cast<int>(gridDim.x) < a.n_items && ok; ++round) {
+                const int idx = item_of_round(round, a.n_items);
+                if (idx < 0) continue;
                 Item it;
                 decode_item(a, idx, it);
                 const int n0 = it.n_tiles_a, n1 = it.n_tiles_b;
@@ -547,7 +559,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         uint32_t s_cnt = 0, o_cnt = 0;
         bool ok = true;
 
-        for (int idx = blockIdx.x; idx < a.n_items && ok; idx += gridDim.x) {
+        for (int round = 0; round * static_cast<int>(gridDim.x) < a.n_items && ok; ++round) {
+            const int idx = item_of_round(round, a.n_items);
+            if (idx < 0) continue;
             Item it;
             decode_item(a, idx, it);
             const int n = s ? it.n_tiles_b : it.n_tiles_a;
