@@ -155,12 +155,15 @@ constexpr int kAttnThreads = 384;             // warps 10 and 11 only take part 
 constexpr int kMmaWarp = 8;
 constexpr int kLoadWarp = 9;
 constexpr float kRescaleThreshold = 8.0f;      // in log2 units
-// Tuning knobs (overridable at build time with -D).
+// Tuning knobs (overridable at build time with -D).  Measured on a 1000 W B200 running the 128K
+// step back to back (power-capped, SM clock ~1.56 GHz): both off 1060 TFLOP/s, speculation only
+// 1048, polynomial only 1032, both on 1020 -- under the power cap the variant that executes the
+// fewest instructions wins, although both options shorten the per-tile latency in short runs.
 #ifndef PULSAR_POLY_PAIRS
-#define PULSAR_POLY_PAIRS 1
+#define PULSAR_POLY_PAIRS 0
 #endif
 #ifndef PULSAR_SPECULATE
-#define PULSAR_SPECULATE 1
+#define PULSAR_SPECULATE 0
 #endif
 constexpr int kPolyPairs = PULSAR_POLY_PAIRS;  // of every four column pairs, how many use the polynomial exp2
 #ifndef PULSAR_SPLIT_FAST
