@@ -62,7 +62,7 @@ class ClockSampler:
             if not uuid.startswith("GPU-"):
                 uuid = "GPU-" + uuid
             self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
+                ["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
@@ -362,7 +362,7 @@ def run_extras(binding, w, dev, K_d, V_d, peaks):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="128k", choices=list(W.CONFIGS))
     ap.add_argument("--impl", default="pulsar", choices=["pulsar", "reference"])

@@ -41,7 +41,8 @@ struct AttnArgs {
     int Hkv;
     int pairs;             // phase 1: query-tile pairs per block; phase 2: query-tile pairs per KV head
     int n_items;           // work items in total
-    const int32_t* order;  // phase 1: (block, pair) combos, costliest first
+    int n_blocks;          // phase 1
+    int32_t* counter;      // phase 1: work counter (zeroed before the launch); null = fixed round order
     float scale_log2;      // softmax scale * log2(e)
     uint16_t* O;           // bf16 [tokens, Hq, d]   (final output mode)
     float* LSE;            // f32  [tokens, Hq] or null
@@ -80,62 +81,6 @@ gather_prefix_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V, c
 }
 
 // ---------------------------------------------------------------------------------------------
-// Phase-1 work order: one entry per (block, pair of query tiles), costliest first, so that a
-// static round-robin over the persistent CTAs ends level (longest-processing-time-first).
-// Cost in key tiles: 2 * prefix tiles + block tiles of both query tiles.  Single CTA.
-// ---------------------------------------------------------------------------------------------
-constexpr int kPlanBins = 4096;
-constexpr int kPlanThreads = 256;
-
-__global__ void __launch_bounds__(kPlanThreads)
-phase1_plan_kernel(const int32_t* __restrict__ prefix_len, int n_blocks, int pairs_per_block, int prefix_total,
-                   int n_bins, int32_t* __restrict__ order, int32_t* status) {
-    __shared__ int bins[kPlanBins];
-    __shared__ int part[kPlanThreads];
-    const int n_combos = n_blocks * pairs_per_block;
-    for (int i = threadIdx.x; i < n_bins; i += blockDim.x) bins[i] = 0;
-    __syncthreads();
-    auto bin_of = [&](int c) {
-        const int blk = c / pairs_per_block, pair = c - blk * pairs_per_block;
-        int pl = prefix_len[blk];
-        if (pl < 0 || pl > prefix_total) {
-            report(status, PULSAR_DEV_BAD_LENGTH);
-            pl = max(0, min(pl, prefix_total));
-        }
-        const int cost = 2 * ((pl + 127) / 128) + 4 * pair + 3;
-        return n_bins - 1 - min(cost, n_bins - 1);              // costliest first
-    };
-    for (int c = threadIdx.x; c < n_combos; c += blockDim.x) atomicAdd(&bins[bin_of(c)], 1);
-    __syncthreads();
-    // exclusive prefix sum over the bins: each thread owns a run of consecutive bins
-    const int per = (n_bins + kPlanThreads - 1) / kPlanThreads;
-    const int lo = threadIdx.x * per, hi = min(lo + per, n_bins);
-    int sum = 0;
-    for (int i = lo; i < hi; ++i) sum += bins[i];
-    part[threadIdx.x] = sum;
-    __syncthreads();
-    if (threadIdx.x < 32) {                                     // scan of the 256 partial sums by one warp
-        int v[kPlanThreads / 32], tot = 0;
-#pragma unroll
-        for (int j = 0; j < kPlanThreads / 32; ++j) { v[j] = part[threadIdx.x * (kPlanThreads / 32) + j]; tot += v[j]; }
-        int incl = tot;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int nb = __shfl_up_sync(0xffffffffu, incl, o);
-            if (static_cast<int>(threadIdx.x) >= o) incl += nb;
-        }
-        int run = incl - tot;
-#pragma unroll
-        for (int j = 0; j < kPlanThreads / 32; ++j) { part[threadIdx.x * (kPlanThreads / 32) + j] = run; run += v[j]; }
-    }
-    __syncthreads();
-    int run = part[threadIdx.x];
-    for (int i = lo; i < hi; ++i) { const int n = bins[i]; bins[i] = run; run += n; }
-    __syncthreads();
-    for (int c = threadIdx.x; c < n_combos; c += blockDim.x) order[atomicAdd(&bins[bin_of(c)], 1)] = c;
-}
-
-// ---------------------------------------------------------------------------------------------
 // Attention kernel: persistent, warp-specialised.
 //
 //   warps 0-3   softmax of query tile 0 (one thread per query row, TMEM lane = row)
@@ -151,6 +96,7 @@ phase1_plan_kernel(const int32_t* __restrict__ prefix_len, int n_blocks, int pai
 // sum, so the result is unchanged); the rare rescale of O is done by the softmax warpgroup.
 // ---------------------------------------------------------------------------------------------
 constexpr int kStages = 5;
+constexpr int kItemQueue = 4;     // work items the loader may publish ahead of the slowest consumer
 constexpr int kAttnThreads = 384;             // warps 10 and 11 only take part in the register hand-back
 constexpr int kMmaWarp = 8;
 constexpr int kLoadWarp = 9;
@@ -187,10 +133,13 @@ struct SmemLayout {
     static constexpr int kBars = kKV + kStages * kTileBytes;
     // barrier indices
     static constexpr int bQFull = 0, bQEmpty = 2, bSFull = 4, bPFull = 6, bOFull = 8, bOEmpty = 10, bPFull2 = 12;
-    static constexpr int bKvFull = 14, bKvEmpty = 14 + kStages, kNumBars = 14 + 2 * kStages;
+    static constexpr int bKvFull = 14, bKvEmpty = 14 + kStages;
+    static constexpr int bItemFull = 14 + 2 * kStages, bItemEmpty = bItemFull + kItemQueue;
+    static constexpr int kNumBars = bItemEmpty + kItemQueue;
     static constexpr int kTmemPtr = kBars + kNumBars * 8;
     static constexpr int kAbort = kTmemPtr + 4;
-    static constexpr int kTotal = kAbort + 4;
+    static constexpr int kItemQ = kAbort + 4;                      // int [kItemQueue]: published work items
+    static constexpr int kTotal = kItemQ + 4 * kItemQueue;
     static constexpr int kDynBytes = kTotal + 1024;                // room to align the base to 1024 bytes
 };
 
@@ -204,6 +153,7 @@ struct Item {
     int n_pref_tiles, pref_len;
     int main_row0, main_len;
     int row0_a, row0_b;          // first row of each query tile within its block (phase 1)
+    int bad_length;              // phase 1: prefix_len of the block was outside [0, prefix_total] (clamped)
 };
 
 // Work item of this CTA in a given round.  Items are sorted costliest first; rounds alternate
@@ -216,7 +166,12 @@ __device__ __forceinline__ int item_of_round(int round, int n_items) {
 
 __device__ __forceinline__ void decode_item(const AttnArgs& a, int idx, Item& it) {
     if (a.mode == kModePhase1) {
-        const int combo = a.order[idx / a.Hq];
+        // Items run block-major from the last block (longest prefix) down and, within a block,
+        // from the last tile pair (most causal tiles) down; the heads of one (block, pair) are
+        // adjacent.  CTAs that run at the same time therefore read the same K/V rows (L2 hits),
+        // and the costliest items are handed out first.
+        const int rank = idx / a.Hq;
+        const int combo = (a.n_blocks - 1 - rank / a.pairs) * a.pairs + (a.pairs - 1 - rank % a.pairs);
         it.head0 = idx - (idx / a.Hq) * a.Hq;
         it.kvh = it.head0 / a.g;
         it.part = 0;
@@ -228,6 +183,7 @@ __device__ __forceinline__ void decode_item(const AttnArgs& a, int idx, Item& it
         it.token0_a = blk * a.block_size + it.row0_a;
         it.token0_b = blk * a.block_size + it.row0_b;
         int pl = a.prefix_len[blk];
+        it.bad_length = (pl < 0 || pl > a.prefix_total) ? 1 : 0;
         pl = max(0, min(pl, a.prefix_total));
         it.pref_len = pl;
         it.n_pref_tiles = (pl + kTileN - 1) / kTileN;
@@ -246,6 +202,7 @@ __device__ __forceinline__ void decode_item(const AttnArgs& a, int idx, Item& it
         it.token0_b = (2 * rp + 1) * tokens_per_tile;
         it.has1 = (it.token0_b < a.n_tokens) ? 1 : 0;
         it.row0_a = it.row0_b = 0;
+        it.bad_length = 0;
         it.pref_len = 0;
         it.n_pref_tiles = 0;
         it.main_row0 = it.part * a.split_len;
@@ -328,6 +285,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             mbar_init(bars + SL::bOFull + s, 1);
             mbar_init(bars + SL::bOEmpty + s, 4);
         }
+        for (int i = 0; i < kItemQueue; ++i) {
+            mbar_init(bars + SL::bItemFull + i, 1);
+            mbar_init(bars + SL::bItemEmpty + i, 9);        // MMA issuer + one lane of each softmax warp
+        }
         for (int i = 0; i < kStages; ++i) {
             mbar_init(bars + SL::bKvFull + i, 1);
             mbar_init(bars + SL::bKvEmpty + i, 1);
@@ -368,11 +329,32 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             uint32_t stage = 0, phase = 0;           // next ring slot to fill
             uint32_t q_use0 = 0, q_use1 = 0;
             bool ok = true;
-            for (int round = 0; round * static_cast<int>(gridDim.x) < a.n_items && ok; ++round) {
-                const int idx = item_of_round(round, a.n_items);
-                if (idx < 0) continue;
+            volatile int* item_q = reinterpret_cast<volatile int*>(smem + SL::kItemQ);
+            for (uint32_t seq = 0; ok; ++seq) {
+                // Next work item: drawn from the global counter (phase 1: items differ in cost, so
+                // they are handed out as CTAs become free) or the fixed round order (phase 2).
+                // It is published through a small queue for the MMA issuer and the softmax warps.
+                const uint32_t slot = seq % kItemQueue;
+                ok = mbar_wait_a(bar0 + 8 * (SL::bItemEmpty + slot), ((seq / kItemQueue) & 1) ^ 1, abort_flag, a.status);
+                if (!ok) break;
+                int idx;
+                if (a.counter != nullptr) {
+                    int v = 0;
+                    if (lane == 0) v = atomicAdd(a.counter, 1);
+                    idx = __shfl_sync(0xffffffffu, v, 0);
+                    if (idx >= a.n_items) idx = -1;
+                } else {
+                    idx = static_cast<int>(seq) * static_cast<int>(gridDim.x) < a.n_items
+                              ? item_of_round(static_cast<int>(seq), a.n_items) : -1;
+                }
+                if (lane == 0) {
+                    item_q[slot] = idx;
+                    mbar_arrive(bars + SL::bItemFull + slot);
+                }
+                if (idx < 0) break;
                 Item it;
                 decode_item(a, idx, it);
+                if (it.bad_length && lane == 0) report(a.status, PULSAR_DEV_BAD_LENGTH);
                 const int x = it.kvh * D;
                 // query tile 0
                 ok = mbar_wait_a(bar0 + 8 * (SL::bQEmpty + 0), (q_use0 & 1) ^ 1, abort_flag, a.status);
@@ -467,9 +449,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         }                                                                                                 \
     } while (0)
 
-            for (int round = 0; round * static_cast<int>(gridDim.x) < a.n_items && ok; ++round) {
-                const int idx = item_of_round(round, a.n_items);
-                if (idx < 0) continue;
+            volatile int* item_q = reinterpret_cast<volatile int*>(smem + SL::kItemQ);
+            for (uint32_t seq = 0; ok; ++seq) {
+                const uint32_t slot = seq % kItemQueue;
+                ok = mbar_wait_a(bar0 + 8 * (SL::bItemFull + slot), (seq / kItemQueue) & 1, abort_flag, a.status);
+                if (!ok) break;
+                const int idx = item_q[slot];
+                if (leader) mbar_arrive(bars + SL::bItemEmpty + slot);
+                if (idx < 0) break;
                 Item it;
                 decode_item(a, idx, it);
                 const int n0 = it.n_tiles_a, n1 = it.n_tiles_b;
@@ -562,9 +549,15 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         uint32_t s_cnt = 0, o_cnt = 0;
         bool ok = true;
 
-        for (int round = 0; round * static_cast<int>(gridDim.x) < a.n_items && ok; ++round) {
-            const int idx = item_of_round(round, a.n_items);
-            if (idx < 0) continue;
+        volatile int* item_q = reinterpret_cast<volatile int*>(smem + SL::kItemQ);
+        for (uint32_t seq = 0; ok; ++seq) {
+            const uint32_t slot = seq % kItemQueue;
+            ok = __all_sync(0xffffffffu, mbar_wait(bars + SL::bItemFull + slot, (seq / kItemQueue) & 1, abort_flag, a.status));
+            if (!ok) break;
+            const int idx = item_q[slot];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bars + SL::bItemEmpty + slot);
+            if (idx < 0) break;
             Item it;
             decode_item(a, idx, it);
             const int n = s ? it.n_tiles_b : it.n_tiles_a;
@@ -796,7 +789,7 @@ int32_t launch_attn(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMa
 
 struct Phase1Plan {
     int n_blocks, tiles_per_block, pairs_per_block;
-    size_t pref_rows, pref_bytes, order_bytes, total;
+    size_t pref_rows, pref_bytes, total;
 };
 
 int32_t plan_phase1(int64_t L, int32_t Hq, int32_t Hkv, int32_t d, int32_t block_size, int32_t prefix_total,
@@ -810,8 +803,7 @@ int32_t plan_phase1(int64_t L, int32_t Hq, int32_t Hkv, int32_t d, int32_t block
     p.pref_rows = static_cast<size_t>(prefix_total > 0 ? prefix_total : 1);
     p.pairs_per_block = (p.tiles_per_block + 1) / 2;
     p.pref_bytes = round_up(p.pref_rows * Hkv * d * 2, 256);
-    p.order_bytes = round_up(static_cast<size_t>(p.n_blocks) * p.pairs_per_block * 4, 256);
-    p.total = 2 * p.pref_bytes + p.order_bytes;
+    p.total = 2 * p.pref_bytes + 256;                        // gathered prefix K, V and the work counter
     if (static_cast<int64_t>(p.n_blocks) * p.pairs_per_block * Hq >= (1ll << 31)) return PULSAR_ERR_SHAPE;
     return PULSAR_OK;
 }
@@ -869,7 +861,7 @@ extern "C" int32_t pulsar_phase1_attn(const uint16_t* Q, const uint16_t* K, cons
 
     uint16_t* Kp = static_cast<uint16_t*>(workspace);
     uint16_t* Vp = reinterpret_cast<uint16_t*>(static_cast<char*>(workspace) + p.pref_bytes);
-    int32_t* order = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + 2 * p.pref_bytes);
+    int32_t* counter = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + 2 * p.pref_bytes);
 
     CUtensorMap tmQ, tmK, tmV, tmKp, tmVp;
     if (!make_map_3d(&tmQ, Q, L, Hq, d, 1, kTileM) || !make_map_2d(&tmK, K, L, static_cast<int64_t>(Hkv) * d) ||
@@ -887,22 +879,15 @@ extern "C" int32_t pulsar_phase1_attn(const uint16_t* Q, const uint16_t* K, cons
         count_launch();
     }
 
-    {
-        // cost of an item in key tiles is at most 2 * prefix tiles + 4 * (pairs - 1) + 3
-        const int64_t max_cost = 2ll * ((prefix_total + 127) / 128) + 4ll * (p.pairs_per_block - 1) + 3;
-        const int n_bins = static_cast<int>(max_cost + 1 < kPlanBins ? max_cost + 1 : kPlanBins);
-        phase1_plan_kernel<<<1, kPlanThreads, 0, stream>>>(prefix_len, p.n_blocks, p.pairs_per_block, prefix_total,
-                                                           n_bins, order, device_status);
-    }
-    PULSAR_CUDA_OK(cudaGetLastError());
-    count_launch();
+    PULSAR_CUDA_OK(cudaMemsetAsync(counter, 0, sizeof(int32_t), stream));
 
     AttnArgs a{};
     a.mode = kModePhase1;
     a.Hkv = Hkv;
     a.pairs = p.pairs_per_block;
     a.n_items = p.n_blocks * p.pairs_per_block * Hq;
-    a.order = order;
+    a.n_blocks = p.n_blocks;
+    a.counter = counter;
     a.n_tokens = static_cast<int>(L);
     a.Hq = Hq;
     a.g = Hq / Hkv;

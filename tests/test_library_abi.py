@@ -40,8 +40,8 @@ def test_workspace_sizes(lib):
     words = (128256 + 31) // 32
     exp = -(-16 * words * 4 // 256) * 256 + -(-128256 * 2 // 256) * 256 + 16 * 256 * 2
     assert binding.maxidf_select_workspace_bytes(131072, 128256, 8192, 32, 16, 64) == exp
-    # phase 1: gathered prefix K and V + the work order (16 blocks x 32 tile pairs, int32)
-    assert binding.phase1_workspace_bytes(131072, 32, 8, 128, 8192, 7744) == 2 * 7744 * 8 * 128 * 2 + 16 * 32 * 4
+    # phase 1: gathered prefix K and V + the work counter
+    assert binding.phase1_workspace_bytes(131072, 32, 8, 128, 8192, 7744) == 2 * 7744 * 8 * 128 * 2 + 256
     # phase 2: fp32 partials for the chosen number of parts
     assert binding.phase2_workspace_bytes(512, 16, 8192, 32, 8, 128, 4) == 4 * 512 * 32 * 129 * 4
     assert binding.phase2_workspace_bytes(512, 16, 8192, 32, 8, 128, 1) == 256
