@@ -808,18 +808,27 @@ int32_t plan_phase1(int64_t L, int32_t Hq, int32_t Hkv, int32_t d, int32_t block
     return PULSAR_OK;
 }
 
-int32_t choose_splits(int32_t nq, int64_t L, int32_t Hq, int32_t Hkv) {
+// Number of KV parts for Phase 2 when the caller leaves the choice to the library: the divisor
+// J of the key-tile count that minimises a simple time model --
+//   rounds(J) * (tiles per part * t_tile + t_item)  +  partial traffic(J) / HBM bandwidth,
+// rounds = ceil(items / CTAs).  More parts fill the last round better and shorten it, but every
+// part writes and re-reads fp32 partials.  Constants are measured on B200 (one pair of query
+// tiles against one 128-key tile: about 2 us; per-item prologue and epilogue: about 6 us).
+int32_t choose_splits(int32_t nq, int64_t L, int32_t Hq, int32_t Hkv, int32_t d) {
     const int g = Hq / Hkv;
     const int64_t row_tiles = (static_cast<int64_t>(nq) * g + kTileM - 1) / kTileM;
     const int64_t items = (row_tiles + 1) / 2 * Hkv;               // a work item is a pair of row tiles
-    const int64_t want = 2ll * sm_count();
     if (L % kTileN != 0) return 1;
     const int64_t kv_tiles = L / kTileN;
+    const double ctas = sm_count(), t_tile_us = 2.0, t_item_us = 6.0, hbm_bytes_per_us = 6.0e6;
+    double best_t = 0;
     int64_t best = 1;
     for (int64_t j = 1; j <= kv_tiles && j <= 1024; ++j) {
         if (kv_tiles % j != 0) continue;
-        best = j;
-        if (items * j >= want) break;
+        const double rounds = static_cast<double>((items * j + static_cast<int64_t>(ctas) - 1) / static_cast<int64_t>(ctas));
+        const double partial = j > 1 ? 2.0 * j * nq * Hq * (d + 1) * 4.0 / hbm_bytes_per_us : 0.0;
+        const double t = rounds * (static_cast<double>(kv_tiles / j) * t_tile_us + t_item_us) + partial;
+        if (best_t == 0 || t < best_t) { best_t = t; best = j; }
     }
     return static_cast<int32_t>(best);
 }
@@ -924,7 +933,7 @@ int32_t plan_phase2(int32_t nq, int32_t B, int32_t block_size, int32_t Hq, int32
     if (g != 1 && g != 2 && g != 4 && g != 8 && g != 16) return PULSAR_ERR_SHAPE;
     const int64_t L = static_cast<int64_t>(B) * block_size;
     if (L >= (1ll << 31) || Hkv > 65535) return PULSAR_ERR_SHAPE;
-    if (n_splits == 0) n_splits = choose_splits(nq, L, Hq, Hkv);
+    if (n_splits == 0) n_splits = choose_splits(nq, L, Hq, Hkv, d);
     if (L % n_splits != 0 || n_splits > 65535) return PULSAR_ERR_SHAPE;
     part_o_bytes = round_up(static_cast<size_t>(n_splits) * nq * Hq * d * 4, 256);
     part_l_bytes = round_up(static_cast<size_t>(n_splits) * nq * Hq * 4, 256);
