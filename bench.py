@@ -34,7 +34,9 @@ from paper_2607_20457_b200 import workloads as W
 
 METRIC = "context_tokens_per_s_per_layer"
 UNIT = "tokens/s"
-LAUNCHES_PER_STEP = None   # measured from the library's own launch counter
+# DRAM bytes (read + write) of one Phase-1 attention launch at the 128K workload, from a
+# single-pass ncu capture of this bench command (summary: profiles/bench_128k_launch_list.md).
+PHASE1_DRAM_TRAFFIC_128K = 2.31e9 + 1.08e9
 
 
 # --------------------------------------------------------------------------------------------
@@ -302,7 +304,10 @@ def run_gpu(args, w):
         roofline=dict(bound="tensor", kernel="attn_kernel<128> (Phase 1)", achieved=achieved_tf,
                       peak=peaks["bf16_sustained"], unit="TFLOP/s", frac=achieved_tf / peaks["bf16_sustained"],
                       peak_source=f"{peaks['source']} sustained bf16 (kernel timed inside a long step)",
-                      algorithmic_flops_per_launch=p1_flops, traffic=args.traffic_bytes,
+                      algorithmic_flops_per_launch=p1_flops,
+                      algorithmic_hbm_bytes_per_launch=cm.phase1_hbm_bytes(wl.L, wl.Hq, wl.Hkv, wl.d),
+                      traffic=args.traffic_bytes if args.traffic_bytes is not None else
+                      (PHASE1_DRAM_TRAFFIC_128K if wl.name == "128k" else None),
                       timed="CUDA events around pulsar_phase1_attn (prefix gather + attention kernel)"),
         e2e=dict(value=world * wl.L / (e2e_ms * 1e-3), unit=UNIT, ms_per_step=e2e_ms,
                  h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h, steps=e2e_steps),
