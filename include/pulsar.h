@@ -68,6 +68,14 @@ int32_t pulsar_abi_version(void);
  * threads).  Bookkeeping for benchmarks; the paper has no counterpart. */
 uint64_t pulsar_launch_count(void);
 
+/* Self-test of the bounded device wait that every kernel of the library uses (the paper has no
+ * counterpart).  Launches one small kernel that waits on a barrier nothing arrives on; after
+ * limit_ns (1 .. 1e9 ns) the wait gives up, ORs PULSAR_DEV_TIMEOUT into *device_status and the
+ * kernel ends normally, leaving the context usable.  *device_result (device int32, may be
+ * NULL) receives 2 when the wait gave up as designed, 1 if it claimed success. */
+int32_t pulsar_wait_selftest(int32_t *device_status, uint64_t limit_ns, int32_t *device_result,
+                             void *stream);
+
 /* ------------------------------------------------------------------------------------------
  * Max-IDF summary selection (Section 3.1; Algorithm 1 lines 3 and 6; Appendix C.1, C.5).
  *

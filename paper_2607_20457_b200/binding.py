@@ -25,7 +25,7 @@ STATUS_NAMES = {
 DEV_BAD_TOKEN, DEV_BAD_PREFIX, DEV_TIMEOUT, DEV_BAD_LENGTH = 0x1, 0x2, 0x4, 0x8
 
 EXPORTS = (
-    "pulsar_status_string", "pulsar_abi_version", "pulsar_launch_count",
+    "pulsar_status_string", "pulsar_abi_version", "pulsar_launch_count", "pulsar_wait_selftest",
     "pulsar_maxidf_select_workspace_bytes", "pulsar_maxidf_select",
     "pulsar_maxidf_select_noalloc_max_scratch", "pulsar_maxidf_select_noalloc",
     "pulsar_phase1_workspace_bytes", "pulsar_phase1_attn",
@@ -66,6 +66,8 @@ def load_library(build_if_missing: bool = False):
     lib.pulsar_abi_version.restype = i32
     lib.pulsar_launch_count.argtypes = []
     lib.pulsar_launch_count.restype = ctypes.c_uint64
+    lib.pulsar_wait_selftest.argtypes = [vp, ctypes.c_uint64, vp, vp]
+    lib.pulsar_wait_selftest.restype = i32
     lib.pulsar_maxidf_select_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, i32]
     lib.pulsar_maxidf_select_workspace_bytes.restype = sz
     lib.pulsar_maxidf_select.argtypes = [vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp, vp]
@@ -117,6 +119,11 @@ def _workspace(nbytes: int, device) -> torch.Tensor:
 def launch_count() -> int:
     """Kernels launched by the library in this process so far."""
     return int(load_library().pulsar_launch_count())
+
+
+def wait_selftest(limit_ns: int, status: torch.Tensor, result: torch.Tensor):
+    """Run the bounded-wait self-test kernel (see pulsar_wait_selftest)."""
+    _check("pulsar_wait_selftest", load_library().pulsar_wait_selftest(_p(status), int(limit_ns), _p(result), _stream()))
 
 
 def new_status(device) -> torch.Tensor:

@@ -56,3 +56,38 @@ extern "C" const char* pulsar_status_string(int32_t status) {
 extern "C" int32_t pulsar_abi_version(void) { return 1; }
 
 extern "C" uint64_t pulsar_launch_count(void) { return pulsar::g_launches.load(std::memory_order_relaxed); }
+
+// ---------------------------------------------------------------------------------------------
+// Self-test of the bounded device wait used by every kernel of the library.
+// ---------------------------------------------------------------------------------------------
+namespace pulsar {
+namespace {
+__global__ void wait_selftest_kernel(int32_t* status, unsigned long long limit_ns, int32_t* result) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(&bar, 1);
+        mbar_fence_init();
+    }
+    __syncthreads();
+    // Nothing ever arrives on the barrier: the wait must give up after limit_ns, report the
+    // time-out and let the kernel finish normally.
+    const bool ok = mbar_wait(&bar, 0, &abort_flag, status, limit_ns);
+    __syncthreads();
+    if (threadIdx.x == 0 && result != nullptr) *result = (ok ? 1 : 0) | (abort_flag ? 2 : 0);
+}
+}  // namespace
+}  // namespace pulsar
+
+extern "C" int32_t pulsar_wait_selftest(int32_t* device_status, uint64_t limit_ns, int32_t* device_result,
+                                        void* stream) {
+    if (limit_ns == 0 || limit_ns > 1000000000ull) return PULSAR_ERR_INVALID_ARG;     // at most one second
+    int32_t rc = pulsar::check_device();
+    if (rc != PULSAR_OK) return rc;
+    pulsar::wait_selftest_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(device_status, limit_ns,
+                                                                                  device_result);
+    PULSAR_CUDA_OK(cudaGetLastError());
+    pulsar::count_launch();
+    return PULSAR_OK;
+}

@@ -87,7 +87,7 @@ constexpr uint64_t kWaitLimitNs = 2000000000ull;
 // thread of the CTA already gave up (abort flag in shared memory).  On expiry the abort
 // flag is raised and PULSAR_DEV_TIMEOUT is reported; callers unwind without spinning again.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                          int32_t* status) {
+                                          int32_t* status, uint64_t limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
     uint64_t t0 = 0;
@@ -98,7 +98,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
             if (*abort_flag) return false;
             uint64_t now = globaltimer_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) {
+            else if (now - t0 > limit_ns) {
                 *abort_flag = 1;
                 report(status, PULSAR_DEV_TIMEOUT);
                 return false;
