@@ -347,6 +347,28 @@ def run_extras(binding, w, dev, K_d, V_d, peaks):
         out[name] = dict(ms=ms, splits=J, gbs=nbytes / (ms * 1e-3) / 1e9,
                          frac_of_measured_hbm=nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                          l2="flushed by a 512 MiB memset before every call (its time subtracted)")
+    # one generation step (Algorithm 1 lines 11-16): a single new token appended to a shard of 64 rows
+    cap = 256
+    Kg = torch.zeros(cap, w.Hkv, w.d, dtype=torch.bfloat16, device=dev)
+    Vg = torch.zeros_like(Kg)
+    qn, kn, vn = (W.phase2_query(w, nq=1, seed=5).to(dev), torch.randn(1, w.Hkv, w.d, device=dev).to(torch.bfloat16),
+                  torch.randn(1, w.Hkv, w.d, device=dev).to(torch.bfloat16))
+    J = binding.phase2_choose_splits(1, w.n_blocks, w.block_size, w.Hq, w.Hkv, w.d)
+    wsg = binding._workspace(binding.load_library().pulsar_phase2_generate_workspace_bytes(
+        1, w.n_blocks, w.block_size, w.Hq, w.Hkv, w.d, J), dev)
+    Og = torch.empty_like(qn)
+
+    def gen_call():
+        flush.zero_()
+        binding.pulsar_phase2_generate_step(qn, kn, vn, K_d, V_d, w.n_blocks, w.block_size, Kg, Vg, 64, n_splits=J,
+                                            out=Og, workspace=wsg)
+    both = time_calls(gen_call, 10)
+    only_flush = time_calls(lambda: flush.zero_(), 10)
+    ms = both["median_ms"] - only_flush["median_ms"]
+    nbytes = cm.phase2_hbm_bytes(1, w.L, w.Hq, w.Hkv, w.d, J + 1)
+    out["phase2_generate_step_1tok"] = dict(ms=ms, context_parts=J, shard_rows=65, gbs=nbytes / (ms * 1e-3) / 1e9,
+                                            frac_of_measured_hbm=nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                            launches="2 copies + attention + merge")
     del flush
     w4 = W.CONFIGS["64k"]
     Q, K, V = (t.to(dev) for t in W.qkv(w4))

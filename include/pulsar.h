@@ -7,6 +7,7 @@
  *   pulsar_phase1_attn     Phase-1 prefix-block attention (Eq. 1 over Input_i of Eq. 4; Alg. 1 l.7-8)
  *   pulsar_phase2_attn     Phase-2 query attention + merge (Section 3.2; Alg. 1 l.12-13; App. H)
  *   pulsar_lse_merge       online-softmax merge alone      (Appendix H, Eq. 12-13)
+ *   pulsar_phase2_generate_step  one generation step: append KV(q), attend, merge (Alg. 1 l.11-16)
  *
  * Conventions that hold for every call
  * ------------------------------------
@@ -214,6 +215,41 @@ int32_t pulsar_phase2_attn(const uint16_t *Qq, int32_t nq,
                            uint16_t *O, float *LSE, float *part_O, float *part_LSE,
                            void *workspace, size_t workspace_bytes,
                            int32_t *device_status, void *stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Phase-2 generation step (Algorithm 1 lines 11-16; Section 3.2).
+ *
+ * The n_new newest tokens (the whole query on the first step, one generated token afterwards)
+ * have their keys and values appended to the "designated generation shard" (Alg. 1 l.15) and
+ * then attend to (1) all B*block_size retained context keys, without mask, and (2) the
+ * generation shard causally: new token u sees shard rows [0, gen_len + u].  The context is cut
+ * into n_splits parts as in pulsar_phase2_attn; the generation shard is one more part; all parts
+ * are merged exactly through their log-sum-exp (Appendix H), so the result equals one softmax
+ * over the concatenation [context | generation shard up to the token].
+ *
+ *   Qnew        in  [n_new, Hq, d] bf16       Knew, Vnew  in [n_new, Hkv, d] bf16
+ *   Kblocks, Vblocks in [B*block_size, Hkv, d] bf16 (retained context KV)
+ *   Kgen, Vgen  in/out [gen_capacity, Hkv, d] bf16: rows [0, gen_len) hold the earlier query /
+ *               generated tokens; rows [gen_len, gen_len + n_new) are written by this call
+ *   n_splits    parts of the context KV: 0 = library's choice, else as in pulsar_phase2_attn
+ *   O           out [n_new, Hq, d] bf16       LSE out [n_new, Hq] float32 or NULL
+ *
+ * Requirements as for pulsar_phase2_attn, plus gen_len >= 0 and gen_len + n_new <= gen_capacity
+ * (else PULSAR_ERR_SHAPE).  The workspace (pulsar_phase2_generate_workspace_bytes) is required.
+ * The caller advances gen_len by n_new after the call.
+ * ------------------------------------------------------------------------------------------ */
+size_t pulsar_phase2_generate_workspace_bytes(int32_t n_new, int32_t B, int32_t block_size,
+                                              int32_t Hq, int32_t Hkv, int32_t d, int32_t n_splits);
+
+int32_t pulsar_phase2_generate_step(const uint16_t *Qnew, const uint16_t *Knew, const uint16_t *Vnew,
+                                    int32_t n_new,
+                                    const uint16_t *Kblocks, const uint16_t *Vblocks,
+                                    int32_t B, int32_t block_size,
+                                    uint16_t *Kgen, uint16_t *Vgen, int32_t gen_len, int32_t gen_capacity,
+                                    int32_t Hq, int32_t Hkv, int32_t d, float softmax_scale,
+                                    int32_t n_splits, uint16_t *O, float *LSE,
+                                    void *workspace, size_t workspace_bytes,
+                                    int32_t *device_status, void *stream);
 
 /* ------------------------------------------------------------------------------------------
  * Online-softmax merge (Appendix H, Eq. 12-13), in its order-free closed form:

@@ -12,6 +12,7 @@ Each wrapper names the passage of the paper its C function follows:
 * :func:`phase1_attn`   -- Eq. 1 over the assembled input of Eq. 4
 * :func:`phase2_attn`   -- Section 3.2 / Appendix H (single global softmax)
 * :func:`lse_merge`     -- Appendix H Eq. 12-13, iterated
+* :func:`generate_step` -- Algorithm 1 lines 11-16 (append KV(q), attend to context + shard)
 """
 from __future__ import annotations
 
@@ -55,6 +56,8 @@ def _load():
                                            vp, vp, vp, vp]
         lib.oracle_phase2_attn.restype = ctypes.c_int
         lib.oracle_lse_merge.argtypes = [vp, vp, i32, i64, i32, vp, vp]
+        lib.oracle_generate_step.argtypes = [vp, vp, vp, i32, vp, vp, i64, vp, vp, i32, i32, i32, i32, i32, f64, vp, vp]
+        lib.oracle_generate_step.restype = ctypes.c_int
         lib.oracle_lse_merge.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -150,4 +153,22 @@ def lse_merge(part_O, part_LSE):
     rc = _load().oracle_lse_merge(_ptr(pO), _ptr(pL), J, rows, d, _ptr(O), _ptr(LSE))
     if rc != 0:
         raise ValueError(f"oracle_lse_merge rejected its arguments (rc={rc})")
+    return O, LSE
+
+
+def generate_step(Qnew, Knew, Vnew, Kctx, Vctx, Kgen_bits, Vgen_bits, gen_len, scale=0.0):
+    """One generation step.  Qnew [n,Hq,d], Knew/Vnew [n,Hkv,d], Kctx/Vctx [L,Hkv,d] bf16;
+    Kgen_bits/Vgen_bits: uint16 ndarrays [capacity,Hkv,d] holding the shard's bf16 patterns,
+    updated in place (rows gen_len .. gen_len+n).  Returns (O [n,Hq,d], LSE [n,Hq]) float64."""
+    q, kn, vn, kc, vc = _bits(Qnew), _bits(Knew), _bits(Vnew), _bits(Kctx), _bits(Vctx)
+    assert Kgen_bits.dtype == np.uint16 and Kgen_bits.flags.c_contiguous and Vgen_bits.flags.c_contiguous
+    n, Hq, d = q.shape
+    Hkv = kc.shape[1]
+    O = np.zeros((n, Hq, d), np.float64)
+    LSE = np.zeros((n, Hq), np.float64)
+    rc = _load().oracle_generate_step(_ptr(q), _ptr(kn), _ptr(vn), n, _ptr(kc), _ptr(vc), kc.shape[0],
+                                      _ptr(Kgen_bits), _ptr(Vgen_bits), gen_len, Kgen_bits.shape[0], Hq, Hkv, d,
+                                      float(scale), _ptr(O), _ptr(LSE))
+    if rc != 0:
+        raise ValueError(f"oracle_generate_step rejected its arguments (rc={rc})")
     return O, LSE

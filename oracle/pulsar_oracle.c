@@ -13,6 +13,8 @@
  *   oracle_phase2_attn     Section 3.2 / Appendix H: one softmax over the
  *                          concatenated retained KV, plus per-block partials
  *   oracle_lse_merge       Appendix H Eq. 12-13, applied iteratively
+ *   oracle_generate_step   Algorithm 1 lines 11-16: append KV(q) to the generation shard,
+ *                          attend to context + shard (causal within the shard)
  *
  * Readings taken where the paper is silent: natural logarithm; N = number of
  * logical blocks; equal chunk scores are ranked by the lower chunk index;
@@ -298,5 +300,50 @@ int oracle_lse_merge(const double *part_O, const double *part_LSE, int32_t n_par
         }
         LSE[r] = l;
     }
+    return 0;
+}
+
+/*
+ * One generation step (Algorithm 1 lines 11-16).  The n_new newest tokens' keys and values are
+ * appended to the generation shard (line 15); new token u then attends with one softmax to all
+ * L context keys and to shard rows 0 .. gen_len + u (itself included), which is what the merged
+ * per-shard results of lines 12-13 equal (Section 3.2).
+ *
+ * Qnew [n_new,Hq,d], Knew,Vnew [n_new,Hkv,d], Kctx,Vctx [L,Hkv,d], Kgen,Vgen [gen_cap,Hkv,d]
+ * bf16 bit patterns; Kgen/Vgen rows [gen_len, gen_len+n_new) are overwritten.
+ * O [n_new,Hq,d], LSE [n_new,Hq] float64.
+ */
+int oracle_generate_step(const uint16_t *Qnew, const uint16_t *Knew, const uint16_t *Vnew, int32_t n_new,
+                         const uint16_t *Kctx, const uint16_t *Vctx, int64_t L,
+                         uint16_t *Kgen, uint16_t *Vgen, int32_t gen_len, int32_t gen_cap,
+                         int32_t Hq, int32_t Hkv, int32_t d, double scale, double *O, double *LSE) {
+    if (n_new <= 0 || L <= 0 || gen_len < 0 || gen_len + n_new > gen_cap || Hkv <= 0 || Hq % Hkv || d <= 0)
+        return -1;
+    if (scale <= 0.0) scale = 1.0 / sqrt((double)d);
+    const int32_t g = Hq / Hkv;
+    const size_t row = (size_t)Hkv * d;
+    memcpy(Kgen + (size_t)gen_len * row, Knew, (size_t)n_new * row * sizeof(uint16_t));
+    memcpy(Vgen + (size_t)gen_len * row, Vnew, (size_t)n_new * row * sizeof(uint16_t));
+    const int64_t total = L + gen_len + n_new;
+    /* context rows followed by shard rows, widened */
+    float *Kf = (float *)malloc((size_t)total * row * sizeof(float));
+    float *Vf = (float *)malloc((size_t)total * row * sizeof(float));
+    int64_t *key = (int64_t *)malloc((size_t)total * sizeof(int64_t));
+    double *z = (double *)malloc((size_t)total * sizeof(double));
+    double *q = (double *)malloc((size_t)d * sizeof(double));
+    if (!Kf || !Vf || !key || !z || !q) return -2;
+    for (size_t i = 0; i < (size_t)L * row; ++i) { Kf[i] = (float)bf16_to_double(Kctx[i]); Vf[i] = (float)bf16_to_double(Vctx[i]); }
+    for (size_t i = 0; i < (size_t)(gen_len + n_new) * row; ++i) {
+        Kf[(size_t)L * row + i] = (float)bf16_to_double(Kgen[i]);
+        Vf[(size_t)L * row + i] = (float)bf16_to_double(Vgen[i]);
+    }
+    for (int64_t j = 0; j < total; ++j) key[j] = j;
+    for (int32_t u = 0; u < n_new; ++u)
+        for (int32_t h = 0; h < Hq; ++h) {
+            for (int32_t e = 0; e < d; ++e) q[e] = bf16_to_double(Qnew[((size_t)u * Hq + h) * d + e]);
+            attend_list(q, Kf, Vf, key, L + gen_len + u + 1, Hkv, h / g, d, scale, z,
+                        O + ((size_t)u * Hq + h) * d, LSE + (size_t)u * Hq + h);
+        }
+    free(Kf); free(Vf); free(key); free(z); free(q);
     return 0;
 }

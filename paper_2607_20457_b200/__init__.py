@@ -8,6 +8,7 @@ from . import cost_model, workloads  # noqa: F401
 
 _BINDING_NAMES = (
     "pulsar_maxidf_select", "pulsar_phase1_attn", "pulsar_phase2_attn", "pulsar_lse_merge",
+    "pulsar_phase2_generate_step", "pulsar_maxidf_select_noalloc",
     "maxidf_select_workspace_bytes", "phase1_workspace_bytes", "phase2_workspace_bytes",
     "PulsarError", "library_path", "load_library",
 )

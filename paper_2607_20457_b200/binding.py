@@ -30,6 +30,7 @@ EXPORTS = (
     "pulsar_maxidf_select_noalloc_max_scratch", "pulsar_maxidf_select_noalloc",
     "pulsar_phase1_workspace_bytes", "pulsar_phase1_attn",
     "pulsar_phase2_choose_splits", "pulsar_phase2_workspace_bytes", "pulsar_phase2_attn",
+    "pulsar_phase2_generate_workspace_bytes", "pulsar_phase2_generate_step",
     "pulsar_lse_merge",
 )
 
@@ -88,6 +89,11 @@ def load_library(build_if_missing: bool = False):
     lib.pulsar_phase2_attn.argtypes = [vp, i32, vp, vp, i32, i32, i32, i32, i32, f32, i32,
                                        vp, vp, vp, vp, vp, sz, vp, vp]
     lib.pulsar_phase2_attn.restype = i32
+    lib.pulsar_phase2_generate_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, i32, i32]
+    lib.pulsar_phase2_generate_workspace_bytes.restype = sz
+    lib.pulsar_phase2_generate_step.argtypes = [vp, vp, vp, i32, vp, vp, i32, i32, vp, vp, i32, i32, i32, i32, i32,
+                                                f32, i32, vp, vp, vp, sz, vp, vp]
+    lib.pulsar_phase2_generate_step.restype = i32
     lib.pulsar_lse_merge.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp]
     lib.pulsar_lse_merge.restype = i32
     _lib = lib
@@ -249,6 +255,34 @@ def pulsar_phase2_attn(Qq, Kblocks, Vblocks, n_blocks: int, block_size: int, sof
                                 _p(workspace), workspace.numel(), _p(status), _stream())
     _check("pulsar_phase2_attn", rc)
     return (O, LSE, pO, pL) if want_partials else (O, LSE)
+
+
+def pulsar_phase2_generate_step(Qnew, Knew, Vnew, Kblocks, Vblocks, n_blocks: int, block_size: int, Kgen, Vgen,
+                                gen_len: int, softmax_scale: float = 0.0, n_splits: int = 0, out=None,
+                                workspace=None, status=None):
+    """One generation step: append Knew/Vnew to the generation shard (rows gen_len..), then the
+    n_new tokens attend to all context KV and, causally, to the shard; merged exactly.
+    Qnew [n_new,Hq,d], Knew/Vnew [n_new,Hkv,d], Kgen/Vgen [capacity,Hkv,d] CUDA bf16 (updated in
+    place).  Returns (O bf16 [n_new,Hq,d], LSE f32 [n_new,Hq]); the caller adds n_new to gen_len."""
+    lib = load_library()
+    for t, n in ((Qnew, "Qnew"), (Knew, "Knew"), (Vnew, "Vnew"), (Kblocks, "Kblocks"), (Vblocks, "Vblocks"),
+                 (Kgen, "Kgen"), (Vgen, "Vgen")):
+        _need(t, torch.bfloat16, n)
+    n_new, Hq, d = Qnew.shape
+    Hkv = Kblocks.shape[-2]
+    if n_splits == 0:
+        n_splits = phase2_choose_splits(n_new, n_blocks, block_size, Hq, Hkv, d)
+    O = torch.empty_like(Qnew) if out is None else out
+    LSE = torch.empty((n_new, Hq), dtype=torch.float32, device=Qnew.device)
+    if workspace is None:
+        workspace = _workspace(lib.pulsar_phase2_generate_workspace_bytes(n_new, n_blocks, block_size, Hq, Hkv, d,
+                                                                          n_splits), Qnew.device)
+    rc = lib.pulsar_phase2_generate_step(_p(Qnew), _p(Knew), _p(Vnew), n_new, _p(Kblocks), _p(Vblocks), n_blocks,
+                                         block_size, _p(Kgen), _p(Vgen), gen_len, Kgen.shape[0], Hq, Hkv, d,
+                                         float(softmax_scale), n_splits, _p(O), _p(LSE), _p(workspace),
+                                         workspace.numel(), _p(status), _stream())
+    _check("pulsar_phase2_generate_step", rc)
+    return O, LSE
 
 
 def pulsar_lse_merge(part_O, part_LSE, want_lse: bool = True):

@@ -38,6 +38,9 @@ struct AttnArgs {
     int prefix_total;      // phase 1: rows in the gathered prefix buffers
     const int32_t* prefix_len;
     int split_len;         // phase 2: keys per KV part
+    int n_ctx_parts;       // phase 2: parts of the context KV; part n_ctx_parts (if any) is the generation shard
+    int gen_len;           // phase 2: rows of the generation shard that precede the new tokens
+    int gen_total;         // phase 2: gen_len + new tokens (0 = no generation shard)
     int Hkv;
     int pairs;             // phase 1: query-tile pairs per block; phase 2: query-tile pairs per KV head
     int n_items;           // work items in total
@@ -154,6 +157,7 @@ struct Item {
     int main_row0, main_len;
     int row0_a, row0_b;          // first row of each query tile within its block (phase 1)
     int bad_length;              // phase 1: prefix_len of the block was outside [0, prefix_total] (clamped)
+    int gen_base;                // >= 0: generation shard, token u sees its rows [0, gen_base + u]; -1 otherwise
 };
 
 // Work item of this CTA in a given round.  Items are sorted costliest first; rounds alternate
@@ -189,6 +193,7 @@ __device__ __forceinline__ void decode_item(const AttnArgs& a, int idx, Item& it
         it.n_pref_tiles = (pl + kTileN - 1) / kTileN;
         it.main_row0 = blk * a.block_size;
         it.main_len = a.block_size;
+        it.gen_base = -1;
         it.n_tiles_a = it.n_pref_tiles + qt0 + 1;
         it.n_tiles_b = it.has1 ? it.n_pref_tiles + qt0 + 2 : 0;
     } else {
@@ -203,11 +208,23 @@ __device__ __forceinline__ void decode_item(const AttnArgs& a, int idx, Item& it
         it.has1 = (it.token0_b < a.n_tokens) ? 1 : 0;
         it.row0_a = it.row0_b = 0;
         it.bad_length = 0;
-        it.pref_len = 0;
-        it.n_pref_tiles = 0;
-        it.main_row0 = it.part * a.split_len;
-        it.main_len = a.split_len;
-        const int n = (a.split_len + kTileN - 1) / kTileN;
+        int n;
+        if (a.gen_total > 0 && it.part == a.n_ctx_parts) {
+            // the generation shard: read through the second pair of tensor maps, causal by token
+            it.pref_len = a.gen_total;
+            it.n_pref_tiles = (a.gen_total + kTileN - 1) / kTileN;
+            it.main_row0 = 0;
+            it.main_len = 0;
+            it.gen_base = a.gen_len;
+            n = it.n_pref_tiles;
+        } else {
+            it.pref_len = 0;
+            it.n_pref_tiles = 0;
+            it.main_row0 = it.part * a.split_len;
+            it.main_len = a.split_len;
+            it.gen_base = -1;
+            n = (a.split_len + kTileN - 1) / kTileN;
+        }
         it.n_tiles_a = n;
         it.n_tiles_b = it.has1 ? n : 0;
     }
@@ -572,6 +589,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 if (t < it.n_pref_tiles) {
                     const int valid = it.pref_len - t * kTileN;
                     if (valid < kTileN) { n_vis = valid; masked = true; }
+                    if (it.gen_base >= 0) {                   // generation shard: causal by token
+                        const int token = (s ? it.token0_b : it.token0_a) + row / a.pack;
+                        n_vis = min(n_vis, it.gen_base + token + 1 - t * kTileN);
+                        masked = true;
+                    }
                 } else {
                     const int j = t - it.n_pref_tiles;
                     const int valid = it.main_len - j * kTileN;
@@ -997,6 +1019,7 @@ extern "C" int32_t pulsar_phase2_attn(const uint16_t* Qq, int32_t nq, const uint
     a.g = g;
     a.pack = g;
     a.split_len = static_cast<int>(L / n_splits);
+    a.n_ctx_parts = n_splits;
     a.scale_log2 = (softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf(static_cast<float>(d))) * 1.4426950408889634f;
     a.O = O;
     a.LSE = LSE;
@@ -1014,4 +1037,87 @@ extern "C" int32_t pulsar_phase2_attn(const uint16_t* Qq, int32_t nq, const uint
     if (partial_out)
         return launch_lse_merge(pO, pL, n_splits, static_cast<int64_t>(nq) * Hq, d, O, LSE, stream);
     return PULSAR_OK;
+}
+
+// =============================================================================================
+// Phase 2, generation step (Algorithm 1 lines 11-16): context parts + the generation shard
+// =============================================================================================
+extern "C" size_t pulsar_phase2_generate_workspace_bytes(int32_t n_new, int32_t B, int32_t block_size, int32_t Hq,
+                                                         int32_t Hkv, int32_t d, int32_t n_splits) {
+    size_t a, b;
+    if (plan_phase2(n_new, B, block_size, Hq, Hkv, d, n_splits, a, b) != PULSAR_OK) return 0;
+    // one more part than the context has: the generation shard
+    return round_up(static_cast<size_t>(n_splits + 1) * n_new * Hq * d * 4, 256) +
+           round_up(static_cast<size_t>(n_splits + 1) * n_new * Hq * 4, 256);
+}
+
+extern "C" int32_t pulsar_phase2_generate_step(const uint16_t* Qnew, const uint16_t* Knew, const uint16_t* Vnew,
+                                               int32_t n_new, const uint16_t* Kb, const uint16_t* Vb, int32_t B,
+                                               int32_t block_size, uint16_t* Kgen, uint16_t* Vgen, int32_t gen_len,
+                                               int32_t gen_capacity, int32_t Hq, int32_t Hkv, int32_t d,
+                                               float softmax_scale, int32_t n_splits, uint16_t* O, float* LSE,
+                                               void* workspace, size_t workspace_bytes, int32_t* device_status,
+                                               void* stream_) {
+    size_t unused_a, unused_b;
+    if (gen_len < 0 || gen_capacity <= 0) return PULSAR_ERR_INVALID_ARG;
+    int32_t rc = plan_phase2(n_new, B, block_size, Hq, Hkv, d, n_splits, unused_a, unused_b);
+    if (rc != PULSAR_OK) return rc;
+    if (static_cast<int64_t>(gen_len) + n_new > gen_capacity) return PULSAR_ERR_SHAPE;
+    if (!Qnew || !Knew || !Vnew || !Kb || !Vb || !Kgen || !Vgen || !O || !workspace) return PULSAR_ERR_INVALID_ARG;
+    if (!aligned(Qnew, 16) || !aligned(Knew, 16) || !aligned(Vnew, 16) || !aligned(Kb, 16) || !aligned(Vb, 16) ||
+        !aligned(Kgen, 16) || !aligned(Vgen, 16) || !aligned(O, 16) || (LSE && !aligned(LSE, 4)) ||
+        !aligned(workspace, 256))
+        return PULSAR_ERR_ALIGNMENT;
+    const int n_parts = n_splits + 1;
+    const size_t po_bytes = round_up(static_cast<size_t>(n_parts) * n_new * Hq * d * 4, 256);
+    const size_t pl_bytes = round_up(static_cast<size_t>(n_parts) * n_new * Hq * 4, 256);
+    if (workspace_bytes < po_bytes + pl_bytes) return PULSAR_ERR_WORKSPACE;
+    rc = check_device();
+    if (rc != PULSAR_OK) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+
+    const int64_t L = static_cast<int64_t>(B) * block_size;
+    const int g = Hq / Hkv;
+    const size_t row_bytes = static_cast<size_t>(Hkv) * d * 2;
+    CUtensorMap tmQ, tmK, tmV, tmKg, tmVg;
+    if (!make_map_3d(&tmQ, Qnew, n_new, Hq, d, g, kTileM / g) ||
+        !make_map_2d(&tmK, Kb, L, static_cast<int64_t>(Hkv) * d) ||
+        !make_map_2d(&tmV, Vb, L, static_cast<int64_t>(Hkv) * d) ||
+        !make_map_2d(&tmKg, Kgen, gen_capacity, static_cast<int64_t>(Hkv) * d) ||
+        !make_map_2d(&tmVg, Vgen, gen_capacity, static_cast<int64_t>(Hkv) * d))
+        return PULSAR_ERR_CUDA;
+
+    // append KV(q) to the generation shard (Algorithm 1 line 15), then attend
+    PULSAR_CUDA_OK(cudaMemcpyAsync(reinterpret_cast<char*>(Kgen) + gen_len * row_bytes, Knew, n_new * row_bytes,
+                                   cudaMemcpyDeviceToDevice, stream));
+    PULSAR_CUDA_OK(cudaMemcpyAsync(reinterpret_cast<char*>(Vgen) + gen_len * row_bytes, Vnew, n_new * row_bytes,
+                                   cudaMemcpyDeviceToDevice, stream));
+
+    float* pO = static_cast<float*>(workspace);
+    float* pL = reinterpret_cast<float*>(static_cast<char*>(workspace) + po_bytes);
+    AttnArgs a{};
+    a.mode = kModePhase2;
+    a.n_tokens = n_new;
+    a.Hq = Hq;
+    a.g = g;
+    a.pack = g;
+    a.split_len = static_cast<int>(L / n_splits);
+    a.n_ctx_parts = n_splits;
+    a.gen_len = gen_len;
+    a.gen_total = gen_len + n_new;
+    a.scale_log2 = (softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf(static_cast<float>(d))) * 1.4426950408889634f;
+    a.O = O;
+    a.LSE = LSE;
+    a.part_O = pO;
+    a.part_LSE = pL;
+    a.status = device_status;
+    const int tokens_per_tile = kTileM / g;
+    const int row_tiles = (n_new + tokens_per_tile - 1) / tokens_per_tile;
+    a.Hkv = Hkv;
+    a.pairs = (row_tiles + 1) / 2;
+    a.n_items = a.pairs * Hkv * n_parts;
+    rc = d == 128 ? launch_attn<128>(tmQ, tmK, tmV, tmKg, tmVg, a, stream)
+                  : launch_attn<64>(tmQ, tmK, tmV, tmKg, tmVg, a, stream);
+    if (rc != PULSAR_OK) return rc;
+    return launch_lse_merge(pO, pL, n_parts, static_cast<int64_t>(n_new) * Hq, d, O, LSE, stream);
 }

@@ -1,0 +1,61 @@
+"""GPU parity: the Phase-2 generation step against the oracle (Algorithm 1 lines 11-16)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import check_attention
+from paper_2607_20457_b200 import binding, workloads as W
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def run_steps(w, steps, cap, q_scale=1.0, n_splits=0):
+    _, K, V = W.qkv(w)
+    Kd, Vd = K.to(DEV), V.to(DEV)
+    gen = torch.Generator().manual_seed(21)
+    Kgen_o = np.zeros((cap, w.Hkv, w.d), np.uint16); Vgen_o = np.zeros_like(Kgen_o)
+    Kgen_d = torch.zeros(cap, w.Hkv, w.d, dtype=torch.bfloat16, device=DEV); Vgen_d = torch.zeros_like(Kgen_d)
+    status = binding.new_status(DEV)
+    gen_len = 0
+    for n_new in steps:
+        Qn = (torch.randn(n_new, w.Hq, w.d, generator=gen) * q_scale).to(torch.bfloat16)
+        Kn = torch.randn(n_new, w.Hkv, w.d, generator=gen).to(torch.bfloat16)
+        Vn = torch.randn(n_new, w.Hkv, w.d, generator=gen).to(torch.bfloat16)
+        O, LSE = binding.pulsar_phase2_generate_step(Qn.to(DEV), Kn.to(DEV), Vn.to(DEV), Kd, Vd, w.n_blocks,
+                                                     w.block_size, Kgen_d, Vgen_d, gen_len, n_splits=n_splits,
+                                                     status=status)
+        Oref, Lref = oracle.generate_step(Qn, Kn, Vn, K, V, Kgen_o, Vgen_o, gen_len)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        print(check_attention(O, LSE, Oref, Lref, f"{w.name} step n_new={n_new} gen_len={gen_len}"))
+        gen_len += n_new
+        # the shard on the device holds the same bits as the oracle's
+        got = Kgen_d[:gen_len].cpu().view(torch.int16).numpy().view(np.uint16)
+        np.testing.assert_array_equal(got, Kgen_o[:gen_len])
+    return gen_len
+
+
+def test_tiny_config_query_then_tokens():
+    run_steps(W.CONFIGS["tiny"], [32, 1, 1, 1, 7], cap=64)
+
+
+def test_shard_longer_than_one_key_tile_and_peaked_logits():
+    # 150 + 140 rows: the shard spans three key tiles, the new tokens two query tiles
+    w = W.shrink(W.CONFIGS["tiny"], L=2048, block_size=512, Hq=8, Hkv=2, d=128)
+    run_steps(w, [150, 140, 1], cap=320, q_scale=3.0, n_splits=4)
+
+
+def test_16k_config_query_of_64_then_decode():
+    run_steps(W.CONFIGS["16k"], [64, 1, 1], cap=128)
+
+
+def test_capacity_is_checked_on_the_host():
+    w = W.CONFIGS["tiny"]
+    _, K, V = W.qkv(w)
+    z = lambda n, h: torch.zeros(n, h, w.d, dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(binding.PulsarError) as e:
+        binding.pulsar_phase2_generate_step(z(4, w.Hq), z(4, w.Hkv), z(4, w.Hkv), K.to(DEV), V.to(DEV), w.n_blocks,
+                                            w.block_size, z(8, w.Hkv), z(8, w.Hkv), gen_len=6)
+    assert e.value.status == 2

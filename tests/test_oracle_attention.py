@@ -214,3 +214,46 @@ def test_uniform_keys_closed_form():
         np.testing.assert_allclose(O[:, h], np.broadcast_to(f64(V)[:, h // g].mean(0), O[:, h].shape), atol=1e-12)
         z = f64(Qq)[:, h] @ f64(K)[0, h // g] / np.sqrt(w.d)
         np.testing.assert_allclose(LSE[:, h], z + np.log(w.L), atol=1e-12)
+
+
+def _bits_of(t):
+    return np.ascontiguousarray(t.contiguous().view(torch.int16).numpy().view(np.uint16))
+
+
+def test_generate_step_is_one_softmax_over_context_and_causal_shard():
+    # Algorithm 1 lines 11-16: query tokens, then generated tokens, are appended to the generation
+    # shard and attend to all context keys plus the shard up to themselves.
+    w = small_workload()
+    _, K, V = W.qkv(w)
+    cap, g = 16, w.Hq // w.Hkv
+    gen = torch.Generator().manual_seed(9)
+    Kgen = np.zeros((cap, w.Hkv, w.d), np.uint16)
+    Vgen = np.zeros((cap, w.Hkv, w.d), np.uint16)
+    gen_len = 0
+    hist_K, hist_V = [], []
+    for n_new in (5, 1, 1, 3):                                  # the query first, then single tokens
+        Qn = torch.randn(n_new, w.Hq, w.d, generator=gen).to(torch.bfloat16)
+        Kn = torch.randn(n_new, w.Hkv, w.d, generator=gen).to(torch.bfloat16)
+        Vn = torch.randn(n_new, w.Hkv, w.d, generator=gen).to(torch.bfloat16)
+        O, LSE = oracle.generate_step(Qn, Kn, Vn, K, V, Kgen, Vgen, gen_len)
+        hist_K.append(Kn); hist_V.append(Vn)
+        Kall = torch.cat([K] + hist_K); Vall = torch.cat([V] + hist_V)
+        # the shard now holds exactly the appended rows
+        np.testing.assert_array_equal(Kgen[: gen_len + n_new], _bits_of(torch.cat(hist_K)))
+        np.testing.assert_array_equal(Vgen[: gen_len + n_new], _bits_of(torch.cat(hist_V)))
+        for u in range(n_new):
+            n_keys = w.L + gen_len + u + 1
+            k, v, q = f64(Kall[:n_keys]), f64(Vall[:n_keys]), f64(Qn[u])
+            for h in range(w.Hq):
+                zz = k[:, h // g] @ q[h] / np.sqrt(w.d)
+                e = np.exp(zz - zz.max())
+                np.testing.assert_allclose(O[u, h], (e / e.sum()) @ v[:, h // g], atol=1e-12)
+                assert abs(LSE[u, h] - (zz.max() + np.log(e.sum()))) < 1e-12
+        gen_len += n_new
+    # the newest token with an empty history and a one-token step is plain Phase 2 over context + itself
+    Kgen2 = np.zeros((4, w.Hkv, w.d), np.uint16); Vgen2 = np.zeros_like(Kgen2)
+    Qn, Kn, Vn = hist_K[1].repeat_interleave(g, 1), hist_K[1], hist_V[1]
+    O1, L1 = oracle.generate_step(Qn, Kn, Vn, K, V, Kgen2, Vgen2, 0)
+    O2, L2 = oracle.phase2_attn(Qn, torch.cat([K, Kn]), torch.cat([V, Vn]), 1, w.L + 1)
+    np.testing.assert_allclose(O1, O2, atol=1e-12)
+    np.testing.assert_allclose(L1, L2, atol=1e-12)
