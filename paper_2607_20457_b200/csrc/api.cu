@@ -5,11 +5,12 @@
 
 namespace pulsar {
 
+// Per-device facts are cached per host thread (a thread may switch devices between calls).
 int32_t check_device() {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return PULSAR_ERR_CUDA; }
-    static int cached_dev = -1;
-    static int32_t cached_rc = PULSAR_ERR_CUDA;
+    thread_local int cached_dev = -1;
+    thread_local int32_t cached_rc = PULSAR_ERR_CUDA;
     if (dev == cached_dev) return cached_rc;
     int major = 0, minor = 0;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
@@ -23,11 +24,16 @@ int32_t check_device() {
 }
 
 int sm_count() {
-    static int cached_dev = -1, cached = 0;
+    thread_local int cached_dev = -1, cached = 148;
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return 148; }
     if (dev != cached_dev) {
-        if (cudaDeviceGetAttribute(&cached, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) cached = 148;
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+            (void)cudaGetLastError();
+            return 148;
+        }
+        cached = n;
         cached_dev = dev;
     }
     return cached;

@@ -796,11 +796,9 @@ template <int D>
 int32_t launch_attn(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& v, const CUtensorMap& kp,
                     const CUtensorMap& vp, const AttnArgs& a, cudaStream_t stream) {
     constexpr int smem = SmemLayout<D>::kDynBytes;
-    static bool configured = false;
-    if (!configured) {
-        PULSAR_CUDA_OK(cudaFuncSetAttribute(attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        configured = true;
-    }
+    // The opt-in to more than 48 KB of dynamic shared memory is a per-device function attribute;
+    // setting it on every launch keeps multi-device processes correct and costs well under a microsecond.
+    PULSAR_CUDA_OK(cudaFuncSetAttribute(attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     const int grid = a.n_items < sm_count() ? a.n_items : sm_count();     // one persistent CTA per SM
     if (grid <= 0) return PULSAR_OK;
     attn_kernel<D><<<grid, kAttnThreads, smem, stream>>>(q, k, v, kp, vp, a);

@@ -126,3 +126,30 @@ def test_retained_kv_is_the_blocks_own_rows_and_runs_repeat_exactly():
     assert torch.equal(Kr, K) and torch.equal(Vr, V) and Kr.data_ptr() != K.data_ptr()
     assert Kv.data_ptr() == K.data_ptr() and Kr.shape[0] == w.L        # exactly block_size rows per block, L in total
     assert torch.equal(O1, O2) and torch.equal(L1, L2)
+
+
+def test_many_small_blocks_long_nested_prefix():
+    # 32 blocks of one tile each: the prefix grows to 31 summaries, every item is a single tile pair
+    w = W.shrink(W.CONFIGS["tiny"], L=4096, block_size=128, chunk=8, k=3, sink=16, Hq=4, Hkv=2, d=64, vocab_size=4096)
+    sel = oracle.maxidf_select(W.needle_ids(w), w.vocab_size, w.block_size, w.chunk, w.k, w.sink)
+    Q, K, V = W.qkv(w, q_scale=2.0)
+    print(run_phase1(w, Q, K, V, sel["prefix_idx"], sel["prefix_len"], what="32 blocks"))
+
+
+def test_prefix_list_present_but_unused():
+    # a prefix list exists, yet every block is told to use none of it
+    w = W.shrink(W.CONFIGS["tiny"], L=1024, block_size=256)
+    Q, K, V = W.qkv(w)
+    pidx, _ = W.first_k_prefix(w)
+    print(run_phase1(w, Q, K, V, pidx, np.zeros(w.n_blocks, np.int32), what="unused prefix"))
+
+
+def test_non_monotone_prefix_lengths():
+    # the scheduler assumes later blocks are costlier; results must not depend on that
+    w = W.shrink(W.CONFIGS["tiny"], L=2048, block_size=512)
+    Q, K, V = W.qkv(w)
+    pidx, plen = W.first_k_prefix(w)
+    plen = np.asarray([0, plen[3], 0, plen[1]], np.int32)      # only indices below 512 are used by block 1
+    pidx = pidx.copy()
+    pidx[:] = np.arange(len(pidx)) % 512                       # all entries lie in block 0
+    print(run_phase1(w, Q, K, V, pidx, plen, what="non-monotone"))

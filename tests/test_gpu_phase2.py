@@ -96,3 +96,14 @@ def test_phase1_then_phase2_chain_on_retained_kv():
     O, LSE = binding.pulsar_phase2_attn(Qq.to(DEV), Kr, Vr, w.n_blocks, w.block_size)
     Oref, Lref = oracle.phase2_attn(Qq, K, V, w.n_blocks, w.block_size)
     check_attention(O, LSE, Oref, Lref, "chain")
+
+
+def test_two_runs_are_bit_identical():
+    w = W.CONFIGS["16k"]
+    _, K, V = W.qkv(w)
+    Qq = W.phase2_query(w).to(DEV)
+    Kd, Vd = K.to(DEV), V.to(DEV)
+    a = binding.pulsar_phase2_attn(Qq, Kd, Vd, w.n_blocks, w.block_size)
+    b = binding.pulsar_phase2_attn(Qq, Kd, Vd, w.n_blocks, w.block_size)
+    torch.cuda.synchronize()
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
