@@ -143,7 +143,7 @@ def maxidf_select_workspace_bytes(L, vocab_size, block_size, chunk, k, sink) -> 
 
 def pulsar_maxidf_select(token_ids: torch.Tensor, vocab_size: int, block_size: int, chunk: int, k: int,
                          sink: int, want_df: bool = False, want_idf: bool = False, workspace=None,
-                         status=None):
+                         status=None, out=None):
     """Max-IDF summary selection.  ``token_ids``: CUDA int32 [L] holding the uint32 ids.
     Returns a dict of CUDA tensors: sel_chunks [B,k], prefix_idx, prefix_len [B] (+ df, idf)."""
     lib = load_library()
@@ -151,9 +151,13 @@ def pulsar_maxidf_select(token_ids: torch.Tensor, vocab_size: int, block_size: i
     L = token_ids.numel()
     dev = token_ids.device
     B = L // block_size if block_size > 0 else 0
-    sel_buf = torch.empty(max(B, 0) * max(k, 0) + 4, dtype=torch.int32, device=dev)
-    pidx = torch.empty(max(sink, 0) + max(B - 1, 0) * max(k, 0) * max(chunk, 0) + 4, dtype=torch.int32, device=dev)
-    plen = torch.empty(max(B, 1), dtype=torch.int32, device=dev)
+    if out is not None:                  # (sel_buf, prefix_idx, prefix_len) preallocated by the caller
+        sel_buf, pidx, plen = out
+    else:
+        sel_buf = torch.empty(max(B, 0) * max(k, 0) + 4, dtype=torch.int32, device=dev)
+        pidx = torch.empty(max(sink, 0) + max(B - 1, 0) * max(k, 0) * max(chunk, 0) + 4, dtype=torch.int32,
+                           device=dev)
+        plen = torch.empty(max(B, 1), dtype=torch.int32, device=dev)
     df = torch.empty(vocab_size, dtype=torch.int32, device=dev) if want_df else None
     idf = torch.empty(vocab_size, dtype=torch.float32, device=dev) if want_idf else None
     if workspace is None:
@@ -195,7 +199,8 @@ def phase1_workspace_bytes(L, Hq, Hkv, d, block_size, prefix_total) -> int:
 
 
 def pulsar_phase1_attn(Q, K, V, block_size: int, prefix_idx, prefix_len, softmax_scale: float = 0.0,
-                       want_lse: bool = True, retain_copy: bool = False, out=None, workspace=None, status=None):
+                       want_lse: bool = True, retain_copy: bool = False, out=None, lse_out=None, workspace=None,
+                       status=None):
     """Phase-1 prefix-block attention.  Q [L,Hq,d], K,V [L,Hkv,d] CUDA bf16; prefix_idx,
     prefix_len CUDA int32.  Returns (O bf16 [L,Hq,d], LSE f32 [L,Hq] or None, K_ret, V_ret)."""
     lib = load_library()
@@ -208,7 +213,8 @@ def pulsar_phase1_attn(Q, K, V, block_size: int, prefix_idx, prefix_len, softmax
     dev = Q.device
     prefix_total = prefix_idx.numel()
     O = torch.empty_like(Q) if out is None else out
-    LSE = torch.empty((L, Hq), dtype=torch.float32, device=dev) if want_lse else None
+    LSE = lse_out if lse_out is not None else (
+        torch.empty((L, Hq), dtype=torch.float32, device=dev) if want_lse else None)
     K_ret = torch.empty_like(K) if retain_copy else None
     V_ret = torch.empty_like(V) if retain_copy else None
     if workspace is None:
@@ -232,7 +238,8 @@ def phase2_workspace_bytes(nq, B, block_size, Hq, Hkv, d, n_splits=0) -> int:
 
 
 def pulsar_phase2_attn(Qq, Kblocks, Vblocks, n_blocks: int, block_size: int, softmax_scale: float = 0.0,
-                       n_splits: int = 0, want_partials: bool = False, out=None, workspace=None, status=None):
+                       n_splits: int = 0, want_partials: bool = False, out=None, lse_out=None, workspace=None,
+                       status=None):
     """Phase-2 query attention with exact LSE merge.  Qq [nq,Hq,d], K/V [n_blocks*block_size,Hkv,d]
     CUDA bf16.  Returns (O bf16 [nq,Hq,d], LSE f32 [nq,Hq]) and, with ``want_partials``
     (needs n_splits > 0), also (part_O f32 [J,nq,Hq,d], part_LSE f32 [J,nq,Hq])."""
@@ -243,7 +250,7 @@ def pulsar_phase2_attn(Qq, Kblocks, Vblocks, n_blocks: int, block_size: int, sof
     Hkv = Kblocks.shape[-2]
     dev = Qq.device
     O = torch.empty_like(Qq) if out is None else out
-    LSE = torch.empty((nq, Hq), dtype=torch.float32, device=dev)
+    LSE = lse_out if lse_out is not None else torch.empty((nq, Hq), dtype=torch.float32, device=dev)
     pO = pL = None
     if want_partials:
         pO = torch.empty((n_splits, nq, Hq, d), dtype=torch.float32, device=dev)

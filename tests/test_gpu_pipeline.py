@@ -1,0 +1,45 @@
+"""The step wrappers: device-resident, host buffers in order, host buffers pipelined -- same results."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2607_20457_b200 import workloads as W
+from paper_2607_20457_b200.pipeline import ContextEncoder
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def test_host_and_pipelined_steps_equal_the_device_step_and_the_oracle_selection():
+    w = W.shrink(W.CONFIGS["tiny"], L=2048, block_size=512, nq=16)
+    ids = W.needle_ids(w)
+    Q, K, V = W.qkv(w)
+    Qq = W.phase2_query(w)
+    enc = ContextEncoder(w, DEV, slots=2)
+    h = enc.host_buffers()
+    h["ids"].copy_(torch.from_numpy(ids.view(np.int32)))
+    h["Q"].copy_(Q); h["K"].copy_(K); h["V"].copy_(V); h["Qq"].copy_(Qq)
+    dev_in = [h[n].to(DEV) for n in ("ids", "Q", "K", "V", "Qq")]
+    ref = enc.step_device(*dev_in)
+    ref = {k: ref[k].clone() for k in ("O1", "LSE1", "O2", "LSE2", "prefix_idx")}
+    torch.cuda.synchronize()
+    sel = oracle.maxidf_select(ids, w.vocab_size, w.block_size, w.chunk, w.k, w.sink)
+    np.testing.assert_array_equal(ref["prefix_idx"].cpu().numpy(), sel["prefix_idx"])
+
+    h2d, d2h = enc.step_host(h)
+    torch.cuda.synchronize()
+    assert h2d == sum(h[n].numel() * h[n].element_size() for n in ("ids", "Q", "K", "V", "Qq"))
+    for k, v in ref.items():
+        assert torch.equal(h[k], v.cpu()), k
+
+    outs = [enc.host_buffers(), enc.host_buffers()]
+    for o in outs:
+        for k in ref:
+            o[k].zero_()
+    enc.run_host_pipelined(h, outs, 5)
+    torch.cuda.synchronize()
+    for o in outs:
+        for k, v in ref.items():
+            assert torch.equal(o[k], v.cpu()), k
+    assert int(enc.status.item()) == 0
