@@ -348,6 +348,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             bool ok = true;
             volatile int* item_q = reinterpret_cast<volatile int*>(smem + SL::kItemQ);
             for (uint32_t seq = 0; ok; ++seq) {
+                // Reconverge once per iteration: every barrier is waited on at most once per
+                // iteration, so a lane that is still polling can never be more than one phase behind
+                // the lanes that went ahead (two phases behind, its parity test would read "not yet"
+                // again and it would stall until the bound expires).
+                __syncwarp();
                 // Next work item: drawn from the global counter (phase 1: items differ in cost, so
                 // they are handed out as CTAs become free) or the fixed round order (phase 2).
                 // It is published through a small queue for the MMA issuer and the softmax warps.
@@ -383,6 +388,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                     if (leader) tma_load_3d_a(q_smem + p * kPanelBytes, &tmQ, bar0 + 8 * (SL::bQFull + 0), p * 64, it.head0,
                                   it.token0_a);
                 for (int t = 0; t < it.n_load && ok; ++t) {
+                    __syncwarp();
                     const bool pref = t < it.n_pref_tiles;
                     const int row = pref ? t * kTileN : it.main_row0 + (t - it.n_pref_tiles) * kTileN;
                     // K_t
@@ -468,6 +474,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
 
             volatile int* item_q = reinterpret_cast<volatile int*>(smem + SL::kItemQ);
             for (uint32_t seq = 0; ok; ++seq) {
+                __syncwarp();              // see the loader: lanes stay within one barrier phase of each other
                 const uint32_t slot = seq % kItemQueue;
                 ok = mbar_wait_a(bar0 + 8 * (SL::bItemFull + slot), (seq / kItemQueue) & 1, abort_flag, a.status);
                 if (!ok) break;
@@ -495,6 +502,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 }
                 if (leader) umma_commit_a(bar0 + 8 * (SL::bKvEmpty + ks));
                 for (int t = 0; t < it.n_load; ++t) {
+                    __syncwarp();
                     const uint32_t vs = stage, vp = phase;                 // V_t
                     PULSAR_RING_NEXT(stage, phase);
                     const bool more = t + 1 < it.n_load;
