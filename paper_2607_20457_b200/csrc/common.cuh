@@ -159,7 +159,7 @@ __device__ __forceinline__ void umma_commit_a(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-// ---- TMA (tiled bulk tensor copies, no multicast) ------------------------------------------
+// ---- TMA (tiled bulk tensor copies, each CTA loads its own tiles) ------------------------------------------
 __device__ __forceinline__ void tma_prefetch_desc(const void* tmap) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
 }
