@@ -192,9 +192,11 @@ int32_t pulsar_phase1_attn(const uint16_t *Q, const uint16_t *K, const uint16_t 
  *
  *   Qq          in  [nq, Hq, d] bf16 (a batch of queries is flattened into nq rows)
  *   Kblocks, Vblocks in [B, block_size, Hkv, d] bf16 (the retained rows, i.e. [L, Hkv, d])
- *   n_splits    number of KV parts: 0 = let the library choose; otherwise 1 <= n_splits,
- *               and (B*block_size) % n_splits == 0.  n_splits == B gives the per-block
- *               (A_h, l_h) of Algorithm 1 line 12.
+ *   n_splits    number of KV parts: 0 = let the library choose, otherwise >= 1.  If n_splits
+ *               divides the B*block_size keys, every part has that many keys (n_splits == B
+ *               gives the per-block (A_h, l_h) of Algorithm 1 line 12); if not, the parts are
+ *               whole 128-key tiles, ceil(tiles / n_splits) each, the last one shorter, and a
+ *               count that would leave a part empty is rejected.
  *   O           out [nq, Hq, d] bf16        LSE out [nq, Hq] float32 (natural log), or NULL
  *   part_O      out [n_splits, nq, Hq, d] float32 or NULL (requires n_splits > 0)
  *   part_LSE    out [n_splits, nq, Hq]    float32 or NULL (both or neither)

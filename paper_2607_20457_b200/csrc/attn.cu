@@ -37,7 +37,8 @@ struct AttnArgs {
     int tiles_per_block;   // phase 1: ceil(block_size / 128)
     int prefix_total;      // phase 1: rows in the gathered prefix buffers
     const int32_t* prefix_len;
-    int split_len;         // phase 2: keys per KV part
+    int split_len;         // phase 2: keys per KV part (the last part may be shorter)
+    int kv_len;            // phase 2: context keys in total
     int n_ctx_parts;       // phase 2: parts of the context KV; part n_ctx_parts (if any) is the generation shard
     int gen_len;           // phase 2: rows of the generation shard that precede the new tokens
     int gen_total;         // phase 2: gen_len + new tokens (0 = no generation shard)
@@ -221,9 +222,9 @@ __device__ __forceinline__ void decode_item(const AttnArgs& a, int idx, Item& it
             it.pref_len = 0;
             it.n_pref_tiles = 0;
             it.main_row0 = it.part * a.split_len;
-            it.main_len = a.split_len;
+            it.main_len = min(a.split_len, a.kv_len - it.main_row0);
             it.gen_base = -1;
-            n = (a.split_len + kTileN - 1) / kTileN;
+            n = (it.main_len + kTileN - 1) / kTileN;
         }
         it.n_tiles_a = n;
         it.n_tiles_b = it.has1 ? n : 0;
@@ -836,8 +837,8 @@ int32_t plan_phase1(int64_t L, int32_t Hq, int32_t Hkv, int32_t d, int32_t block
     return PULSAR_OK;
 }
 
-// Number of KV parts for Phase 2 when the caller leaves the choice to the library: the divisor
-// J of the key-tile count that minimises a simple time model --
+// Number of KV parts for Phase 2 when the caller leaves the choice to the library: the J that
+// minimises a simple time model --
 //   rounds(J) * (tiles per part * t_tile + t_item)  +  partial traffic(J) / HBM bandwidth,
 // rounds = ceil(items / CTAs).  More parts fill the last round better and shorten it, but every
 // part writes and re-reads fp32 partials.  Constants are measured on B200 (one pair of query
@@ -846,19 +847,30 @@ int32_t choose_splits(int32_t nq, int64_t L, int32_t Hq, int32_t Hkv, int32_t d)
     const int g = Hq / Hkv;
     const int64_t row_tiles = (static_cast<int64_t>(nq) * g + kTileM - 1) / kTileM;
     const int64_t items = (row_tiles + 1) / 2 * Hkv;               // a work item is a pair of row tiles
-    if (L % kTileN != 0) return 1;
-    const int64_t kv_tiles = L / kTileN;
+    const int64_t kv_tiles = (L + kTileN - 1) / kTileN;
     const double ctas = sm_count(), t_tile_us = 2.0, t_item_us = 6.0, hbm_bytes_per_us = 6.0e6;
     double best_t = 0;
     int64_t best = 1;
     for (int64_t j = 1; j <= kv_tiles && j <= 1024; ++j) {
-        if (kv_tiles % j != 0) continue;
+        const int64_t tiles_per_part = (kv_tiles + j - 1) / j;
+        if ((kv_tiles + tiles_per_part - 1) / tiles_per_part != j) continue;      // some part would be empty
         const double rounds = static_cast<double>((items * j + static_cast<int64_t>(ctas) - 1) / static_cast<int64_t>(ctas));
         const double partial = j > 1 ? 2.0 * j * nq * Hq * (d + 1) * 4.0 / hbm_bytes_per_us : 0.0;
-        const double t = rounds * (static_cast<double>(kv_tiles / j) * t_tile_us + t_item_us) + partial;
+        const double t = rounds * (static_cast<double>(tiles_per_part) * t_tile_us + t_item_us) + partial;
         if (best_t == 0 || t < best_t) { best_t = t; best = j; }
     }
     return static_cast<int32_t>(best);
+}
+
+// Keys per KV part: L / n_splits when that divides; otherwise the parts are whole 128-key tiles,
+// ceil(tiles / n_splits) each, the last one shorter.  0 if some part would be empty.
+int64_t phase2_split_len(int64_t L, int32_t n_splits) {
+    if (n_splits <= 0) return 0;
+    if (L % n_splits == 0) return L / n_splits;
+    const int64_t kv_tiles = (L + kTileN - 1) / kTileN;
+    const int64_t tiles_per_part = (kv_tiles + n_splits - 1) / n_splits;
+    if ((kv_tiles + tiles_per_part - 1) / tiles_per_part != n_splits) return 0;
+    return tiles_per_part * kTileN;
 }
 
 }  // namespace
@@ -962,7 +974,7 @@ int32_t plan_phase2(int32_t nq, int32_t B, int32_t block_size, int32_t Hq, int32
     const int64_t L = static_cast<int64_t>(B) * block_size;
     if (L >= (1ll << 31) || Hkv > 65535) return PULSAR_ERR_SHAPE;
     if (n_splits == 0) n_splits = choose_splits(nq, L, Hq, Hkv, d);
-    if (L % n_splits != 0 || n_splits > 65535) return PULSAR_ERR_SHAPE;
+    if (n_splits > 65535 || phase2_split_len(L, n_splits) == 0) return PULSAR_ERR_SHAPE;
     part_o_bytes = round_up(static_cast<size_t>(n_splits) * nq * Hq * d * 4, 256);
     part_l_bytes = round_up(static_cast<size_t>(n_splits) * nq * Hq * 4, 256);
     return PULSAR_OK;
@@ -1024,7 +1036,8 @@ extern "C" int32_t pulsar_phase2_attn(const uint16_t* Qq, int32_t nq, const uint
     a.Hq = Hq;
     a.g = g;
     a.pack = g;
-    a.split_len = static_cast<int>(L / n_splits);
+    a.split_len = static_cast<int>(phase2_split_len(L, n_splits));
+    a.kv_len = static_cast<int>(L);
     a.n_ctx_parts = n_splits;
     a.scale_log2 = (softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf(static_cast<float>(d))) * 1.4426950408889634f;
     a.O = O;
@@ -1107,7 +1120,8 @@ extern "C" int32_t pulsar_phase2_generate_step(const uint16_t* Qnew, const uint1
     a.Hq = Hq;
     a.g = g;
     a.pack = g;
-    a.split_len = static_cast<int>(L / n_splits);
+    a.split_len = static_cast<int>(phase2_split_len(L, n_splits));
+    a.kv_len = static_cast<int>(L);
     a.n_ctx_parts = n_splits;
     a.gen_len = gen_len;
     a.gen_total = gen_len + n_new;

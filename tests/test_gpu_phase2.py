@@ -107,3 +107,20 @@ def test_two_runs_are_bit_identical():
     b = binding.pulsar_phase2_attn(Qq, Kd, Vd, w.n_blocks, w.block_size)
     torch.cuda.synchronize()
     assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+
+
+@pytest.mark.parametrize("n_splits", [3, 6])
+def test_uneven_parts(n_splits):
+    # 2048 keys = 16 key tiles cut into runs of whole tiles, the last run shorter: 6+6+4, 3*5+1
+    w = W.shrink(W.CONFIGS["tiny"], L=2048, block_size=512, Hq=8, Hkv=2, d=128, nq=40)
+    _, K, V = W.qkv(w)
+    print(run_phase2(w, W.phase2_query(w, q_scale=2.0), K, V, n_splits, what=f"uneven J={n_splits}"))
+
+
+def test_part_count_that_leaves_a_part_empty_is_rejected():
+    # 16 key tiles in 5 parts would be runs of 4 tiles: only 4 parts are non-empty
+    w = W.shrink(W.CONFIGS["tiny"], L=2048, block_size=512, Hq=8, Hkv=2, d=128, nq=8)
+    _, K, V = W.qkv(w)
+    with pytest.raises(binding.PulsarError) as e:
+        binding.pulsar_phase2_attn(W.phase2_query(w).to(DEV), K.to(DEV), V.to(DEV), w.n_blocks, w.block_size, n_splits=5)
+    assert e.value.status == 2

@@ -64,9 +64,10 @@ def test_host_validation_launches_nothing(lib):
     args = lambda d, Hq, Hkv: (one, one, one, 4096, Hq, Hkv, d, 1024, one, one, 64, 0.0, one, null, null, null, one, 1 << 30, null, null)
     assert lib.pulsar_phase1_attn(*args(96, 4, 1)) == 2
     assert lib.pulsar_phase1_attn(*args(64, 5, 2)) == 2
-    # phase 2: partial outputs need an explicit split count; n_splits must divide the keys
+    # phase 2: partial outputs need an explicit split count; a split count that would leave a part
+    # empty is rejected (32 key tiles cannot be cut into 31 non-empty runs of whole tiles)
     assert lib.pulsar_phase2_attn(one, 8, one, one, 4, 1024, 4, 1, 64, 0.0, 0, one, null, one, one, one, 1 << 30, null, null) == 1
-    assert lib.pulsar_phase2_attn(one, 8, one, one, 4, 1024, 4, 1, 64, 0.0, 3, one, null, null, null, one, 1 << 30, null, null) == 2
+    assert lib.pulsar_phase2_attn(one, 8, one, one, 4, 1024, 4, 1, 64, 0.0, 31, one, null, null, null, one, 1 << 30, null, null) == 2
     # merge: d must be a multiple of 4
     assert lib.pulsar_lse_merge(one, one, 2, 8, 6, one, null, null) == 2
 
