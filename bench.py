@@ -397,6 +397,22 @@ def run_extras(binding, w, dev, K_d, V_d, peaks):
         t = time_calls(lambda: binding.pulsar_phase1_attn(Q, K, V, w4.block_size, pi, pl, out=O, workspace=ws), 5)
         fl = cm.phase1_flops(w4.block_size, plen, w4.Hq, w4.d)
         res[tag] = dict(ms=t["median_ms"], tflop=fl / 1e12, tflops=fl / (t["median_ms"] * 1e-3) / 1e12)
+    # the same 64K inputs as whole assembled sequences (every token of Input_i a query, Alg. 1 l.8)
+    pidx, plen = W.first_k_prefix(w4)
+    cu = [0]
+    rows = []
+    for i in range(w4.n_blocks):
+        rows += list(pidx[: plen[i]]) + list(range(i * w4.block_size, (i + 1) * w4.block_size))
+        cu.append(len(rows))
+    sel_rows = torch.tensor(rows, device=dev)
+    Qa, Ka, Va = Q[sel_rows].contiguous(), K[sel_rows].contiguous(), V[sel_rows].contiguous()
+    Oa = torch.empty_like(Qa)
+    wsa = binding._workspace(256, dev)
+    t = time_calls(lambda: binding.pulsar_causal_varlen_attn(Qa, Ka, Va, cu, out=Oa, workspace=wsa, want_lse=False), 5)
+    pairs = sum((b - a) * (b - a + 1) // 2 for a, b in zip(cu[:-1], cu[1:]))
+    fl = 4 * w4.d * w4.Hq * pairs
+    res["pulsar_assembled_all_rows"] = dict(ms=t["median_ms"], rows=cu[-1], tflop=fl / 1e12,
+                                            tflops=fl / (t["median_ms"] * 1e-3) / 1e12)
     res["flop_ratio_star_over_pulsar"] = res["star_anchor"]["tflop"] / res["pulsar"]["tflop"]
     res["time_ratio_star_over_pulsar"] = res["star_anchor"]["ms"] / res["pulsar"]["ms"]
     out["phase1_64k_prefix_comparison"] = res

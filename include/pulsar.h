@@ -7,6 +7,7 @@
  *   pulsar_phase1_attn     Phase-1 prefix-block attention (Eq. 1 over Input_i of Eq. 4; Alg. 1 l.7-8)
  *   pulsar_phase2_attn     Phase-2 query attention + merge (Section 3.2; Alg. 1 l.12-13; App. H)
  *   pulsar_lse_merge       online-softmax merge alone      (Appendix H, Eq. 12-13)
+ *   pulsar_causal_varlen_attn    causal attention over assembled inputs of any lengths (Alg. 1 l.8)
  *   pulsar_phase2_generate_step  one generation step: append KV(q), attend, merge (Alg. 1 l.11-16)
  *
  * Conventions that hold for every call
@@ -179,6 +180,34 @@ int32_t pulsar_phase1_attn(const uint16_t *Q, const uint16_t *K, const uint16_t 
                            uint16_t *O, float *LSE, uint16_t *K_ret, uint16_t *V_ret,
                            void *workspace, size_t workspace_bytes,
                            int32_t *device_status, void *stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Causal attention over assembled inputs (Algorithm 1 line 8 as the paper runs it; Eq. 1, Eq. 4,
+ * Appendix F).
+ *
+ * In the paper every block's assembled input Input_i = [sink | Sigma_0 .. Sigma_{i-1} | B_i]
+ * goes through the whole model, so above the first layer the prefix tokens have keys and values
+ * of their own per block and are queries as well.  This call is the attention of one layer over
+ * such inputs: n_seq independent sequences of different lengths packed back to back, plain
+ * causal attention inside each (row p of sequence j sees rows cu_seqlens[j] .. p).  The caller
+ * assembles Q, K, V (with pulsar_maxidf_select's prefix list) and afterwards keeps the last
+ * block_size key/value rows of each sequence as the retained KV.
+ *
+ *   Q           in  [total_rows, Hq, d] bf16     K, V in [total_rows, Hkv, d] bf16
+ *   cu_seqlens  in  HOST pointer, [n_seq + 1] int32, cu[0] = 0 < cu[1] < ... < cu[n_seq] = total_rows
+ *               (read before the call returns)
+ *   O           out [total_rows, Hq, d] bf16     LSE out [total_rows, Hq] float32 or NULL
+ *   workspace   256 bytes (the work counter)
+ *
+ * Requirements (else PULSAR_ERR_SHAPE): d in {64,128}; Hq % Hkv == 0; 1 <= n_seq <= 64;
+ * total_rows < 2^31.
+ * ------------------------------------------------------------------------------------------ */
+int32_t pulsar_causal_varlen_attn(const uint16_t *Q, const uint16_t *K, const uint16_t *V,
+                                  int64_t total_rows, const int32_t *cu_seqlens /* host */, int32_t n_seq,
+                                  int32_t Hq, int32_t Hkv, int32_t d, float softmax_scale,
+                                  uint16_t *O, float *LSE,
+                                  void *workspace, size_t workspace_bytes,
+                                  int32_t *device_status, void *stream);
 
 /* ------------------------------------------------------------------------------------------
  * Phase-2 query attention over the retained KV of all blocks, merged exactly (Section 3.2;

@@ -13,6 +13,7 @@ Each wrapper names the passage of the paper its C function follows:
 * :func:`phase2_attn`   -- Section 3.2 / Appendix H (single global softmax)
 * :func:`lse_merge`     -- Appendix H Eq. 12-13, iterated
 * :func:`generate_step` -- Algorithm 1 lines 11-16 (append KV(q), attend to context + shard)
+* :func:`causal_varlen_attn` -- Eq. 1 over whole assembled inputs (Algorithm 1 line 8)
 """
 from __future__ import annotations
 
@@ -171,4 +172,18 @@ def generate_step(Qnew, Knew, Vnew, Kctx, Vctx, Kgen_bits, Vgen_bits, gen_len, s
                                       float(scale), _ptr(O), _ptr(LSE))
     if rc != 0:
         raise ValueError(f"oracle_generate_step rejected its arguments (rc={rc})")
+    return O, LSE
+
+
+def causal_varlen_attn(Q, K, V, cu_seqlens, scale=0.0):
+    """Causal attention inside each of the sequences packed back to back (Eq. 1 over every
+    assembled input of Eq. 4, all rows as queries).  Each sequence is one block without a
+    prefix.  Q [T,Hq,d], K,V [T,Hkv,d] bf16.  Returns (O [T,Hq,d], LSE [T,Hq]) float64."""
+    q, kk, v = _bits(Q), _bits(K), _bits(V)
+    T, Hq, d = q.shape
+    O = np.zeros((T, Hq, d), np.float64)
+    LSE = np.zeros((T, Hq), np.float64)
+    none = np.zeros(0, np.int32)
+    for a, b in zip(cu_seqlens[:-1], cu_seqlens[1:]):
+        O[a:b], LSE[a:b] = phase1_attn(q[a:b], kk[a:b], v[a:b], b - a, none, np.zeros(1, np.int32), scale)
     return O, LSE

@@ -28,7 +28,7 @@ EXPORTS = (
     "pulsar_status_string", "pulsar_abi_version", "pulsar_launch_count", "pulsar_wait_selftest",
     "pulsar_maxidf_select_workspace_bytes", "pulsar_maxidf_select",
     "pulsar_maxidf_select_noalloc_max_scratch", "pulsar_maxidf_select_noalloc",
-    "pulsar_phase1_workspace_bytes", "pulsar_phase1_attn",
+    "pulsar_phase1_workspace_bytes", "pulsar_phase1_attn", "pulsar_causal_varlen_attn",
     "pulsar_phase2_choose_splits", "pulsar_phase2_workspace_bytes", "pulsar_phase2_attn",
     "pulsar_phase2_generate_workspace_bytes", "pulsar_phase2_generate_step",
     "pulsar_lse_merge",
@@ -82,6 +82,8 @@ def load_library(build_if_missing: bool = False):
     lib.pulsar_phase1_attn.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, vp, vp, i32, f32,
                                        vp, vp, vp, vp, vp, sz, vp, vp]
     lib.pulsar_phase1_attn.restype = i32
+    lib.pulsar_causal_varlen_attn.argtypes = [vp, vp, vp, i64, vp, i32, i32, i32, i32, f32, vp, vp, vp, sz, vp, vp]
+    lib.pulsar_causal_varlen_attn.restype = i32
     lib.pulsar_phase2_choose_splits.argtypes = [i32, i32, i32, i32, i32, i32]
     lib.pulsar_phase2_choose_splits.restype = i32
     lib.pulsar_phase2_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, i32, i32]
@@ -227,6 +229,28 @@ def pulsar_phase1_attn(Q, K, V, block_size: int, prefix_idx, prefix_len, softmax
     if not retain_copy:
         K_ret, V_ret = K, V          # the retained KV is the block's own rows of K and V
     return O, LSE, K_ret, V_ret
+
+
+def pulsar_causal_varlen_attn(Q, K, V, cu_seqlens, softmax_scale: float = 0.0, want_lse: bool = True, out=None,
+                              workspace=None, status=None):
+    """Causal attention over sequences packed back to back (the assembled Phase-1 inputs of the
+    paper's whole-model pass).  Q [T,Hq,d], K,V [T,Hkv,d] CUDA bf16; cu_seqlens: host sequence of
+    n_seq+1 ascending row offsets.  Returns (O bf16 [T,Hq,d], LSE f32 [T,Hq] or None)."""
+    lib = load_library()
+    for t, n in ((Q, "Q"), (K, "K"), (V, "V")):
+        _need(t, torch.bfloat16, n)
+    T, Hq, d = Q.shape
+    Hkv = K.shape[1]
+    cu = (ctypes.c_int32 * len(cu_seqlens))(*[int(x) for x in cu_seqlens])
+    O = torch.empty_like(Q) if out is None else out
+    LSE = torch.empty((T, Hq), dtype=torch.float32, device=Q.device) if want_lse else None
+    if workspace is None:
+        workspace = _workspace(256, Q.device)
+    rc = lib.pulsar_causal_varlen_attn(_p(Q), _p(K), _p(V), T, ctypes.cast(cu, ctypes.c_void_p), len(cu_seqlens) - 1,
+                                       Hq, Hkv, d, float(softmax_scale), _p(O), _p(LSE), _p(workspace),
+                                       workspace.numel(), _p(status), _stream())
+    _check("pulsar_causal_varlen_attn", rc)
+    return O, LSE
 
 
 def phase2_choose_splits(nq, B, block_size, Hq, Hkv, d) -> int:

@@ -27,7 +27,15 @@ constexpr int kTileM = 128;   // query rows per CTA
 constexpr int kTileN = 128;   // keys per tile
 constexpr int kPanelBytes = kTileN * 128;   // one 64-column panel of a 128-row bf16 tile (128-byte lines)
 
-enum : int { kModePhase1 = 0, kModePhase2 = 1 };
+enum : int { kModePhase1 = 0, kModePhase2 = 1, kModeVarlen = 2 };
+
+// Sequence table of the variable-length causal mode (passed by value with the launch).
+constexpr int kMaxVarlenSeqs = 64;
+struct VarlenTable {
+    int start[kMaxVarlenSeqs + 1];      // first row of sequence j; start[n] = total rows
+    int pair_cum[kMaxVarlenSeqs + 1];   // tile pairs of the sequences n-1, n-2, ... j summed (scheduling order)
+    int n_seq;
+};
 
 struct AttnArgs {
     int mode;
@@ -169,8 +177,36 @@ __device__ __forceinline__ int item_of_round(int round, int n_items) {
     return idx < n_items ? idx : -1;
 }
 
-__device__ __forceinline__ void decode_item(const AttnArgs& a, int idx, Item& it) {
-    if (a.mode == kModePhase1) {
+__device__ __forceinline__ void decode_item(const AttnArgs& a, const VarlenTable& vt, int idx, Item& it) {
+    if (a.mode == kModeVarlen) {
+        // Independent sequences of different lengths, plain causal attention inside each.
+        // Items run from the last sequence down and, inside a sequence, from its last tile
+        // pair down (for assembled Pulsar inputs the later blocks are the longer ones).
+        const int rank = idx / a.Hq;
+        it.head0 = idx - rank * a.Hq;
+        it.kvh = it.head0 / a.g;
+        it.part = 0;
+        int k = 0;                                             // k-th sequence from the end
+        while (k + 1 < vt.n_seq && vt.pair_cum[k + 1] <= rank) ++k;
+        const int seq = vt.n_seq - 1 - k;
+        const int start = vt.start[seq], len = vt.start[seq + 1] - start;
+        const int tiles = (len + kTileM - 1) / kTileM, pairs = (tiles + 1) / 2;
+        const int pair = pairs - 1 - (rank - vt.pair_cum[k]);
+        const int qt0 = 2 * pair;
+        it.has1 = (qt0 + 1 < tiles) ? 1 : 0;
+        it.row0_a = qt0 * kTileM;
+        it.row0_b = (qt0 + 1) * kTileM;
+        it.token0_a = start + it.row0_a;
+        it.token0_b = start + it.row0_b;
+        it.bad_length = 0;
+        it.pref_len = 0;
+        it.n_pref_tiles = 0;
+        it.main_row0 = start;
+        it.main_len = len;
+        it.gen_base = -1;
+        it.n_tiles_a = qt0 + 1;
+        it.n_tiles_b = it.has1 ? qt0 + 2 : 0;
+    } else if (a.mode == kModePhase1) {
         // Items run block-major from the last block (longest prefix) down and, within a block,
         // from the last tile pair (most causal tiles) down; the heads of one (block, pair) are
         // adjacent.  CTAs that run at the same time therefore read the same K/V rows (L2 hits),
@@ -280,7 +316,8 @@ template <int D>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
             const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmKp,
-            const __grid_constant__ CUtensorMap tmVp, const AttnArgs a) {
+            const __grid_constant__ CUtensorMap tmVp, const AttnArgs a,
+            const __grid_constant__ VarlenTable vt) {
     using SL = SmemLayout<D>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -376,7 +413,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 }
                 if (idx < 0) break;
                 Item it;
-                decode_item(a, idx, it);
+                decode_item(a, vt, idx, it);
                 if (it.bad_length && lane == 0) report(a.status, PULSAR_DEV_BAD_LENGTH);
                 const int x = it.kvh * D;
                 // query tile 0
@@ -483,7 +520,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 if (leader) mbar_arrive(bars + SL::bItemEmpty + slot);
                 if (idx < 0) break;
                 Item it;
-                decode_item(a, idx, it);
+                decode_item(a, vt, idx, it);
                 const int n0 = it.n_tiles_a, n1 = it.n_tiles_b;
                 // K_0
                 uint32_t ks = stage, kp = phase;
@@ -585,7 +622,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             if (lane == 0) mbar_arrive(bars + SL::bItemEmpty + slot);
             if (idx < 0) break;
             Item it;
-            decode_item(a, idx, it);
+            decode_item(a, vt, idx, it);
             const int n = s ? it.n_tiles_b : it.n_tiles_a;
             if (n == 0) continue;
             float m_used = -INFINITY, l_run = 0.f;
@@ -607,7 +644,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                     const int j = t - it.n_pref_tiles;
                     const int valid = it.main_len - j * kTileN;
                     if (valid < kTileN) { n_vis = valid; masked = true; }
-                    if (a.mode == kModePhase1 && t == n - 1) {
+                    if (a.mode != kModePhase2 && t == n - 1) {
                         n_vis = min(n_vis, my_row_in_block - j * kTileN + 1);
                         masked = true;
                     }
@@ -705,7 +742,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 const int token = (s ? it.token0_b : it.token0_a) + row / a.pack;
                 const int head = it.head0 + row % a.pack;
                 bool store = token < a.n_tokens;
-                if (a.mode == kModePhase1) store = store && my_row_in_block < a.block_size;
+                if (a.mode != kModePhase2) store = store && my_row_in_block < it.main_len;
                 const float inv_l = l_run > 0.f ? 1.f / l_run : 0.f;
                 const float lse = (l_run > 0.f) ? (m_used + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
                 const size_t orow = static_cast<size_t>(token) * a.Hq + head;
@@ -803,14 +840,16 @@ bool make_map_2d(CUtensorMap* m, const void* base, int64_t rows, int64_t width) 
 
 template <int D>
 int32_t launch_attn(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& v, const CUtensorMap& kp,
-                    const CUtensorMap& vp, const AttnArgs& a, cudaStream_t stream) {
+                    const CUtensorMap& vp, const AttnArgs& a, cudaStream_t stream,
+                    const VarlenTable* table = nullptr) {
     constexpr int smem = SmemLayout<D>::kDynBytes;
     // The opt-in to more than 48 KB of dynamic shared memory is a per-device function attribute;
     // setting it on every launch keeps multi-device processes correct and costs well under a microsecond.
     PULSAR_CUDA_OK(cudaFuncSetAttribute(attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     const int grid = a.n_items < sm_count() ? a.n_items : sm_count();     // one persistent CTA per SM
     if (grid <= 0) return PULSAR_OK;
-    attn_kernel<D><<<grid, kAttnThreads, smem, stream>>>(q, k, v, kp, vp, a);
+    static const VarlenTable kNoTable{};
+    attn_kernel<D><<<grid, kAttnThreads, smem, stream>>>(q, k, v, kp, vp, a, table ? *table : kNoTable);
     PULSAR_CUDA_OK(cudaGetLastError());
     count_launch();
     return PULSAR_OK;
@@ -1140,4 +1179,66 @@ extern "C" int32_t pulsar_phase2_generate_step(const uint16_t* Qnew, const uint1
                   : launch_attn<64>(tmQ, tmK, tmV, tmKg, tmVg, a, stream);
     if (rc != PULSAR_OK) return rc;
     return launch_lse_merge(pO, pL, n_parts, static_cast<int64_t>(n_new) * Hq, d, O, LSE, stream);
+}
+
+// =============================================================================================
+// Causal attention over assembled inputs of different lengths (Algorithm 1 line 8 as the paper
+// runs it: every token of Input_i is a query, the keys and values are those of Input_i itself)
+// =============================================================================================
+extern "C" int32_t pulsar_causal_varlen_attn(const uint16_t* Q, const uint16_t* K, const uint16_t* V,
+                                             int64_t total_rows, const int32_t* cu_seqlens_host, int32_t n_seq,
+                                             int32_t Hq, int32_t Hkv, int32_t d, float softmax_scale, uint16_t* O,
+                                             float* LSE, void* workspace, size_t workspace_bytes,
+                                             int32_t* device_status, void* stream_) {
+    if (total_rows <= 0 || n_seq <= 0 || Hq <= 0 || Hkv <= 0 || !cu_seqlens_host) return PULSAR_ERR_INVALID_ARG;
+    if ((d != 64 && d != 128) || Hq % Hkv != 0 || total_rows >= (1ll << 31) || n_seq > kMaxVarlenSeqs || Hq > 65535)
+        return PULSAR_ERR_SHAPE;
+    if (cu_seqlens_host[0] != 0 || cu_seqlens_host[n_seq] != total_rows) return PULSAR_ERR_SHAPE;
+    for (int j = 0; j < n_seq; ++j)
+        if (cu_seqlens_host[j + 1] <= cu_seqlens_host[j]) return PULSAR_ERR_SHAPE;       // empty or descending
+    if (!Q || !K || !V || !O || !workspace) return PULSAR_ERR_INVALID_ARG;
+    if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) || (LSE && !aligned(LSE, 4)) ||
+        !aligned(workspace, 256))
+        return PULSAR_ERR_ALIGNMENT;
+    if (workspace_bytes < 256) return PULSAR_ERR_WORKSPACE;
+    int32_t rc = check_device();
+    if (rc != PULSAR_OK) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+
+    VarlenTable vt{};
+    vt.n_seq = n_seq;
+    for (int j = 0; j <= n_seq; ++j) vt.start[j] = cu_seqlens_host[j];
+    int64_t pairs_total = 0;
+    for (int k = 0; k < n_seq; ++k) {
+        vt.pair_cum[k] = static_cast<int>(pairs_total);
+        const int len = vt.start[n_seq - k] - vt.start[n_seq - 1 - k];
+        pairs_total += ((len + kTileM - 1) / kTileM + 1) / 2;
+    }
+    vt.pair_cum[n_seq] = static_cast<int>(pairs_total);
+    if (pairs_total * Hq >= (1ll << 31)) return PULSAR_ERR_SHAPE;
+
+    CUtensorMap tmQ, tmK, tmV;
+    if (!make_map_3d(&tmQ, Q, total_rows, Hq, d, 1, kTileM) ||
+        !make_map_2d(&tmK, K, total_rows, static_cast<int64_t>(Hkv) * d) ||
+        !make_map_2d(&tmV, V, total_rows, static_cast<int64_t>(Hkv) * d))
+        return PULSAR_ERR_CUDA;
+
+    int32_t* counter = static_cast<int32_t*>(workspace);
+    PULSAR_CUDA_OK(cudaMemsetAsync(counter, 0, sizeof(int32_t), stream));
+
+    AttnArgs a{};
+    a.mode = kModeVarlen;
+    a.n_tokens = static_cast<int>(total_rows);
+    a.Hq = Hq;
+    a.g = Hq / Hkv;
+    a.pack = 1;
+    a.Hkv = Hkv;
+    a.n_items = static_cast<int>(pairs_total) * Hq;
+    a.counter = counter;
+    a.scale_log2 = (softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf(static_cast<float>(d))) * 1.4426950408889634f;
+    a.O = O;
+    a.LSE = LSE;
+    a.status = device_status;
+    return d == 128 ? launch_attn<128>(tmQ, tmK, tmV, tmK, tmV, a, stream, &vt)
+                    : launch_attn<64>(tmQ, tmK, tmV, tmK, tmV, a, stream, &vt);
 }

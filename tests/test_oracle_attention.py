@@ -257,3 +257,17 @@ def test_generate_step_is_one_softmax_over_context_and_causal_shard():
     O2, L2 = oracle.phase2_attn(Qn, torch.cat([K, Kn]), torch.cat([V, Vn]), 1, w.L + 1)
     np.testing.assert_allclose(O1, O2, atol=1e-12)
     np.testing.assert_allclose(L1, L2, atol=1e-12)
+
+
+def test_varlen_causal_is_library_causal_attention_per_sequence():
+    w = small_workload()
+    Q, K, V = W.qkv(w)
+    cu = [0, 37, 101, 256]
+    O, LSE = oracle.causal_varlen_attn(Q, K, V, cu)
+    g = w.Hq // w.Hkv
+    for a, b in zip(cu[:-1], cu[1:]):
+        q = Q[a:b].to(torch.float64).permute(1, 0, 2)[None]
+        k = K[a:b].to(torch.float64).repeat_interleave(g, dim=1).permute(1, 0, 2)[None]
+        v = V[a:b].to(torch.float64).repeat_interleave(g, dim=1).permute(1, 0, 2)[None]
+        ref = torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True)[0]
+        np.testing.assert_allclose(O[a:b], ref.permute(1, 0, 2).numpy(), rtol=0, atol=1e-12)
