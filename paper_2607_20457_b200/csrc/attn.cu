@@ -106,6 +106,9 @@ gather_prefix_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V, c
 // P_s (bf16 pairs) overwrites the first 64 columns of S_s.  The running maximum is only moved
 // when it grows by more than 2^8 (the stale maximum is used consistently for P, O and the row
 // sum, so the result is unchanged); the rare rescale of O is done by the softmax warpgroup.
+// P goes to the issuer in two halves of 64 keys (two barriers), so the first half of PV runs while
+// the second half of the row is exponentiated.  The loader publishes the CTA's work items through
+// a small shared-memory queue; all device waits are bounded (see mbar_wait).
 // ---------------------------------------------------------------------------------------------
 constexpr int kStages = 5;
 constexpr int kItemQueue = 4;     // work items the loader may publish ahead of the slowest consumer
@@ -124,10 +127,6 @@ constexpr float kRescaleThreshold = 8.0f;      // in log2 units
 #define PULSAR_SPECULATE 0
 #endif
 constexpr int kPolyPairs = PULSAR_POLY_PAIRS;  // of every four column pairs, how many use the polynomial exp2
-#ifndef PULSAR_SPLIT_FAST
-#define PULSAR_SPLIT_FAST 1
-#endif
-constexpr bool kSplitFast = PULSAR_SPLIT_FAST;   // fast path hands the first half of P over before forming the second
 constexpr bool kSpeculate = PULSAR_SPECULATE;  // form P with the maximum in use while the tile maximum is computed
 // Registers per thread: the kernel is compiled for 168 (twelve warps).  setmaxnreg moves
 // registers inside the CTA's own pool of 12 * 168 per lane slot and acts on whole warpgroups:
@@ -673,18 +672,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                     const float m_tile = row_max128(r) * a.scale_log2;
                     if (__any_sync(0xffffffffu, m_tile > m_used + kRescaleThreshold)) {
                         exact = true;
-                    } else if (kSplitFast) {
-                        tmem_wait_st();
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(bar_p);
-                        l_run += l_lo + exp_row128<kPolyPairs, 64, 128>(r, a.scale_log2, -m_used, tS);
                     } else {
-                        l_run += l_lo + exp_row128<kPolyPairs, 64, 128>(r, a.scale_log2, -m_used, tS);
                         tmem_wait_st();
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(bar_p);
+                        l_run += l_lo + exp_row128<kPolyPairs, 64, 128>(r, a.scale_log2, -m_used, tS);
                     }
                 }
                 if (exact) {
