@@ -250,6 +250,9 @@ def run_gpu(args, w):
     sel_ms = statistics.mean(m[0].elapsed_time(m[1]) for m in marks)
     p1_ms = statistics.mean(m[1].elapsed_time(m[2]) for m in marks)
     p2_ms = statistics.mean(m[2].elapsed_time(m[3]) for m in marks)
+    p1_all = sorted(m[1].elapsed_time(m[2]) for m in marks)
+    p2_all = sorted(m[2].elapsed_time(m[3]) for m in marks)
+    sel_all = sorted(m[0].elapsed_time(m[1]) for m in marks)
 
     # ---- end to end from pinned host buffers ---------------------------------------------
     # (a) one step at a time, everything in order on one stream (latency of a single call);
@@ -310,6 +313,12 @@ def run_gpu(args, w):
                     cache="inputs (2.5 GiB) larger than the 126 MB L2; no flush needed",
                     sequences_per_gpu=1),
         parts=dict(select_us=sel_ms * 1e3, phase1_ms=p1_ms, phase2_ms=p2_ms,
+                   select_us_median=sel_all[len(sel_all) // 2] * 1e3, select_us_min=sel_all[0] * 1e3,
+                   select_bytes=cm.select_bytes(wl.L, wl.vocab_size, wl.n_blocks, wl.prefix_total, wl.k),
+                   phase1_ms_median=p1_all[len(p1_all) // 2], phase1_ms_min=p1_all[0],
+                   phase2_ms_median=p2_all[len(p2_all) // 2], phase2_ms_min=p2_all[0],
+                   phase2_tensor_floor_ms=p2_flops / (peaks["bf16_burst"] * 1e12) * 1e3,
+                   phase2_hbm_floor_ms=p2_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3,
                    phase1_tokens_per_s=wl.L / (p1_ms * 1e-3),
                    phase1_tflops=achieved_tf, phase1_frac_of_spec_2250=achieved_tf / 2250.0,
                    phase1_frac_of_measured_burst=achieved_tf / peaks["bf16_burst"],
