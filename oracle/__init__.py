@@ -14,6 +14,7 @@ Each wrapper names the passage of the paper its C function follows:
 * :func:`lse_merge`     -- Appendix H Eq. 12-13, iterated
 * :func:`generate_step` -- Algorithm 1 lines 11-16 (append KV(q), attend to context + shard)
 * :func:`causal_varlen_attn` -- Eq. 1 over whole assembled inputs (Algorithm 1 line 8)
+* :func:`chunk_select`  -- Appendix C: TF-IDF, BM25, type-token and Max-IDF chunk scores
 """
 from __future__ import annotations
 
@@ -60,6 +61,8 @@ def _load():
         lib.oracle_generate_step.argtypes = [vp, vp, vp, i32, vp, vp, i64, vp, vp, i32, i32, i32, i32, i32, f64, vp, vp]
         lib.oracle_generate_step.restype = ctypes.c_int
         lib.oracle_lse_merge.restype = ctypes.c_int
+        lib.oracle_chunk_select.argtypes = [vp, i64, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
+        lib.oracle_chunk_select.restype = ctypes.c_int
         _lib = lib
     return _lib
 
@@ -187,3 +190,24 @@ def causal_varlen_attn(Q, K, V, cu_seqlens, scale=0.0):
     for a, b in zip(cu_seqlens[:-1], cu_seqlens[1:]):
         O[a:b], LSE[a:b] = phase1_attn(q[a:b], kk[a:b], v[a:b], b - a, none, np.zeros(1, np.int32), scale)
     return O, LSE
+
+
+SCORE_MODES = {"max_idf": 0, "tf_idf": 1, "bm25": 2, "type_token": 3}
+
+
+def chunk_select(token_ids, vocab_size, block_size, chunk, k, sink, mode):
+    """Chunk selection under one of the Appendix C heuristics (``mode`` a key of SCORE_MODES or
+    its number).  Returns sel_chunks [B,k], prefix_idx, prefix_len and score [B,C] (float64)."""
+    ids = np.ascontiguousarray(np.asarray(token_ids, dtype=np.uint32))
+    L = ids.shape[0]
+    B, C = L // block_size, block_size // chunk
+    m = SCORE_MODES.get(mode, mode)
+    sel = np.zeros((B, k), np.int32)
+    pidx = np.zeros(sink + max(B - 1, 0) * k * chunk, np.int32)
+    plen = np.zeros(B, np.int32)
+    score = np.zeros((B, C), np.float64)
+    rc = _load().oracle_chunk_select(_ptr(ids), L, vocab_size, block_size, chunk, k, sink, int(m),
+                                     _ptr(sel), _ptr(pidx), _ptr(plen), _ptr(score))
+    if rc != 0:
+        raise ValueError(f"oracle_chunk_select rejected its arguments (rc={rc})")
+    return dict(sel_chunks=sel, prefix_idx=pidx, prefix_len=plen, score=score)

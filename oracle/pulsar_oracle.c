@@ -13,6 +13,8 @@
  *   oracle_phase2_attn     Section 3.2 / Appendix H: one softmax over the
  *                          concatenated retained KV, plus per-block partials
  *   oracle_lse_merge       Appendix H Eq. 12-13, applied iteratively
+ *   oracle_chunk_select    Appendix C: the TF-IDF (Eq. 6), BM25 (Eq. 7), type-token (Eq. 8) and
+ *                          Max-IDF (Eq. 9) chunk scores with the same top-k and prefix list
  *   oracle_generate_step   Algorithm 1 lines 11-16: append KV(q) to the generation shard,
  *                          attend to context + shard (causal within the shard)
  *
@@ -345,5 +347,101 @@ int oracle_generate_step(const uint16_t *Qnew, const uint16_t *Knew, const uint1
                         O + ((size_t)u * Hq + h) * d, LSE + (size_t)u * Hq + h);
         }
     free(Kf); free(Vf); free(key); free(z); free(q);
+    return 0;
+}
+
+/*
+ * Chunk selection under any of the four scoring heuristics of Appendix C.
+ *   mode 0  Max-IDF   score = max_p IDF(t_p)                               (Eq. 9)
+ *   mode 1  TF-IDF    score = (1/|C|) sum_p IDF(t_p)                       (Eq. 6)
+ *   mode 2  BM25      score = sum over types t of IDF_BM25(t) * tf(t)(k1+1) / (tf(t) + k1 D(C)),
+ *                     D(C) = 1 - b + b |C| / lbar, k1 = 1.2, b = 0.75, lbar = mean chunk length,
+ *                     IDF_BM25(t) = ln((N - df + 0.5)/(df + 0.5) + 1)      (Eq. 7)
+ *   mode 3  type-token ratio ("Entropy")  score = distinct tokens / |C|    (Eq. 8)
+ * IDF(t) = ln(N / max(df, 1)) (Eq. 5).  Sums run over the chunk's positions in order (BM25:
+ * over its types in order of first occurrence), in float64.  Top-k, tie rule, positional order
+ * and the prefix list are those of oracle_maxidf_select.
+ * Outputs as there; score_out [B*C] float64.
+ */
+int oracle_chunk_select(const uint32_t *token_ids, int64_t L, int32_t vocab_size, int32_t block_size,
+                        int32_t chunk, int32_t k, int32_t sink, int32_t mode,
+                        int32_t *sel_chunks, int32_t *prefix_idx, int32_t *prefix_len, double *score_out) {
+    if (L <= 0 || block_size <= 0 || chunk <= 0 || vocab_size <= 0 || mode < 0 || mode > 3) return -1;
+    if (L % block_size != 0 || block_size % chunk != 0) return -1;
+    const int64_t B = L / block_size, C = block_size / chunk;
+    if (k < 0 || k > C || sink < 0 || sink > block_size) return -1;
+    for (int64_t p = 0; p < L; ++p)
+        if (token_ids[p] >= (uint32_t)vocab_size) return -1;
+    uint32_t *df = (uint32_t *)calloc((size_t)vocab_size, sizeof(uint32_t));
+    int64_t *last_block = (int64_t *)malloc((size_t)vocab_size * sizeof(int64_t));
+    double *score = (double *)malloc((size_t)C * sizeof(double));
+    char *taken = (char *)malloc((size_t)C);
+    if (!df || !last_block || !score || !taken) return -2;
+    for (int64_t t = 0; t < vocab_size; ++t) last_block[t] = -1;
+    for (int64_t b = 0; b < B; ++b)
+        for (int64_t p = b * block_size; p < (b + 1) * block_size; ++p) {
+            uint32_t t = token_ids[p];
+            if (last_block[t] != b) { last_block[t] = b; df[t] += 1; }
+        }
+    const double N = (double)B, k1 = 1.2, bb = 0.75;
+    const double lbar = (double)chunk;                     /* every chunk has the same length */
+    const double Dc = 1.0 - bb + bb * ((double)chunk / lbar);
+    if (prefix_idx) for (int32_t j = 0; j < sink; ++j) prefix_idx[j] = j;
+    for (int64_t b = 0; b < B; ++b) {
+        for (int64_t c = 0; c < C; ++c) {
+            const uint32_t *tok = token_ids + b * block_size + c * chunk;
+            double s = 0.0;
+            if (mode == 0) {
+                s = -INFINITY;
+                for (int32_t p = 0; p < chunk; ++p) {
+                    uint32_t f = df[tok[p]] > 1 ? df[tok[p]] : 1;
+                    double v = log(N / (double)f);
+                    if (v > s) s = v;
+                }
+            } else if (mode == 1) {
+                for (int32_t p = 0; p < chunk; ++p) {
+                    uint32_t f = df[tok[p]] > 1 ? df[tok[p]] : 1;
+                    s = s + log(N / (double)f);
+                }
+                s = s / (double)chunk;
+            } else {
+                int32_t distinct = 0;
+                for (int32_t p = 0; p < chunk; ++p) {
+                    int first = 1;
+                    for (int32_t q = 0; q < p; ++q) if (tok[q] == tok[p]) first = 0;
+                    if (!first) continue;
+                    ++distinct;
+                    if (mode == 2) {
+                        int32_t tf = 0;
+                        for (int32_t q = 0; q < chunk; ++q) if (tok[q] == tok[p]) ++tf;
+                        double f = (double)df[tok[p]];
+                        double idf = log((N - f + 0.5) / (f + 0.5) + 1.0);
+                        s = s + (idf * ((double)tf * (k1 + 1.0))) / ((double)tf + k1 * Dc);
+                    }
+                }
+                if (mode == 3) s = (double)distinct / (double)chunk;
+            }
+            score[c] = s;
+            if (score_out) score_out[b * C + c] = s;
+        }
+        memset(taken, 0, (size_t)C);
+        for (int32_t j = 0; j < k; ++j) {
+            int64_t best = -1;
+            for (int64_t c = 0; c < C; ++c)
+                if (!taken[c] && (best < 0 || score[c] > score[best])) best = c;
+            if (best >= 0) taken[best] = 1;
+        }
+        int32_t j = 0;
+        for (int64_t c = 0; c < C; ++c) {
+            if (!taken[c]) continue;
+            if (sel_chunks) sel_chunks[b * k + j] = (int32_t)c;
+            if (prefix_idx && b < B - 1)
+                for (int64_t p = 0; p < chunk; ++p)
+                    prefix_idx[sink + (b * k + j) * chunk + p] = (int32_t)(b * block_size + c * chunk + p);
+            ++j;
+        }
+        if (prefix_len) prefix_len[b] = b == 0 ? 0 : (int32_t)(sink + b * k * chunk);
+    }
+    free(df); free(last_block); free(score); free(taken);
     return 0;
 }

@@ -141,3 +141,73 @@ def test_rejects_shapes_outside_the_definition():
         oracle.maxidf_select(ids, 8, 24, 4, 1, 0)       # L not a multiple of the block
     with pytest.raises(ValueError):
         oracle.maxidf_select(ids, 8, 32, 4, 9, 0)       # k above chunks per block
+
+
+# ---- the other scoring heuristics of Appendix C -------------------------------------------------
+def python_scores(ids, nb, m, V, mode):
+    """Eq. 6-9 re-derived with Python floats, collections and math.log."""
+    from collections import Counter
+    B = len(ids) // nb
+    df = brute_df(ids, nb, V)
+    out = np.zeros((B, nb // m))
+    for b in range(B):
+        for c in range(nb // m):
+            toks = [int(t) for t in ids[b * nb + c * m: b * nb + (c + 1) * m]]
+            if mode == "max_idf":
+                out[b, c] = max(math.log(B / max(df[t], 1)) for t in toks)
+            elif mode == "tf_idf":
+                out[b, c] = sum(math.log(B / max(df[t], 1)) for t in toks) / m
+            elif mode == "type_token":
+                out[b, c] = len(set(toks)) / m
+            else:
+                cnt = Counter(toks)
+                D = 1 - 0.75 + 0.75 * (m / m)                  # every chunk has the mean length
+                out[b, c] = sum(math.log((B - df[t] + 0.5) / (df[t] + 0.5) + 1) * tf * 2.2 / (tf + 1.2 * D)
+                                for t, tf in cnt.items())
+    return out
+
+
+@pytest.mark.parametrize("mode", ["max_idf", "tf_idf", "bm25", "type_token"])
+def test_heuristic_scores_and_selection(mode):
+    rng = np.random.default_rng(11)
+    B, C, m, k, V = 5, 9, 6, 3, 40
+    nb = C * m
+    ids = rng.integers(0, V, size=B * nb).astype(np.uint32)
+    ids[: nb] = np.arange(nb) % 7                              # a block of few, much repeated types
+    r = oracle.chunk_select(ids, V, nb, m, k, 4, mode)
+    sc = python_scores(ids, nb, m, V, mode)
+    np.testing.assert_allclose(r["score"], sc, rtol=0, atol=1e-12)
+    for b in range(B):
+        S = r["sel_chunks"][b].tolist()
+        assert S == sorted(S) and len(set(S)) == k
+        for c in S:
+            for c2 in set(range(C)) - set(S):
+                a, bb = r["score"][b, c], r["score"][b, c2]
+                assert a > bb or (a == bb and c < c2)
+    assert r["prefix_len"].tolist() == [0] + [4 + i * k * m for i in range(1, B)]
+
+
+def test_mode_zero_is_the_max_idf_selection():
+    w = W.CONFIGS["tiny"]
+    ids = W.needle_ids(w)
+    a = oracle.maxidf_select(ids, w.vocab_size, w.block_size, w.chunk, w.k, w.sink)
+    b = oracle.chunk_select(ids, w.vocab_size, w.block_size, w.chunk, w.k, w.sink, "max_idf")
+    np.testing.assert_array_equal(a["sel_chunks"], b["sel_chunks"])
+    np.testing.assert_array_equal(a["prefix_idx"], b["prefix_idx"])
+    np.testing.assert_array_equal(a["score"], b["score"])
+
+
+def test_heuristic_closed_forms():
+    nb, m, B = 16, 4, 4
+    ids = np.zeros(B * nb, np.uint32)                         # token 0 everywhere ...
+    ids[0:4] = [1, 2, 3, 4]                                   # ... one chunk of four distinct tokens unique to block 0
+    ids[4:8] = [5, 5, 5, 5]                                   # ... one chunk of a repeated token unique to block 0
+    tt = oracle.chunk_select(ids, 8, nb, m, 1, 0, "type_token")["score"]
+    assert tt[0, 0] == 1.0 and tt[0, 1] == 0.25 and tt[1, 0] == 0.25
+    tf = oracle.chunk_select(ids, 8, nb, m, 1, 0, "tf_idf")["score"]
+    assert tf[1, 0] == 0.0                                    # tokens present in every block carry no IDF
+    assert abs(tf[0, 0] - math.log(4.0)) < 1e-15              # four tokens, each in one block of four
+    bm = oracle.chunk_select(ids, 8, nb, m, 1, 0, "bm25")["score"]
+    idf1 = math.log((4 - 1 + 0.5) / (1 + 0.5) + 1)
+    assert abs(bm[0, 1] - idf1 * 4 * 2.2 / (4 + 1.2)) < 1e-15  # one type with tf = 4
+    assert abs(bm[0, 0] - 4 * idf1 * 2.2 / (1 + 1.2)) < 1e-14  # four types with tf = 1
