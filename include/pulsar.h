@@ -112,6 +112,46 @@ int32_t pulsar_maxidf_select(const uint32_t *token_ids, int64_t L, int32_t vocab
                              int32_t *device_status, void *stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Selection under a chosen chunk score (Appendix C: Eq. 6 TF-IDF, Eq. 7 BM25, Eq. 8 type-token
+ * ratio, Eq. 9 Max-IDF).  Blocks, chunks, top-k, tie rule, positional order, prefix list and
+ * the first ten arguments' meaning are those of pulsar_maxidf_select; only the score differs:
+ *
+ *   PULSAR_SCORE_MAX_IDF     max over the chunk's tokens of IDF(t)
+ *   PULSAR_SCORE_TF_IDF      (1/|C|) * sum over the chunk's positions of IDF(t_p)
+ *   PULSAR_SCORE_BM25        sum over the chunk's distinct tokens of
+ *                            ln((B - df + 0.5)/(df + 0.5) + 1) * tf (k1 + 1) / (tf + k1 D),
+ *                            k1 = 1.2, b = 0.75, D = 1 - b + b |C| / mean chunk length (= 1 here,
+ *                            all chunks having one length), tf = occurrences within the chunk
+ *   PULSAR_SCORE_TYPE_TOKEN  distinct tokens in the chunk / |C|
+ *
+ * with IDF(t) = ln(B / max(df(t),1)).  Scores are float64, accumulated left to right over the
+ * positions (BM25: over the types in order of first occurrence) with one rounding per add,
+ * multiply and divide; chunks whose scores are the same double tie and the lower index wins.
+ *
+ *   score_out   out [B*C] float64 device, or NULL
+ *
+ * Requirements beyond pulsar_maxidf_select's (else PULSAR_ERR_SHAPE): B <= 1024, chunk <= 1024,
+ * C <= 4096.  score_mode outside the enum: PULSAR_ERR_INVALID_ARG.
+ * ------------------------------------------------------------------------------------------ */
+enum {
+    PULSAR_SCORE_MAX_IDF = 0,
+    PULSAR_SCORE_TF_IDF = 1,
+    PULSAR_SCORE_BM25 = 2,
+    PULSAR_SCORE_TYPE_TOKEN = 3
+};
+
+size_t pulsar_chunk_select_workspace_bytes(int64_t L, int32_t vocab_size, int32_t block_size,
+                                           int32_t chunk, int32_t k, int32_t sink, int32_t score_mode);
+
+int32_t pulsar_chunk_select(const uint32_t *token_ids, int64_t L, int32_t vocab_size,
+                            int32_t block_size, int32_t chunk, int32_t k, int32_t sink,
+                            int32_t score_mode,
+                            int32_t *sel_chunks, int32_t *prefix_idx, int32_t *prefix_len,
+                            double *score_out,
+                            void *workspace, size_t workspace_bytes,
+                            int32_t *device_status, void *stream);
+
+/* ------------------------------------------------------------------------------------------
  * Selection for callers that cannot allocate device memory (the paper has no counterpart; this
  * is a packaging variant of pulsar_maxidf_select, same kernels, same results).
  *

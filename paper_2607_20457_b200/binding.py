@@ -28,6 +28,7 @@ EXPORTS = (
     "pulsar_status_string", "pulsar_abi_version", "pulsar_launch_count", "pulsar_wait_selftest",
     "pulsar_maxidf_select_workspace_bytes", "pulsar_maxidf_select",
     "pulsar_maxidf_select_noalloc_max_scratch", "pulsar_maxidf_select_noalloc",
+    "pulsar_chunk_select_workspace_bytes", "pulsar_chunk_select",
     "pulsar_phase1_workspace_bytes", "pulsar_phase1_attn", "pulsar_causal_varlen_attn",
     "pulsar_phase2_choose_splits", "pulsar_phase2_workspace_bytes", "pulsar_phase2_attn",
     "pulsar_phase2_generate_workspace_bytes", "pulsar_phase2_generate_step",
@@ -77,6 +78,10 @@ def load_library(build_if_missing: bool = False):
     lib.pulsar_maxidf_select_noalloc_max_scratch.restype = sz
     lib.pulsar_maxidf_select_noalloc.argtypes = [vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.pulsar_maxidf_select_noalloc.restype = i32
+    lib.pulsar_chunk_select_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, i32, i32]
+    lib.pulsar_chunk_select_workspace_bytes.restype = sz
+    lib.pulsar_chunk_select.argtypes = [vp, i64, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp, vp]
+    lib.pulsar_chunk_select.restype = i32
     lib.pulsar_phase1_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, i32]
     lib.pulsar_phase1_workspace_bytes.restype = sz
     lib.pulsar_phase1_attn.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, vp, vp, i32, f32,
@@ -194,6 +199,39 @@ def pulsar_maxidf_select_noalloc(token_ids: torch.Tensor, vocab_size: int, block
                                           _p(sel_chunks), _p(prefix_idx), _p(prefix_len), None, None, _p(status),
                                           _stream())
     _check("pulsar_maxidf_select_noalloc", rc)
+
+
+SCORE_MODES = {"max_idf": 0, "tf_idf": 1, "bm25": 2, "type_token": 3}
+
+
+def pulsar_chunk_select(token_ids: torch.Tensor, vocab_size: int, block_size: int, chunk: int, k: int, sink: int,
+                        score_mode, want_score: bool = False, workspace=None, status=None):
+    """Selection under one of the chunk scores of the paper's Appendix C (``score_mode``: a key of
+    SCORE_MODES or its number).  Returns a dict of CUDA tensors: sel_chunks [B,k], prefix_idx,
+    prefix_len [B] and, if asked for, score [B,C] float64."""
+    lib = load_library()
+    _need(token_ids, torch.int32, "token_ids")
+    mode = SCORE_MODES.get(score_mode, score_mode)
+    L = token_ids.numel()
+    dev = token_ids.device
+    B = L // block_size if block_size > 0 else 0
+    C = block_size // chunk if chunk > 0 else 0
+    sel_buf = torch.empty(max(B, 0) * max(k, 0) + 4, dtype=torch.int32, device=dev)
+    pidx = torch.empty(max(sink, 0) + max(B - 1, 0) * max(k, 0) * max(chunk, 0) + 4, dtype=torch.int32, device=dev)
+    plen = torch.empty(max(B, 1), dtype=torch.int32, device=dev)
+    score = torch.empty((max(B, 1), max(C, 1)), dtype=torch.float64, device=dev) if want_score else None
+    if workspace is None:
+        workspace = _workspace(lib.pulsar_chunk_select_workspace_bytes(L, vocab_size, block_size, chunk, k, sink,
+                                                                       int(mode)), dev)
+    rc = lib.pulsar_chunk_select(_p(token_ids), L, vocab_size, block_size, chunk, k, sink, int(mode), _p(sel_buf),
+                                 _p(pidx), _p(plen), _p(score), _p(workspace), workspace.numel(), _p(status),
+                                 _stream())
+    _check("pulsar_chunk_select", rc)
+    out = dict(sel_chunks=sel_buf[: B * k].view(B, k), prefix_idx=pidx[: sink + max(B - 1, 0) * k * chunk],
+               prefix_len=plen[:B])
+    if want_score:
+        out["score"] = score
+    return out
 
 
 def phase1_workspace_bytes(L, Hq, Hkv, d, block_size, prefix_total) -> int:

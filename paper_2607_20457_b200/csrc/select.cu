@@ -10,7 +10,14 @@
 //   topk_kernel       one CTA per block: a counting select of the k best chunks with ties to the
 //                     lower index, then the block's part of the prefix list (Eq. 4)
 // Ranking uses the integer df only, so the selection is exact.
+//
+// pulsar_chunk_select runs the same first two launches, then chunk_score_kernel (a float64 score
+// per chunk under TF-IDF, BM25, the type-token ratio or Max-IDF, Appendix C Eq. 6-9) and
+// topk_score_kernel (rank by score, ties to the lower index).
+#include <cmath>
 #include <mutex>
+
+#include <math_constants.h>
 
 #include "common.cuh"
 
@@ -93,6 +100,24 @@ chunk_level_kernel(const uint32_t* __restrict__ ids, const uint16_t* __restrict_
     if (lane == 0) level[c] = static_cast<uint16_t>(mn);
 }
 
+// Block b's part of the prefix list (Eq. 4): its k chosen chunks (ascending, in shared memory)
+// as global token positions, the sink entries (written by block 0) and prefix_len[b].
+__device__ __forceinline__ void write_block_prefix(int b, int n_blocks, int block_size, int chunk, int k, int sink,
+                                                   const int* chosen, int32_t* __restrict__ prefix_idx,
+                                                   int32_t* __restrict__ prefix_len) {
+    const int sigma = k * chunk;
+    if (b < n_blocks - 1) {
+        int32_t* dst = prefix_idx + sink + static_cast<size_t>(b) * sigma;
+        for (int i = threadIdx.x; i < sigma; i += blockDim.x) {
+            const int j = i / chunk, p = i - j * chunk;
+            dst[i] = b * block_size + chosen[j] * chunk + p;
+        }
+    }
+    if (b == 0)
+        for (int i = threadIdx.x; i < sink; i += blockDim.x) prefix_idx[i] = i;
+    if (threadIdx.x == 0) prefix_len[b] = b == 0 ? 0 : sink + b * sigma;
+}
+
 __global__ void __launch_bounds__(kTopkThreads)
 topk_kernel(const uint16_t* __restrict__ level_all, int n_blocks, int block_size, int chunk, int k, int sink,
             int32_t* __restrict__ sel_chunks, int32_t* __restrict__ prefix_idx, int32_t* __restrict__ prefix_len) {
@@ -148,17 +173,104 @@ topk_kernel(const uint16_t* __restrict__ level_all, int n_blocks, int block_size
     }
     __syncthreads();
 
-    const int sigma = k * chunk;
-    if (b < n_blocks - 1) {
-        int32_t* dst = prefix_idx + sink + static_cast<size_t>(b) * sigma;
-        for (int i = threadIdx.x; i < sigma; i += blockDim.x) {
-            const int j = i / chunk, p = i - j * chunk;
-            dst[i] = b * block_size + chosen[j] * chunk + p;
+    write_block_prefix(b, n_blocks, block_size, chunk, k, sink, chosen, prefix_idx, prefix_len);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Selection under the other chunk scores of Appendix C (Eq. 6-8) and Max-IDF as a score (Eq. 9).
+// Scores are float64 and every operation is an explicitly rounded add, multiply or divide in
+// the order the equations are written (positions left to right, types by first occurrence), so
+// two chunks tie exactly when their scores are the same double.  The logarithms are a table over
+// df = 0..B that the host fills (B + 1 values) and passes as a kernel parameter.
+// ---------------------------------------------------------------------------------------------
+constexpr int kMaxScoreBlocks = 1024;
+constexpr int kMaxScoreChunk = 1024;
+constexpr int kMaxScoreChunksPerBlock = 4096;
+struct ScoreTable {
+    double by_df[kMaxScoreBlocks + 1];   // Eq. 5 (TF-IDF, Max-IDF) or the BM25 IDF of Eq. 7, per df
+    double k1_plus_1, k1_times_D;        // BM25 constants: k1 + 1 and k1 * D(C)
+};
+
+// One thread per chunk.
+__global__ void __launch_bounds__(128)
+chunk_score_kernel(const uint32_t* __restrict__ ids, const uint16_t* __restrict__ df_table, int n_chunks_total,
+                   int chunk, int vocab_size, int mode, const __grid_constant__ ScoreTable tab,
+                   double* __restrict__ score) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= n_chunks_total) return;
+    const uint32_t* tok = ids + static_cast<size_t>(c) * chunk;
+    const uint32_t V = static_cast<uint32_t>(vocab_size);
+    double s = 0.0;
+    if (mode == PULSAR_SCORE_MAX_IDF) {
+        s = -CUDART_INF;
+        for (int p = 0; p < chunk; ++p) {
+            const uint32_t t = tok[p];
+            if (t < V) s = fmax(s, tab.by_df[df_table[t]]);
         }
+    } else if (mode == PULSAR_SCORE_TF_IDF) {
+        for (int p = 0; p < chunk; ++p) {
+            const uint32_t t = tok[p];
+            if (t < V) s = __dadd_rn(s, tab.by_df[df_table[t]]);
+        }
+        s = __ddiv_rn(s, static_cast<double>(chunk));
+    } else {
+        int distinct = 0;
+        for (int p = 0; p < chunk; ++p) {
+            const uint32_t t = tok[p];
+            bool first = true;
+            for (int q = 0; q < p; ++q) first = first && (tok[q] != t);
+            if (!first) continue;
+            ++distinct;
+            if (mode == PULSAR_SCORE_BM25 && t < V) {
+                int tf = 0;
+                for (int q = p; q < chunk; ++q) tf += (tok[q] == t) ? 1 : 0;
+                const double tfd = static_cast<double>(tf);
+                const double num = __dmul_rn(tab.by_df[df_table[t]], __dmul_rn(tfd, tab.k1_plus_1));
+                s = __dadd_rn(s, __ddiv_rn(num, __dadd_rn(tfd, tab.k1_times_D)));
+            }
+        }
+        if (mode == PULSAR_SCORE_TYPE_TOKEN) s = __ddiv_rn(static_cast<double>(distinct), static_cast<double>(chunk));
     }
-    if (b == 0)
-        for (int i = threadIdx.x; i < sink; i += blockDim.x) prefix_idx[i] = i;
-    if (threadIdx.x == 0) prefix_len[b] = b == 0 ? 0 : sink + b * sigma;
+    score[c] = s;
+}
+
+// One CTA per block: chunk c is taken when fewer than k chunks beat it (a larger score, or the
+// same score at a lower index); the taken chunks are compacted in index order.
+__global__ void __launch_bounds__(kTopkThreads)
+topk_score_kernel(const double* __restrict__ score_all, int n_blocks, int block_size, int chunk, int k, int sink,
+                  int32_t* __restrict__ sel_chunks, int32_t* __restrict__ prefix_idx,
+                  int32_t* __restrict__ prefix_len) {
+    extern __shared__ double smem_d[];
+    const int C = block_size / chunk;
+    double* sc = smem_d;                                   // [C]
+    int* chosen = reinterpret_cast<int*>(sc + C);          // [k]
+    __shared__ int warp_sums[kTopkThreads / 32];
+    const int b = blockIdx.x;
+    for (int c = threadIdx.x; c < C; c += blockDim.x) sc[c] = score_all[static_cast<size_t>(b) * C + c];
+    __syncthreads();
+    int taken_before = 0;
+    for (int c0 = 0; c0 < C; c0 += kTopkThreads) {
+        const int c = c0 + threadIdx.x;
+        int take = 0;
+        if (c < C) {
+            const double mine = sc[c];
+            int better = 0;
+            for (int o = 0; o < C; ++o) {
+                const double v = sc[o];
+                better += (v > mine || (v == mine && o < c)) ? 1 : 0;
+            }
+            take = better < k ? 1 : 0;
+        }
+        int tot;
+        const int pos = taken_before + block_exclusive_scan(take, warp_sums, tot);
+        if (take && pos < k) {
+            chosen[pos] = c;
+            sel_chunks[static_cast<size_t>(b) * k + pos] = c;
+        }
+        taken_before += tot;
+    }
+    __syncthreads();
+    write_block_prefix(b, n_blocks, block_size, chunk, k, sink, chosen, prefix_idx, prefix_len);
 }
 
 struct SelectPlan {
@@ -242,6 +354,95 @@ extern "C" int32_t pulsar_maxidf_select(const uint32_t* token_ids, int64_t L, in
     count_launch();
     topk_kernel<<<p.n_blocks, kTopkThreads, p.topk_smem, stream>>>(level, p.n_blocks, block_size, chunk, k, sink,
                                                                    sel_chunks, prefix_idx, prefix_len);
+    PULSAR_CUDA_OK(cudaGetLastError());
+    count_launch();
+    return PULSAR_OK;
+}
+
+// =============================================================================================
+// Selection under a chosen chunk score
+// =============================================================================================
+namespace {
+struct ScorePlan {
+    SelectPlan base;
+    size_t score_bytes, total, topk_smem;
+};
+int32_t plan_score(int64_t L, int32_t vocab_size, int32_t block_size, int32_t chunk, int32_t k, int32_t sink,
+                   int32_t mode, ScorePlan& p) {
+    if (mode < PULSAR_SCORE_MAX_IDF || mode > PULSAR_SCORE_TYPE_TOKEN) return PULSAR_ERR_INVALID_ARG;
+    int32_t rc = plan_select(L, vocab_size, block_size, chunk, k, sink, p.base);
+    if (rc != PULSAR_OK) return rc;
+    if (p.base.n_blocks > kMaxScoreBlocks || chunk > kMaxScoreChunk || p.base.C > kMaxScoreChunksPerBlock)
+        return PULSAR_ERR_SHAPE;
+    p.score_bytes = round_up(static_cast<size_t>(p.base.n_blocks) * p.base.C * 8, 256);
+    p.total = p.base.bitmap_bytes + p.base.df_bytes + p.score_bytes;
+    p.topk_smem = static_cast<size_t>(p.base.C) * 8 + static_cast<size_t>(k) * 4;
+    return PULSAR_OK;
+}
+}  // namespace
+
+extern "C" size_t pulsar_chunk_select_workspace_bytes(int64_t L, int32_t vocab_size, int32_t block_size,
+                                                      int32_t chunk, int32_t k, int32_t sink, int32_t score_mode) {
+    ScorePlan p;
+    if (plan_score(L, vocab_size, block_size, chunk, k, sink, score_mode, p) != PULSAR_OK) return 0;
+    return p.total;
+}
+
+extern "C" int32_t pulsar_chunk_select(const uint32_t* token_ids, int64_t L, int32_t vocab_size, int32_t block_size,
+                                       int32_t chunk, int32_t k, int32_t sink, int32_t score_mode,
+                                       int32_t* sel_chunks, int32_t* prefix_idx, int32_t* prefix_len,
+                                       double* score_out, void* workspace, size_t workspace_bytes,
+                                       int32_t* device_status, void* stream_) {
+    ScorePlan p;
+    int32_t rc = plan_score(L, vocab_size, block_size, chunk, k, sink, score_mode, p);
+    if (rc != PULSAR_OK) return rc;
+    if (!token_ids || !sel_chunks || !prefix_idx || !prefix_len || !workspace) return PULSAR_ERR_INVALID_ARG;
+    if (!aligned(token_ids, 16) || !aligned(sel_chunks, 16) || !aligned(prefix_idx, 16) || !aligned(prefix_len, 16) ||
+        (score_out && !aligned(score_out, 16)) || !aligned(workspace, 256))
+        return PULSAR_ERR_ALIGNMENT;
+    if (workspace_bytes < p.total) return PULSAR_ERR_WORKSPACE;
+    rc = check_device();
+    if (rc != PULSAR_OK) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const SelectPlan& b = p.base;
+
+    uint32_t* bitmaps = static_cast<uint32_t*>(workspace);
+    uint16_t* df_table = reinterpret_cast<uint16_t*>(static_cast<char*>(workspace) + b.bitmap_bytes);
+    double* score = score_out ? score_out
+                              : reinterpret_cast<double*>(static_cast<char*>(workspace) + b.bitmap_bytes + b.df_bytes);
+
+    // The logarithms of Eq. 5 / Eq. 7 for every possible df, in float64 from the host's libm.
+    ScoreTable tab;
+    const double N = static_cast<double>(b.n_blocks);
+    for (int f = 0; f <= b.n_blocks; ++f) {
+        const double fd = static_cast<double>(f);
+        tab.by_df[f] = score_mode == PULSAR_SCORE_BM25 ? std::log((N - fd + 0.5) / (fd + 0.5) + 1.0)
+                                                       : std::log(N / static_cast<double>(f > 1 ? f : 1));
+    }
+    const double k1 = 1.2, bb = 0.75;
+    const double mean_len = static_cast<double>(chunk);          // all chunks have one length
+    const double D = 1.0 - bb + bb * (static_cast<double>(chunk) / mean_len);
+    tab.k1_plus_1 = k1 + 1.0;
+    tab.k1_times_D = k1 * D;
+
+    if (b.presence_smem > 48 * 1024)
+        PULSAR_CUDA_OK(cudaFuncSetAttribute(presence_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            static_cast<int>(b.presence_smem)));
+    presence_kernel<<<b.n_blocks, kPresenceThreads, b.presence_smem, stream>>>(token_ids, block_size, vocab_size,
+                                                                               b.words, bitmaps, device_status);
+    PULSAR_CUDA_OK(cudaGetLastError());
+    count_launch();
+    df_idf_kernel<<<(vocab_size + 255) / 256, 256, 0, stream>>>(bitmaps, b.n_blocks, b.words, vocab_size, df_table,
+                                                                nullptr, nullptr);
+    PULSAR_CUDA_OK(cudaGetLastError());
+    count_launch();
+    const int n_chunks_total = b.n_blocks * b.C;
+    chunk_score_kernel<<<(n_chunks_total + 127) / 128, 128, 0, stream>>>(token_ids, df_table, n_chunks_total, chunk,
+                                                                         vocab_size, score_mode, tab, score);
+    PULSAR_CUDA_OK(cudaGetLastError());
+    count_launch();
+    topk_score_kernel<<<b.n_blocks, kTopkThreads, p.topk_smem, stream>>>(score, b.n_blocks, block_size, chunk, k,
+                                                                         sink, sel_chunks, prefix_idx, prefix_len);
     PULSAR_CUDA_OK(cudaGetLastError());
     count_launch();
     return PULSAR_OK;
