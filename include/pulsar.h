@@ -222,6 +222,63 @@ int32_t pulsar_phase1_attn(const uint16_t *Q, const uint16_t *K, const uint16_t 
                            int32_t *device_status, void *stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Phase 1 with the B logical blocks spread over H GPUs by a block-to-host mapping pi (Section 3;
+ * Appendix J, Eq. 14-15).  Every GPU holds Q, K, V of its own blocks only, stored back to back
+ * in ascending logical order, and runs the selection itself on the replicated token ids (no
+ * communication).  The prefix rows a block needs live on other GPUs; they are brought into
+ * local memory before the attention kernel, which never reads a peer:
+ *
+ *   1. pulsar_pack_summary_kv    this GPU's contribution: sink rows and the summary K/V rows of
+ *                                each local block, in one fixed-size buffer
+ *   2. an all-gather of those buffers (the caller's collective, e.g. NCCL)
+ *   3. pulsar_gather_kv_rows     rows of the gathered buffers put into prefix-list order
+ *   4. pulsar_phase1_attn_sharded  the Phase-1 attention over the local blocks with that prefix
+ *
+ * The result equals pulsar_phase1_attn on the whole sequence, row for row.
+ *
+ * pulsar_pack_summary_kv
+ *   K, V        in  [n_local*block_size, Hkv, d] bf16: the local blocks
+ *   sel_chunks  in  [n_blocks*k] int32 (pulsar_maxidf_select), for all logical blocks
+ *   block_ids   in  [n_local] int32 device: logical index of each local block
+ *   K_send, V_send out [sink + n_local*k*chunk, Hkv, d] bf16: rows 0..sink-1 = the first rows of
+ *               the first local block (the sink when that is logical block 0, unused otherwise);
+ *               then k*chunk rows per local block, chunks ascending
+ *   A block id or chunk index out of range sets PULSAR_DEV_BAD_PREFIX.
+ *
+ * pulsar_gather_kv_rows   K_out[j] = K[idx[j]], V_out[j] = V[idx[j]], j < n_idx
+ *   K, V        in  [rows_in, Hkv, d] bf16     idx in [n_idx] int32 device, each in [0, rows_in)
+ *   (an index out of range sets PULSAR_DEV_BAD_PREFIX and row 0 is used).  Hkv*d*2 % 16 == 0.
+ *
+ * pulsar_phase1_attn_sharded
+ *   Q           in  [L_local, Hq, d] bf16, K, V in [L_local, Hkv, d] bf16: the local blocks
+ *   K_prefix, V_prefix in [prefix_total, Hkv, d] bf16, this GPU's memory, prefix-list order
+ *               [sink | Sigma_0 | ... ]; may be NULL when prefix_total == 0
+ *   prefix_len_local in [L_local/block_size] int32 device: prefix rows each local block sees
+ *               (sink + i*k*chunk for logical block i > 0, 0 for block 0)
+ *   O, LSE      out as pulsar_phase1_attn, for the local rows
+ *   workspace   256 bytes (the work counter), 256-byte aligned
+ * Requirements and status codes otherwise as pulsar_phase1_attn.
+ * ------------------------------------------------------------------------------------------ */
+int32_t pulsar_pack_summary_kv(const uint16_t *K, const uint16_t *V, int32_t n_local, int32_t block_size,
+                               int32_t Hkv, int32_t d, const int32_t *sel_chunks,
+                               const int32_t *block_ids, int32_t n_blocks, int32_t chunk, int32_t k,
+                               int32_t sink, uint16_t *K_send, uint16_t *V_send,
+                               int32_t *device_status, void *stream);
+
+int32_t pulsar_gather_kv_rows(const uint16_t *K, const uint16_t *V, int64_t rows_in, int32_t Hkv,
+                              int32_t d, const int32_t *idx, int32_t n_idx,
+                              uint16_t *K_out, uint16_t *V_out, int32_t *device_status, void *stream);
+
+int32_t pulsar_phase1_attn_sharded(const uint16_t *Q, const uint16_t *K, const uint16_t *V,
+                                   int64_t L_local, int32_t Hq, int32_t Hkv, int32_t d,
+                                   int32_t block_size,
+                                   const uint16_t *K_prefix, const uint16_t *V_prefix,
+                                   int32_t prefix_total, const int32_t *prefix_len_local,
+                                   float softmax_scale, uint16_t *O, float *LSE,
+                                   void *workspace, size_t workspace_bytes,
+                                   int32_t *device_status, void *stream);
+
+/* ------------------------------------------------------------------------------------------
  * Causal attention over assembled inputs (Algorithm 1 line 8 as the paper runs it; Eq. 1, Eq. 4,
  * Appendix F).
  *
@@ -334,6 +391,20 @@ int32_t pulsar_phase2_generate_step(const uint16_t *Qnew, const uint16_t *Knew, 
  * ------------------------------------------------------------------------------------------ */
 int32_t pulsar_lse_merge(const float *part_O, const float *part_LSE, int32_t n_parts,
                          int64_t rows, int32_t d, uint16_t *O, float *LSE, void *stream);
+
+/* The same merge for partials that are not stored back to back, and optionally with a float32
+ * result that can itself be a part of a later merge: the two-level merge of Phase 2 on several
+ * GPUs (each GPU merges its own KV parts into one float32 partial, the partials are all-gathered
+ * as Appendix H describes, and every GPU merges the gathered set).
+ *
+ *   part_O   part j starts at part_O + j*part_stride_O floats, [rows, d] float32
+ *   part_LSE part j starts at part_LSE + j*part_stride_LSE floats, [rows] float32
+ *   O        out [rows, d]: float32 if out_is_f32 != 0 (16-byte aligned), else bf16
+ * Requirements as pulsar_lse_merge, plus part_stride_O >= rows*d and a multiple of 4,
+ * part_stride_LSE >= rows (else PULSAR_ERR_SHAPE). */
+int32_t pulsar_lse_merge_strided(const float *part_O, const float *part_LSE, int32_t n_parts,
+                                 int64_t part_stride_O, int64_t part_stride_LSE, int64_t rows,
+                                 int32_t d, void *O, int32_t out_is_f32, float *LSE, void *stream);
 
 #ifdef __cplusplus
 }

@@ -29,10 +29,11 @@ EXPORTS = (
     "pulsar_maxidf_select_workspace_bytes", "pulsar_maxidf_select",
     "pulsar_maxidf_select_noalloc_max_scratch", "pulsar_maxidf_select_noalloc",
     "pulsar_chunk_select_workspace_bytes", "pulsar_chunk_select",
-    "pulsar_phase1_workspace_bytes", "pulsar_phase1_attn", "pulsar_causal_varlen_attn",
+    "pulsar_phase1_workspace_bytes", "pulsar_phase1_attn",
+    "pulsar_pack_summary_kv", "pulsar_gather_kv_rows", "pulsar_phase1_attn_sharded", "pulsar_causal_varlen_attn",
     "pulsar_phase2_choose_splits", "pulsar_phase2_workspace_bytes", "pulsar_phase2_attn",
     "pulsar_phase2_generate_workspace_bytes", "pulsar_phase2_generate_step",
-    "pulsar_lse_merge",
+    "pulsar_lse_merge", "pulsar_lse_merge_strided",
 )
 
 
@@ -87,6 +88,15 @@ def load_library(build_if_missing: bool = False):
     lib.pulsar_phase1_attn.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, vp, vp, i32, f32,
                                        vp, vp, vp, vp, vp, sz, vp, vp]
     lib.pulsar_phase1_attn.restype = i32
+    lib.pulsar_pack_summary_kv.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp]
+    lib.pulsar_pack_summary_kv.restype = i32
+    lib.pulsar_gather_kv_rows.argtypes = [vp, vp, i64, i32, i32, vp, i32, vp, vp, vp, vp]
+    lib.pulsar_gather_kv_rows.restype = i32
+    lib.pulsar_phase1_attn_sharded.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, vp, vp, i32, vp, f32, vp, vp,
+                                               vp, sz, vp, vp]
+    lib.pulsar_phase1_attn_sharded.restype = i32
+    lib.pulsar_lse_merge_strided.argtypes = [vp, vp, i32, i64, i64, i64, i32, vp, i32, vp, vp]
+    lib.pulsar_lse_merge_strided.restype = i32
     lib.pulsar_causal_varlen_attn.argtypes = [vp, vp, vp, i64, vp, i32, i32, i32, i32, f32, vp, vp, vp, sz, vp, vp]
     lib.pulsar_causal_varlen_attn.restype = i32
     lib.pulsar_phase2_choose_splits.argtypes = [i32, i32, i32, i32, i32, i32]
@@ -364,4 +374,77 @@ def pulsar_lse_merge(part_O, part_LSE, want_lse: bool = True):
     LSE = torch.empty(rows, dtype=torch.float32, device=part_O.device) if want_lse else None
     rc = lib.pulsar_lse_merge(_p(part_O), _p(part_LSE), J, rows, d, _p(O), _p(LSE), _stream())
     _check("pulsar_lse_merge", rc)
+    return O, LSE
+
+
+def pulsar_lse_merge_strided(part_O, part_LSE, n_parts: int, part_stride_O: int, part_stride_LSE: int, rows: int,
+                             d: int, out, lse_out=None):
+    """Merge ``n_parts`` partials that start ``part_stride_*`` floats apart (part_O, part_LSE: CUDA
+    float32 tensors or views whose data pointer is part 0).  ``out``: [rows, d] float32 (the result
+    stays a partial) or bf16."""
+    lib = load_library()
+    _need(part_O, torch.float32, "part_O")
+    _need(part_LSE, torch.float32, "part_LSE")
+    if out.dtype not in (torch.float32, torch.bfloat16):
+        raise TypeError("out must be float32 or bfloat16")
+    rc = lib.pulsar_lse_merge_strided(_p(part_O), _p(part_LSE), n_parts, part_stride_O, part_stride_LSE, rows, d,
+                                      _p(out), 1 if out.dtype == torch.float32 else 0, _p(lse_out), _stream())
+    _check("pulsar_lse_merge_strided", rc)
+    return out, lse_out
+
+
+def pulsar_pack_summary_kv(K, V, block_size: int, sel_chunks, block_ids, n_blocks: int, chunk: int, k: int,
+                           sink: int, K_send, V_send, status=None):
+    """This GPU's contribution to the prefix exchange: K, V [n_local*block_size, Hkv, d] bf16 (its
+    blocks), sel_chunks int32 [n_blocks, k], block_ids int32 [n_local] (CUDA) -> K_send, V_send
+    [sink + n_local*k*chunk, Hkv, d] bf16."""
+    lib = load_library()
+    for t, n in ((K, "K"), (V, "V"), (K_send, "K_send"), (V_send, "V_send")):
+        _need(t, torch.bfloat16, n)
+    _need(sel_chunks, torch.int32, "sel_chunks")
+    _need(block_ids, torch.int32, "block_ids")
+    Hkv, d = K.shape[-2], K.shape[-1]
+    rc = lib.pulsar_pack_summary_kv(_p(K), _p(V), block_ids.numel(), block_size, Hkv, d, _p(sel_chunks), _p(block_ids),
+                                    n_blocks, chunk, k, sink, _p(K_send), _p(V_send), _p(status), _stream())
+    _check("pulsar_pack_summary_kv", rc)
+
+
+def pulsar_gather_kv_rows(K, V, idx, K_out, V_out, status=None):
+    """K_out[j] = K[idx[j]], V_out[j] = V[idx[j]] (rows of [rows, Hkv, d] bf16; idx CUDA int32)."""
+    lib = load_library()
+    for t, n in ((K, "K"), (V, "V"), (K_out, "K_out"), (V_out, "V_out")):
+        _need(t, torch.bfloat16, n)
+    _need(idx, torch.int32, "idx")
+    rc = lib.pulsar_gather_kv_rows(_p(K), _p(V), K.shape[0], K.shape[-2], K.shape[-1], _p(idx), idx.numel(),
+                                   _p(K_out), _p(V_out), _p(status), _stream())
+    _check("pulsar_gather_kv_rows", rc)
+
+
+def pulsar_phase1_attn_sharded(Q, K, V, block_size: int, K_prefix, V_prefix, prefix_len_local,
+                               softmax_scale: float = 0.0, want_lse: bool = True, out=None, lse_out=None,
+                               workspace=None, status=None):
+    """Phase-1 attention over this GPU's blocks (Q [L_local,Hq,d], K,V [L_local,Hkv,d]) with the
+    prefix K/V rows already in local memory in prefix-list order (K_prefix, V_prefix
+    [prefix_total,Hkv,d]); prefix_len_local int32 [L_local/block_size].  Returns (O, LSE)."""
+    lib = load_library()
+    for t, n in ((Q, "Q"), (K, "K"), (V, "V")):
+        _need(t, torch.bfloat16, n)
+    _need(prefix_len_local, torch.int32, "prefix_len_local")
+    L, Hq, d = Q.shape
+    Hkv = K.shape[1]
+    prefix_total = 0 if K_prefix is None else K_prefix.shape[0]
+    if prefix_total:
+        _need(K_prefix, torch.bfloat16, "K_prefix")
+        _need(V_prefix, torch.bfloat16, "V_prefix")
+    O = torch.empty_like(Q) if out is None else out
+    LSE = lse_out if lse_out is not None else (
+        torch.empty((L, Hq), dtype=torch.float32, device=Q.device) if want_lse else None)
+    if workspace is None:
+        workspace = _workspace(256, Q.device)
+    rc = lib.pulsar_phase1_attn_sharded(_p(Q), _p(K), _p(V), L, Hq, Hkv, d, block_size,
+                                        _p(K_prefix) if prefix_total else None,
+                                        _p(V_prefix) if prefix_total else None, prefix_total,
+                                        _p(prefix_len_local), float(softmax_scale), _p(O), _p(LSE), _p(workspace),
+                                        workspace.numel(), _p(status), _stream())
+    _check("pulsar_phase1_attn_sharded", rc)
     return O, LSE

@@ -67,3 +67,40 @@ def select_bytes(L: int, vocab_size: int, n_blocks: int, prefix_total: int, k: i
     read, df table written and read, outputs."""
     bitmap = n_blocks * ((vocab_size + 31) // 32) * 4
     return 2 * 4 * L + 2 * bitmap + 2 * 4 * vocab_size + 4 * (prefix_total + n_blocks * k + n_blocks)
+
+
+# ---- block-to-host mapping (Appendix J, Eq. 15) -------------------------------------------------
+MAPPINGS = ("contiguous", "round_robin", "zigzag")
+
+
+def block_to_host(n_blocks: int, n_hosts: int, kind: str = "zigzag"):
+    """pi: logical block -> host, every host getting n_blocks / n_hosts blocks.
+
+    ``contiguous``  host h holds blocks [h*m, (h+1)*m)
+    ``round_robin`` block i goes to host i mod H
+    ``zigzag``      rounds of H blocks dealt alternately forwards and backwards, so that early
+                    (cheap) and late (costly) blocks meet on one host
+    The paper leaves pi open (its 128K runs put two blocks on each of four hosts)."""
+    if n_hosts <= 0 or n_blocks % n_hosts != 0:
+        raise ValueError("n_blocks must be a positive multiple of n_hosts")
+    m = n_blocks // n_hosts
+    if kind == "contiguous":
+        return [i // m for i in range(n_blocks)]
+    if kind == "round_robin":
+        return [i % n_hosts for i in range(n_blocks)]
+    if kind == "zigzag":
+        return [(i % n_hosts) if (i // n_hosts) % 2 == 0 else (n_hosts - 1 - i % n_hosts) for i in range(n_blocks)]
+    raise ValueError(f"unknown mapping {kind!r}")
+
+
+def host_costs(pi, block_cost):
+    """C_h = sum of block_cost(i) over the blocks with pi(i) = h (Eq. 15)."""
+    costs = [0] * (max(pi) + 1)
+    for i, h in enumerate(pi):
+        costs[h] += block_cost(i)
+    return costs
+
+
+def critical_path(pi, block_cost):
+    """C_crit = max_h C_h (Eq. 15)."""
+    return max(host_costs(pi, block_cost))

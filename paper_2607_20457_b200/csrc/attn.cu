@@ -92,6 +92,61 @@ gather_prefix_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V, c
     }
 }
 
+// Row gather without the prefix check: Kout[j] = K[idx[j]], Vout[j] = V[idx[j]].  An index outside
+// [0, rows_in) is reported and row 0 used.
+__global__ void __launch_bounds__(128)
+gather_rows_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V, const int32_t* __restrict__ idx,
+                   int64_t rows_in, int row_vecs, uint4* __restrict__ Kout, uint4* __restrict__ Vout,
+                   int32_t* status) {
+    const int j = blockIdx.x;
+    int src_row = idx[j];
+    if (src_row < 0 || src_row >= rows_in) {
+        if (threadIdx.x == 0) report(status, PULSAR_DEV_BAD_PREFIX);
+        src_row = 0;
+    }
+    const size_t src = static_cast<size_t>(src_row) * row_vecs, dst = static_cast<size_t>(j) * row_vecs;
+    for (int v = threadIdx.x; v < row_vecs; v += blockDim.x) {
+        Kout[dst + v] = K[src + v];
+        Vout[dst + v] = V[src + v];
+    }
+}
+
+// What one GPU contributes to the prefix exchange: row j < sink is row j of its first local block
+// (meaningful only on the GPU that holds logical block 0); row sink + (s*k + c)*chunk + p is token
+// p of the c-th selected chunk of local block s (logical block block_ids[s]).
+__global__ void __launch_bounds__(128)
+pack_summary_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V, const int32_t* __restrict__ sel_chunks,
+                    const int32_t* __restrict__ block_ids, int n_local, int n_blocks, int block_size, int chunk,
+                    int k, int sink, int row_vecs, uint4* __restrict__ Kout, uint4* __restrict__ Vout,
+                    int32_t* status) {
+    const int j = blockIdx.x;
+    int src_row;
+    if (j < sink) {
+        src_row = j;
+    } else {
+        const int t = j - sink, sigma = k * chunk;
+        const int s = t / sigma, r = t - s * sigma;
+        const int c = r / chunk, p = r - c * chunk;
+        const int blk = block_ids[s];
+        int ch = 0;
+        if (blk < 0 || blk >= n_blocks) {
+            if (threadIdx.x == 0) report(status, PULSAR_DEV_BAD_PREFIX);
+        } else {
+            ch = sel_chunks[static_cast<size_t>(blk) * k + c];
+            if (ch < 0 || (ch + 1) * chunk > block_size) {
+                if (threadIdx.x == 0) report(status, PULSAR_DEV_BAD_PREFIX);
+                ch = 0;
+            }
+        }
+        src_row = s * block_size + ch * chunk + p;
+    }
+    const size_t src = static_cast<size_t>(src_row) * row_vecs, dst = static_cast<size_t>(j) * row_vecs;
+    for (int v = threadIdx.x; v < row_vecs; v += blockDim.x) {
+        Kout[dst + v] = K[src + v];
+        Vout[dst + v] = V[src + v];
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Attention kernel: persistent, warp-specialised.
 //
@@ -991,6 +1046,113 @@ extern "C" int32_t pulsar_phase1_attn(const uint16_t* Q, const uint16_t* K, cons
         PULSAR_CUDA_OK(cudaMemcpyAsync(V_ret, V, bytes, cudaMemcpyDeviceToDevice, stream));
     }
     return PULSAR_OK;
+}
+
+// =============================================================================================
+// Phase 1 with the logical blocks spread over several GPUs (block-to-host mapping, Section 3 and
+// Appendix J): what one GPU runs before and after the exchange of summary K/V rows.
+// =============================================================================================
+extern "C" int32_t pulsar_pack_summary_kv(const uint16_t* K, const uint16_t* V, int32_t n_local, int32_t block_size,
+                                          int32_t Hkv, int32_t d, const int32_t* sel_chunks,
+                                          const int32_t* block_ids, int32_t n_blocks, int32_t chunk, int32_t k,
+                                          int32_t sink, uint16_t* K_send, uint16_t* V_send, int32_t* device_status,
+                                          void* stream) {
+    if (n_local <= 0 || block_size <= 0 || Hkv <= 0 || d <= 0 || n_blocks <= 0 || chunk <= 0 || k < 0 || sink < 0)
+        return PULSAR_ERR_INVALID_ARG;
+    if ((static_cast<int64_t>(Hkv) * d * 2) % 16 != 0 || block_size % chunk != 0 || k > block_size / chunk ||
+        sink > block_size || n_local > n_blocks || static_cast<int64_t>(n_local) * block_size >= (1ll << 31))
+        return PULSAR_ERR_SHAPE;
+    if (!K || !V || !sel_chunks || !block_ids || !K_send || !V_send) return PULSAR_ERR_INVALID_ARG;
+    if (!aligned(K, 16) || !aligned(V, 16) || !aligned(K_send, 16) || !aligned(V_send, 16) ||
+        !aligned(sel_chunks, 4) || !aligned(block_ids, 4))
+        return PULSAR_ERR_ALIGNMENT;
+    int32_t rc = check_device();
+    if (rc != PULSAR_OK) return rc;
+    const int64_t rows = sink + static_cast<int64_t>(n_local) * k * chunk;
+    if (rows == 0) return PULSAR_OK;
+    if (rows > 0x7fffffffll) return PULSAR_ERR_SHAPE;
+    pack_summary_kernel<<<static_cast<unsigned>(rows), 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        reinterpret_cast<const uint4*>(K), reinterpret_cast<const uint4*>(V), sel_chunks, block_ids, n_local, n_blocks,
+        block_size, chunk, k, sink, Hkv * d * 2 / 16, reinterpret_cast<uint4*>(K_send),
+        reinterpret_cast<uint4*>(V_send), device_status);
+    PULSAR_CUDA_OK(cudaGetLastError());
+    count_launch();
+    return PULSAR_OK;
+}
+
+extern "C" int32_t pulsar_gather_kv_rows(const uint16_t* K, const uint16_t* V, int64_t rows_in, int32_t Hkv, int32_t d,
+                                         const int32_t* idx, int32_t n_idx, uint16_t* K_out, uint16_t* V_out,
+                                         int32_t* device_status, void* stream) {
+    if (rows_in <= 0 || Hkv <= 0 || d <= 0 || n_idx < 0) return PULSAR_ERR_INVALID_ARG;
+    if ((static_cast<int64_t>(Hkv) * d * 2) % 16 != 0 || rows_in >= (1ll << 31)) return PULSAR_ERR_SHAPE;
+    if (n_idx == 0) return PULSAR_OK;
+    if (!K || !V || !idx || !K_out || !V_out) return PULSAR_ERR_INVALID_ARG;
+    if (!aligned(K, 16) || !aligned(V, 16) || !aligned(K_out, 16) || !aligned(V_out, 16) || !aligned(idx, 4))
+        return PULSAR_ERR_ALIGNMENT;
+    int32_t rc = check_device();
+    if (rc != PULSAR_OK) return rc;
+    gather_rows_kernel<<<n_idx, 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        reinterpret_cast<const uint4*>(K), reinterpret_cast<const uint4*>(V), idx, rows_in, Hkv * d * 2 / 16,
+        reinterpret_cast<uint4*>(K_out), reinterpret_cast<uint4*>(V_out), device_status);
+    PULSAR_CUDA_OK(cudaGetLastError());
+    count_launch();
+    return PULSAR_OK;
+}
+
+extern "C" int32_t pulsar_phase1_attn_sharded(const uint16_t* Q, const uint16_t* K, const uint16_t* V, int64_t L_local,
+                                              int32_t Hq, int32_t Hkv, int32_t d, int32_t block_size,
+                                              const uint16_t* K_prefix, const uint16_t* V_prefix,
+                                              int32_t prefix_total, const int32_t* prefix_len_local,
+                                              float softmax_scale, uint16_t* O, float* LSE, void* workspace,
+                                              size_t workspace_bytes, int32_t* device_status, void* stream_) {
+    Phase1Plan p;
+    int32_t rc = plan_phase1(L_local, Hq, Hkv, d, block_size, prefix_total, p);
+    if (rc != PULSAR_OK) return rc;
+    if (!Q || !K || !V || !O || !prefix_len_local || !workspace || (prefix_total > 0 && (!K_prefix || !V_prefix)))
+        return PULSAR_ERR_INVALID_ARG;
+    if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) || !aligned(prefix_len_local, 4) ||
+        !aligned(K_prefix, 16) || !aligned(V_prefix, 16) || (LSE && !aligned(LSE, 4)) || !aligned(workspace, 256))
+        return PULSAR_ERR_ALIGNMENT;
+    if (workspace_bytes < 256) return PULSAR_ERR_WORKSPACE;
+    rc = check_device();
+    if (rc != PULSAR_OK) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    int32_t* counter = static_cast<int32_t*>(workspace);
+
+    // With no prefix at all the two prefix maps still have to describe valid memory: use K, V.
+    const uint16_t* Kp = prefix_total > 0 ? K_prefix : K;
+    const uint16_t* Vp = prefix_total > 0 ? V_prefix : V;
+    CUtensorMap tmQ, tmK, tmV, tmKp, tmVp;
+    if (!make_map_3d(&tmQ, Q, L_local, Hq, d, 1, kTileM) ||
+        !make_map_2d(&tmK, K, L_local, static_cast<int64_t>(Hkv) * d) ||
+        !make_map_2d(&tmV, V, L_local, static_cast<int64_t>(Hkv) * d) ||
+        !make_map_2d(&tmKp, Kp, static_cast<int64_t>(p.pref_rows), static_cast<int64_t>(Hkv) * d) ||
+        !make_map_2d(&tmVp, Vp, static_cast<int64_t>(p.pref_rows), static_cast<int64_t>(Hkv) * d))
+        return PULSAR_ERR_CUDA;
+
+    PULSAR_CUDA_OK(cudaMemsetAsync(counter, 0, sizeof(int32_t), stream));
+
+    AttnArgs a{};
+    a.mode = kModePhase1;
+    a.Hkv = Hkv;
+    a.pairs = p.pairs_per_block;
+    a.n_items = p.n_blocks * p.pairs_per_block * Hq;
+    a.n_blocks = p.n_blocks;
+    a.counter = counter;
+    a.n_tokens = static_cast<int>(L_local);
+    a.Hq = Hq;
+    a.g = Hq / Hkv;
+    a.pack = 1;
+    a.block_size = block_size;
+    a.tiles_per_block = p.tiles_per_block;
+    a.prefix_total = prefix_total;
+    a.prefix_len = prefix_len_local;
+    a.scale_log2 = (softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf(static_cast<float>(d))) * 1.4426950408889634f;
+    a.O = O;
+    a.LSE = LSE;
+    a.status = device_status;
+    return d == 128 ? launch_attn<128>(tmQ, tmK, tmV, tmKp, tmVp, a, stream)
+                    : launch_attn<64>(tmQ, tmK, tmV, tmKp, tmVp, a, stream);
 }
 
 // =============================================================================================

@@ -6,9 +6,13 @@
 
 namespace pulsar {
 
+// stride_O / stride_L: floats between consecutive parts of part_O / part_LSE.  kF32: the merged
+// output stays float32 (a partial for a later merge) instead of being rounded to bf16.
+template <bool kF32>
 __global__ void __launch_bounds__(256)
 lse_merge_kernel(const float* __restrict__ part_O, const float* __restrict__ part_LSE, int n_parts,
-                 int64_t rows, int d, uint16_t* __restrict__ O, float* __restrict__ LSE) {
+                 int64_t stride_O, int64_t stride_L, int64_t rows, int d, void* __restrict__ O_,
+                 float* __restrict__ LSE) {
     const int vec_per_row = d >> 2;
     const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (idx >= rows * vec_per_row) return;
@@ -16,37 +20,53 @@ lse_merge_kernel(const float* __restrict__ part_O, const float* __restrict__ par
     const int v = static_cast<int>(idx - row * vec_per_row);
 
     float m = -INFINITY;
-    for (int j = 0; j < n_parts; ++j) m = fmaxf(m, part_LSE[static_cast<size_t>(j) * rows + row]);
+    for (int j = 0; j < n_parts; ++j) m = fmaxf(m, part_LSE[static_cast<size_t>(j) * stride_L + row]);
 
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float denom = 0.f;
     if (m > -INFINITY) {
         for (int j = 0; j < n_parts; ++j) {
-            const float w = __expf(part_LSE[static_cast<size_t>(j) * rows + row] - m);
-            const float4 o = *reinterpret_cast<const float4*>(part_O + (static_cast<size_t>(j) * rows + row) * d + v * 4);
+            const float w = __expf(part_LSE[static_cast<size_t>(j) * stride_L + row] - m);
+            const float4 o = *reinterpret_cast<const float4*>(part_O + static_cast<size_t>(j) * stride_O + row * d + v * 4);
             denom += w;
             acc.x += w * o.x; acc.y += w * o.y; acc.z += w * o.z; acc.w += w * o.w;
         }
         const float inv = 1.f / denom;
         acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
     }
-    uint2 packed;
-    packed.x = pack_bf16x2(acc.x, acc.y);
-    packed.y = pack_bf16x2(acc.z, acc.w);
-    *reinterpret_cast<uint2*>(O + row * d + v * 4) = packed;
+    if (kF32) {
+        *reinterpret_cast<float4*>(static_cast<float*>(O_) + row * d + v * 4) = acc;
+    } else {
+        uint2 packed;
+        packed.x = pack_bf16x2(acc.x, acc.y);
+        packed.y = pack_bf16x2(acc.z, acc.w);
+        *reinterpret_cast<uint2*>(static_cast<uint16_t*>(O_) + row * d + v * 4) = packed;
+    }
     if (LSE != nullptr && v == 0) LSE[row] = (m > -INFINITY) ? m + logf(denom) : -INFINITY;
 }
 
-int32_t launch_lse_merge(const float* part_O, const float* part_LSE, int32_t n_parts, int64_t rows, int32_t d,
-                         uint16_t* O, float* LSE, cudaStream_t stream) {
+namespace {
+int32_t launch_merge(const float* part_O, const float* part_LSE, int32_t n_parts, int64_t stride_O, int64_t stride_L,
+                     int64_t rows, int32_t d, void* O, bool f32, float* LSE, cudaStream_t stream) {
     if (rows == 0) return PULSAR_OK;
     const int64_t threads = rows * (d >> 2);
     const int64_t blocks = (threads + 255) / 256;
     if (blocks > 0x7fffffffll) return PULSAR_ERR_SHAPE;
-    lse_merge_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(part_O, part_LSE, n_parts, rows, d, O, LSE);
+    if (f32)
+        lse_merge_kernel<true><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(part_O, part_LSE, n_parts, stride_O,
+                                                                                 stride_L, rows, d, O, LSE);
+    else
+        lse_merge_kernel<false><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(part_O, part_LSE, n_parts, stride_O,
+                                                                                  stride_L, rows, d, O, LSE);
     PULSAR_CUDA_OK(cudaGetLastError());
     count_launch();
     return PULSAR_OK;
+}
+}  // namespace
+
+int32_t launch_lse_merge(const float* part_O, const float* part_LSE, int32_t n_parts, int64_t rows, int32_t d,
+                         uint16_t* O, float* LSE, cudaStream_t stream) {
+    return launch_merge(part_O, part_LSE, n_parts, rows * d, rows, rows, d, O, false, LSE, stream);
 }
 
 }  // namespace pulsar
@@ -62,4 +82,18 @@ extern "C" int32_t pulsar_lse_merge(const float* part_O, const float* part_LSE, 
     int32_t rc = check_device();
     if (rc != PULSAR_OK) return rc;
     return launch_lse_merge(part_O, part_LSE, n_parts, rows, d, O, LSE, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int32_t pulsar_lse_merge_strided(const float* part_O, const float* part_LSE, int32_t n_parts,
+                                            int64_t part_stride_O, int64_t part_stride_LSE, int64_t rows, int32_t d,
+                                            void* O, int32_t out_is_f32, float* LSE, void* stream) {
+    if (n_parts < 1 || rows < 0 || d <= 0) return PULSAR_ERR_INVALID_ARG;
+    if (d % 4 != 0 || d > 1024) return PULSAR_ERR_SHAPE;
+    if (part_stride_O < rows * d || part_stride_LSE < rows || part_stride_O % 4 != 0) return PULSAR_ERR_SHAPE;
+    if (rows > 0 && (!part_O || !part_LSE || !O)) return PULSAR_ERR_INVALID_ARG;
+    if (!aligned(part_O, 16) || !aligned(part_LSE, 4) || !aligned(O, out_is_f32 ? 16 : 8)) return PULSAR_ERR_ALIGNMENT;
+    int32_t rc = check_device();
+    if (rc != PULSAR_OK) return rc;
+    return launch_merge(part_O, part_LSE, n_parts, part_stride_O, part_stride_LSE, rows, d, O, out_is_f32 != 0, LSE,
+                        static_cast<cudaStream_t>(stream));
 }

@@ -1,0 +1,189 @@
+"""Context encoding with the logical blocks spread over several GPUs (block-to-host mapping pi,
+Section 3 and Appendix J; Phase-2 exchange of Appendix H).
+
+One process per GPU.  Every rank holds Q, K, V of its own blocks only (ascending logical order,
+back to back) and the replicated token ids.  Two exchanges, both one all-gather into local
+memory followed by a kernel that reads only local memory:
+
+* Phase 1: each rank packs the summary K/V rows of its blocks (``pulsar_pack_summary_kv``); the
+  packed buffers are all-gathered; ``pulsar_gather_kv_rows`` puts them into prefix-list order;
+  ``pulsar_phase1_attn_sharded`` attends over the local blocks.
+* Phase 2: each rank attends the query to its retained KV (``pulsar_phase2_attn``), merges its
+  own parts into one float32 partial (``pulsar_lse_merge_strided``); the partials (o_h, l_h) are
+  all-gathered and every rank merges the gathered set.
+
+All arithmetic is in the CUDA library; this module computes layouts on the host and calls the
+collective.  ``TorchCollective`` wraps ``torch.distributed``; a test can pass any object with
+the same ``all_gather`` method (e.g. one that concatenates buffers of ranks run in turn).
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import numpy as np
+import torch
+
+from . import cost_model
+
+
+@dataclass(frozen=True)
+class ShardLayout:
+    """Host-side index arithmetic of the sharded path (no tensors on any device)."""
+    n_blocks: int
+    n_hosts: int
+    block_size: int
+    chunk: int
+    k: int
+    sink: int
+    pi: tuple
+
+    @staticmethod
+    def make(n_blocks, n_hosts, block_size, chunk, k, sink, mapping="zigzag") -> "ShardLayout":
+        pi = tuple(cost_model.block_to_host(n_blocks, n_hosts, mapping))
+        return ShardLayout(n_blocks, n_hosts, block_size, chunk, k, sink, pi)
+
+    @property
+    def sigma(self) -> int:
+        return self.k * self.chunk
+
+    @property
+    def n_local(self) -> int:
+        return self.n_blocks // self.n_hosts
+
+    @property
+    def send_rows(self) -> int:
+        """Rows each rank contributes to the prefix exchange."""
+        return self.sink + self.n_local * self.sigma
+
+    @property
+    def prefix_total(self) -> int:
+        return self.sink + (self.n_blocks - 1) * self.sigma
+
+    def local_blocks(self, h: int):
+        return [i for i in range(self.n_blocks) if self.pi[i] == h]
+
+    def local_token_rows(self, h: int) -> np.ndarray:
+        """Global token positions of rank h's rows, in its local order."""
+        return np.concatenate([np.arange(i * self.block_size, (i + 1) * self.block_size)
+                               for i in self.local_blocks(h)])
+
+    def prefix_len_local(self, h: int) -> np.ndarray:
+        return np.array([0 if i == 0 else self.sink + i * self.sigma for i in self.local_blocks(h)], np.int32)
+
+    def prefix_order(self) -> np.ndarray:
+        """For each position of the prefix list, its row in the all-gathered send buffers, the
+        buffer of rank h holding [K rows | V rows], ``send_rows`` each (so rank h's K rows start at
+        row 2*h*send_rows; V rows lie send_rows further on)."""
+        slot = {}
+        for h in range(self.n_hosts):
+            for s, i in enumerate(self.local_blocks(h)):
+                slot[i] = (h, s)
+        out = np.empty(self.prefix_total, np.int64)
+        h0 = self.pi[0]
+        out[: self.sink] = 2 * h0 * self.send_rows + np.arange(self.sink)
+        for i in range(self.n_blocks - 1):
+            h, s = slot[i]
+            base = 2 * h * self.send_rows + self.sink + s * self.sigma
+            out[self.sink + i * self.sigma: self.sink + (i + 1) * self.sigma] = base + np.arange(self.sigma)
+        return out.astype(np.int32)
+
+
+class TorchCollective:
+    """all_gather over a ``torch.distributed`` process group (NCCL on GPUs, gloo on CPU)."""
+
+    def __init__(self, group=None):
+        import torch.distributed as dist
+        self._dist, self._group = dist, group
+        self.world = dist.get_world_size(group)
+        self.rank = dist.get_rank(group)
+
+    def all_gather(self, send: torch.Tensor) -> torch.Tensor:
+        flat = send.contiguous().view(-1)
+        out = torch.empty(self.world * flat.numel(), dtype=send.dtype, device=send.device)
+        self._dist.all_gather_into_tensor(out, flat, group=self._group)
+        return out.view((self.world,) + tuple(send.shape))
+
+
+class ShardedContextEncoder:
+    """One rank's part of the sharded context encoding.  ``collective`` supplies all_gather."""
+
+    def __init__(self, layout: ShardLayout, rank: int, Hq: int, Hkv: int, d: int, vocab_size: int, device,
+                 collective=None):
+        from . import binding
+        self.b = binding
+        self.lay, self.rank, self.Hq, self.Hkv, self.d, self.V = layout, rank, Hq, Hkv, d, vocab_size
+        self.dev = torch.device(device)
+        self.coll = collective
+        self.status = binding.new_status(self.dev)
+        self.block_ids = torch.tensor(layout.local_blocks(rank), dtype=torch.int32, device=self.dev)
+        self.plen_local = torch.from_numpy(layout.prefix_len_local(rank)).to(self.dev)
+        self.order = torch.from_numpy(layout.prefix_order()).to(self.dev)
+        self.send_kv = torch.empty((2, layout.send_rows, Hkv, d), dtype=torch.bfloat16, device=self.dev)
+        self.Kp = torch.empty((max(layout.prefix_total, 1), Hkv, d), dtype=torch.bfloat16, device=self.dev)
+        self.Vp = torch.empty_like(self.Kp)
+
+    # ---- selection: replicated, no communication ------------------------------------------------
+    def select(self, token_ids: torch.Tensor):
+        lay = self.lay
+        self.sel = self.b.pulsar_maxidf_select(token_ids, self.V, lay.block_size, lay.chunk, lay.k, lay.sink,
+                                               status=self.status)
+        return self.sel
+
+    # ---- Phase 1 ---------------------------------------------------------------------------------
+    def phase1_pack(self, K: torch.Tensor, V: torch.Tensor) -> torch.Tensor:
+        lay = self.lay
+        self.b.pulsar_pack_summary_kv(K, V, lay.block_size, self.sel["sel_chunks"], self.block_ids, lay.n_blocks,
+                                      lay.chunk, lay.k, lay.sink, self.send_kv[0], self.send_kv[1],
+                                      status=self.status)
+        return self.send_kv
+
+    def phase1_finish(self, gathered: torch.Tensor, Q, K, V, softmax_scale: float = 0.0):
+        """gathered: [H, 2, send_rows, Hkv, d] bf16 in local memory."""
+        lay = self.lay
+        if lay.prefix_total > 0:
+            rows = gathered.reshape(-1, self.Hkv, self.d)
+            n = rows.shape[0] - lay.send_rows
+            self.b.pulsar_gather_kv_rows(rows[:n], rows[lay.send_rows:], self.order, self.Kp[: lay.prefix_total],
+                                         self.Vp[: lay.prefix_total], status=self.status)
+            Kp, Vp = self.Kp[: lay.prefix_total], self.Vp[: lay.prefix_total]
+        else:
+            Kp = Vp = None
+        return self.b.pulsar_phase1_attn_sharded(Q, K, V, lay.block_size, Kp, Vp, self.plen_local,
+                                                 softmax_scale=softmax_scale, status=self.status)
+
+    def phase1(self, Q, K, V, softmax_scale: float = 0.0):
+        return self.phase1_finish(self.coll.all_gather(self.phase1_pack(K, V)), Q, K, V, softmax_scale)
+
+    # ---- Phase 2 ---------------------------------------------------------------------------------
+    def partial_stride(self, nq: int) -> int:
+        """Floats per rank in the Phase-2 exchange: [nq*Hq*d outputs | nq*Hq LSE], padded to 4."""
+        rows = nq * self.Hq
+        return (rows * (self.d + 1) + 3) // 4 * 4
+
+    def phase2_local(self, Qq, K, V, softmax_scale: float = 0.0, n_splits: int = 0) -> torch.Tensor:
+        """(o_h, l_h) of this rank's retained KV as one float32 buffer."""
+        lay = self.lay
+        nq = Qq.shape[0]
+        rows = nq * self.Hq
+        J = n_splits or self.b.phase2_choose_splits(nq, lay.n_local, lay.block_size, self.Hq, self.Hkv, self.d)
+        _, _, pO, pL = self.b.pulsar_phase2_attn(Qq, K, V, lay.n_local, lay.block_size, softmax_scale, n_splits=J,
+                                                 want_partials=True, status=self.status)
+        send = torch.empty(self.partial_stride(nq), dtype=torch.float32, device=self.dev)
+        self.b.pulsar_lse_merge_strided(pO.view(-1), pL.view(-1), J, rows * self.d, rows, rows, self.d,
+                                        send[: rows * self.d].view(rows, self.d), send[rows * self.d:])
+        return send
+
+    def phase2_finish(self, gathered: torch.Tensor, nq: int):
+        """gathered: [H, partial_stride] float32 in local memory -> (O bf16 [nq,Hq,d], LSE f32 [nq,Hq])."""
+        rows = nq * self.Hq
+        stride = self.partial_stride(nq)
+        flat = gathered.reshape(-1)
+        O = torch.empty((nq, self.Hq, self.d), dtype=torch.bfloat16, device=self.dev)
+        LSE = torch.empty((nq, self.Hq), dtype=torch.float32, device=self.dev)
+        self.b.pulsar_lse_merge_strided(flat, flat[rows * self.d:], gathered.shape[0], stride, stride, rows, self.d,
+                                        O.view(rows, self.d), LSE.view(rows))
+        return O, LSE
+
+    def phase2(self, Qq, K, V, softmax_scale: float = 0.0, n_splits: int = 0):
+        send = self.phase2_local(Qq, K, V, softmax_scale, n_splits)
+        return self.phase2_finish(self.coll.all_gather(send), Qq.shape[0])

@@ -1,0 +1,129 @@
+"""GPU parity of the sharded path (block-to-host mapping, Appendix J; Phase-2 exchange, Appendix H).
+
+One GPU: the H ranks run one after the other in this process and the all-gather is a concatenation
+of their send buffers (no kernel waits on another).  The sharded result is compared with the
+oracle and, row for row, with the unsharded entry points."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import check_attention, to_dev_ids
+from paper_2607_20457_b200 import binding, cost_model as cm, workloads as W
+from paper_2607_20457_b200.sharding import ShardLayout, ShardedContextEncoder
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def make_ranks(w, H, kind):
+    lay = ShardLayout.make(w.n_blocks, H, w.block_size, w.chunk, w.k, w.sink, kind)
+    return lay, [ShardedContextEncoder(lay, h, w.Hq, w.Hkv, w.d, w.vocab_size, DEV) for h in range(H)]
+
+
+def sharded_phase1(w, H, kind, ids, Q, K, V):
+    lay, ranks = make_ranks(w, H, kind)
+    dev_ids = to_dev_ids(ids, DEV)
+    local = []
+    for h, r in enumerate(ranks):
+        rows = torch.from_numpy(lay.local_token_rows(h)).to(DEV)
+        local.append((Q[rows].contiguous(), K[rows].contiguous(), V[rows].contiguous(), rows))
+        r.select(dev_ids)
+    sends = [r.phase1_pack(l[1], l[2]).clone() for r, l in zip(ranks, local)]
+    gathered = torch.stack(sends)                                  # what all_gather returns on every rank
+    O = torch.empty_like(Q)
+    LSE = torch.empty((w.L, w.Hq), dtype=torch.float32, device=DEV)
+    for r, (q, k, v, rows) in zip(ranks, local):
+        o, lse = r.phase1_finish(gathered, q, k, v)
+        O[rows] = o
+        LSE[rows] = lse
+    torch.cuda.synchronize()
+    assert all(int(r.status.item()) == 0 for r in ranks)
+    return O, LSE
+
+
+@pytest.mark.parametrize("kind", cm.MAPPINGS)
+@pytest.mark.parametrize("H", [1, 2, 4])
+def test_phase1_sharded_equals_unsharded(H, kind):
+    w = W.CONFIGS["tiny"]
+    ids = W.needle_ids(w)
+    Q, K, V = (t.to(DEV) for t in W.qkv(w))
+    O, LSE = sharded_phase1(w, H, kind, ids, Q, K, V)
+    sel = binding.pulsar_maxidf_select(to_dev_ids(ids, DEV), w.vocab_size, w.block_size, w.chunk, w.k, w.sink)
+    O1, LSE1, _, _ = binding.pulsar_phase1_attn(Q, K, V, w.block_size, sel["prefix_idx"], sel["prefix_len"])
+    torch.cuda.synchronize()
+    assert torch.equal(O, O1) and torch.equal(LSE, LSE1)            # same kernel, same key order
+    ref = oracle.maxidf_select(ids, w.vocab_size, w.block_size, w.chunk, w.k, w.sink)
+    O_ref, LSE_ref = oracle.phase1_attn(Q.cpu(), K.cpu(), V.cpu(), w.block_size, ref["prefix_idx"], ref["prefix_len"])
+    check_attention(O, LSE, O_ref, LSE_ref, f"sharded phase 1 H={H} {kind}")
+
+
+def test_phase1_sharded_16k_sampled_rows():
+    w = W.CONFIGS["16k"]
+    ids = W.needle_ids(w)
+    Q, K, V = (t.to(DEV) for t in W.qkv(w))
+    O, LSE = sharded_phase1(w, 4, "zigzag", ids, Q, K, V)
+    ref = oracle.maxidf_select(ids, w.vocab_size, w.block_size, w.chunk, w.k, w.sink)
+    rows = W.sample_rows(w, per_block=6)
+    O_ref, LSE_ref = oracle.phase1_attn(Q.cpu(), K.cpu(), V.cpu(), w.block_size, ref["prefix_idx"], ref["prefix_len"],
+                                        rows=rows)
+    r = torch.from_numpy(np.asarray(rows)).to(DEV)
+    check_attention(O[r], LSE[r], O_ref, LSE_ref, "sharded phase 1, 16k")
+
+
+@pytest.mark.parametrize("H,kind", [(1, "contiguous"), (2, "zigzag"), (4, "round_robin"), (4, "zigzag")])
+@pytest.mark.parametrize("nq", [1, 37, 512])
+def test_phase2_sharded(H, kind, nq):
+    w = W.CONFIGS["tiny"]
+    _, K, V = (t.to(DEV) for t in W.qkv(w))
+    Qq = W.phase2_query(w)
+    Qq = (Qq[:nq] if nq <= Qq.shape[0] else Qq.repeat((nq + Qq.shape[0] - 1) // Qq.shape[0], 1, 1)[:nq]).to(DEV)
+    Qq = Qq.contiguous()
+    lay, ranks = make_ranks(w, H, kind)
+    sends = []
+    for h, r in enumerate(ranks):
+        rows = torch.from_numpy(lay.local_token_rows(h)).to(DEV)
+        sends.append(r.phase2_local(Qq, K[rows].contiguous(), V[rows].contiguous()))
+    gathered = torch.stack(sends)
+    outs = [r.phase2_finish(gathered, nq) for r in ranks]
+    torch.cuda.synchronize()
+    assert all(int(r.status.item()) == 0 for r in ranks)
+    for o, lse in outs[1:]:                                          # every rank ends with the same result
+        assert torch.equal(o, outs[0][0]) and torch.equal(lse, outs[0][1])
+    O_ref, LSE_ref = oracle.phase2_attn(Qq.cpu(), K.cpu(), V.cpu(), w.n_blocks, w.block_size)
+    check_attention(outs[0][0], outs[0][1], O_ref, LSE_ref, f"sharded phase 2 H={H} {kind} nq={nq}")
+
+
+def test_strided_merge_float32_partial_matches_oracle():
+    rng = np.random.default_rng(3)
+    J, rows, d, stride = 5, 77, 64, 77 * 64 + 77 + 3 + 16
+    stride = (stride + 3) // 4 * 4
+    buf = torch.zeros(J * stride, dtype=torch.float32)
+    pO = rng.standard_normal((J, rows, d))
+    pL = rng.standard_normal((J, rows)) * 4
+    pL[2, :5] = -np.inf
+    for j in range(J):
+        buf[j * stride: j * stride + rows * d] = torch.from_numpy(pO[j].reshape(-1)).float()
+        buf[j * stride + rows * d: j * stride + rows * d + rows] = torch.from_numpy(pL[j]).float()
+    buf = buf.to(DEV)
+    out = torch.empty((rows, d), dtype=torch.float32, device=DEV)
+    lse = torch.empty(rows, dtype=torch.float32, device=DEV)
+    binding.pulsar_lse_merge_strided(buf, buf[rows * d:], J, stride, stride, rows, d, out, lse)
+    O_ref, L_ref = oracle.lse_merge(pO.astype(np.float32).astype(np.float64), pL.astype(np.float32).astype(np.float64))
+    assert np.abs(out.cpu().numpy() - O_ref).max() < 2e-6 * max(1.0, np.abs(O_ref).max())
+    assert np.abs(lse.cpu().numpy() - L_ref).max() < 1e-5
+    with pytest.raises(binding.PulsarError):
+        binding.pulsar_lse_merge_strided(buf, buf[rows * d:], J, rows * d - 4, stride, rows, d, out, lse)
+
+
+def test_gather_rows_and_bad_index():
+    K = torch.randn(300, 2, 64, device=DEV).bfloat16()
+    V = torch.randn(300, 2, 64, device=DEV).bfloat16()
+    idx = torch.tensor([5, 0, 299, 5, 17], dtype=torch.int32, device=DEV)
+    Ko, Vo = torch.empty(5, 2, 64, device=DEV, dtype=torch.bfloat16), torch.empty(5, 2, 64, device=DEV, dtype=torch.bfloat16)
+    st = binding.new_status(DEV)
+    binding.pulsar_gather_kv_rows(K, V, idx, Ko, Vo, status=st)
+    assert torch.equal(Ko, K[idx.long()]) and torch.equal(Vo, V[idx.long()]) and int(st.item()) == 0
+    idx[2] = 300
+    binding.pulsar_gather_kv_rows(K, V, idx, Ko, Vo, status=st)
+    assert int(st.item()) & 0x2 and torch.equal(Ko[2], K[0])
