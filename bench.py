@@ -6,6 +6,8 @@ attention, Phase-2 query attention with LSE merge -- over one synthetic 128K-tok
 sequence with Llama-3.1-8B attention shapes (one layer).  The metric is context
 tokens per second per layer.  One process per GPU; with N > 1 every rank encodes
 its own sequence (independent problems, no data-path collective: weak scaling).
+``--shard blocks`` instead spreads the blocks of ONE sequence over the N GPUs the way the
+paper does (block-to-host mapping, two all-gathers per step: strong scaling).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 128k] [--impl reference]
 
@@ -352,6 +354,119 @@ def run_gpu(args, w):
         dist.destroy_process_group()
 
 
+def run_gpu_blocks(args, w):
+    """One sequence, its logical blocks spread over the ranks (the paper's own layout): selection
+    replicated, the summary K/V rows all-gathered before Phase 1, the Phase-2 partials all-gathered
+    before the merge.  Whole-job throughput = L / slowest rank's time."""
+    from paper_2607_20457_b200 import binding
+    from paper_2607_20457_b200.sharding import (ShardLayout, ShardedContextEncoder, SingleRankCollective,
+                                                TorchCollective)
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (B200); there is no CPU path")
+    rank, world, local = dist_setup(args.gpus)
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    binding.load_library()
+    peaks = load_peaks()
+    if w.n_blocks % world != 0:
+        raise SystemExit(f"--shard blocks needs the {w.n_blocks} blocks to divide over {world} ranks")
+    lay = ShardLayout.make(w.n_blocks, world, w.block_size, w.chunk, w.k, w.sink, args.mapping)
+    coll = TorchCollective() if world > 1 else SingleRankCollective()
+    enc = ShardedContextEncoder(lay, rank, w.Hq, w.Hkv, w.d, w.vocab_size, dev, coll)
+
+    # every rank generates the same sequence and keeps its own blocks (pinned host copies for e2e)
+    ids = W.token_ids(w)
+    Q, K, V = W.qkv(w)
+    Qq = W.phase2_query(w)
+    rows = torch.from_numpy(lay.local_token_rows(rank))
+    host = dict(ids=torch.from_numpy(ids.view(np.int32)).pin_memory(), Q=Q[rows].pin_memory(),
+                K=K[rows].pin_memory(), V=V[rows].pin_memory(), Qq=Qq.pin_memory())
+    d_ = {n: t.to(dev) for n, t in host.items()}
+    out_host = dict(O=torch.empty_like(host["Q"]).pin_memory(),
+                    O2=torch.empty((w.nq, w.Hq, w.d), dtype=torch.bfloat16).pin_memory())
+
+    def step(t, record=None):
+        if record: record[0].record()
+        enc.select(t["ids"])
+        if record: record[1].record()
+        O1, _ = enc.phase1(t["Q"], t["K"], t["V"])
+        if record: record[2].record()
+        O2, _ = enc.phase2(t["Qq"], t["K"], t["V"])
+        if record: record[3].record()
+        return O1, O2
+
+    for _ in range(args.warmup):
+        step(d_)
+    torch.cuda.synchronize()
+    marks = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local) if rank == 0 else None
+    launches0 = binding.launch_count()
+    barrier(world); torch.cuda.synchronize()
+    start.record()
+    for i in range(args.steps):
+        step(d_, marks[i])
+    stop.record()
+    torch.cuda.synchronize(); barrier(world)
+    launches = binding.launch_count() - launches0
+    clocks = sampler.stop() if sampler else None
+    dev_ms = max_over_ranks(start.elapsed_time(stop), world, dev) / args.steps
+    p1_ms = max_over_ranks(statistics.mean(m[1].elapsed_time(m[2]) for m in marks), world, dev)
+    p2_ms = max_over_ranks(statistics.mean(m[2].elapsed_time(m[3]) for m in marks), world, dev)
+    sel_ms = statistics.mean(m[0].elapsed_time(m[1]) for m in marks)
+
+    # end to end: this rank's inputs from pinned host memory, its results back, every step
+    e2e_steps = max(2, min(args.steps, 5))
+    def host_step():
+        t = {n: h.to(dev, non_blocking=True) for n, h in host.items()}
+        O1, O2 = step(t)
+        out_host["O"].copy_(O1, non_blocking=True)
+        out_host["O2"].copy_(O2, non_blocking=True)
+    host_step()
+    torch.cuda.synchronize(); barrier(world)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        host_step()
+    e1.record()
+    torch.cuda.synchronize(); barrier(world)
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, dev) / e2e_steps
+    status = int(enc.status.item())
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+    if rank != 0:
+        return
+
+    plen = cm.prefix_lens(w.n_blocks, w.sink, w.sigma)
+    mine = lay.local_blocks(0)
+    crit = cm.critical_path(lay.pi, lambda i: cm.phase1_flops(w.block_size, [plen[i]], w.Hq, w.d))
+    achieved_tf = crit / (p1_ms * 1e-3) / 1e12
+    nbytes = lambda ts: sum(t.numel() * t.element_size() for t in ts)
+    line = dict(
+        metric=METRIC, value=w.L / (dev_ms * 1e-3), unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+        ms_per_step=dev_ms, higher_is_better=True, scaling="strong", vs_baseline=None, dtype="bf16",
+        data="synthetic",
+        config=dict(workload=w.name, L=w.L, blocks=w.n_blocks, block_size=w.block_size, chunk=w.chunk, k=w.k,
+                    sink=w.sink, vocab=w.vocab_size, Hq=w.Hq, Hkv=w.Hkv, d=w.d, phase2_query_rows=w.nq,
+                    shard="blocks", mapping=args.mapping, blocks_per_gpu=lay.n_local, rank0_blocks=mine,
+                    collectives_per_step="all_gather of summary K/V rows + all_gather of Phase-2 partials",
+                    cache="inputs larger than the 126 MB L2; no flush needed"),
+        parts=dict(select_us=sel_ms * 1e3, phase1_ms_slowest_rank=p1_ms, phase2_ms_slowest_rank=p2_ms,
+                   phase1_exchange_bytes_per_rank=2 * lay.send_rows * w.Hkv * w.d * 2,
+                   phase2_exchange_bytes_per_rank=enc.partial_stride(w.nq) * 4),
+        roofline=dict(bound="tensor", kernel="attn_kernel<128> (Phase 1, costliest rank)", achieved=achieved_tf,
+                      peak=peaks["bf16_sustained"], unit="TFLOP/s", frac=achieved_tf / peaks["bf16_sustained"],
+                      peak_source=f"{peaks['source']} sustained bf16", algorithmic_flops_per_launch=crit,
+                      traffic=None, timed="CUDA events around pack + all_gather + reorder + attention, max over ranks"),
+        e2e=dict(value=w.L / (e2e_ms * 1e-3), unit=UNIT, ms_per_step=e2e_ms,
+                 h2d_bytes_per_step=nbytes(host.values()), d2h_bytes_per_step=nbytes(out_host.values()),
+                 steps=e2e_steps, how="per rank: pinned host buffers in, results out, one stream"),
+        gpu_launches=launches, device_status=status, clocks=clocks)
+    print(json.dumps(line), flush=True)
+
+
 def run_extras(binding, w, dev, K_d, V_d, peaks):
     """Context measurements beside the headline: decode-shaped Phase 2 (HBM-bound) and the
     Star-anchor prefix against the Pulsar prefix through the same Phase-1 kernel (64K config)."""
@@ -435,6 +550,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="128k", choices=list(W.CONFIGS))
     ap.add_argument("--impl", default="pulsar", choices=["pulsar", "reference"])
+    ap.add_argument("--shard", default="sequences", choices=["sequences", "blocks"],
+                    help="sequences: every GPU encodes its own sequence; blocks: one sequence, blocks spread over GPUs")
+    ap.add_argument("--mapping", default="zigzag", choices=list(cm.MAPPINGS), help="block-to-GPU mapping for --shard blocks")
     ap.add_argument("--no-extras", dest="extras", action="store_false")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--traffic-bytes", type=float, default=None,
@@ -449,7 +567,10 @@ def main():
     if world > 1:
         args.extras = False
         args.cpu_baseline = False
-    run_gpu(args, w)
+    if args.shard == "blocks":
+        run_gpu_blocks(args, w)
+    else:
+        run_gpu(args, w)
 
 
 if __name__ == "__main__":

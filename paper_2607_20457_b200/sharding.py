@@ -104,6 +104,14 @@ class TorchCollective:
         return out.view((self.world,) + tuple(send.shape))
 
 
+class SingleRankCollective:
+    """The all_gather of a one-rank job: the send buffer with a leading dimension of 1."""
+    world, rank = 1, 0
+
+    def all_gather(self, send: torch.Tensor) -> torch.Tensor:
+        return send.unsqueeze(0)
+
+
 class ShardedContextEncoder:
     """One rank's part of the sharded context encoding.  ``collective`` supplies all_gather."""
 
