@@ -15,6 +15,7 @@ Each wrapper names the passage of the paper its C function follows:
 * :func:`generate_step` -- Algorithm 1 lines 11-16 (append KV(q), attend to context + shard)
 * :func:`causal_varlen_attn` -- Eq. 1 over whole assembled inputs (Algorithm 1 line 8)
 * :func:`chunk_select`  -- Appendix C: TF-IDF, BM25, type-token and Max-IDF chunk scores
+* :func:`assemble_positions`, :func:`rope_apply` -- Appendix E: position ids and rotary embedding
 """
 from __future__ import annotations
 
@@ -63,6 +64,10 @@ def _load():
         lib.oracle_lse_merge.restype = ctypes.c_int
         lib.oracle_chunk_select.argtypes = [vp, i64, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
         lib.oracle_chunk_select.restype = ctypes.c_int
+        lib.oracle_assemble_positions.argtypes = [vp, vp, i32, i32, i32, vp]
+        lib.oracle_assemble_positions.restype = ctypes.c_int64
+        lib.oracle_rope_apply.argtypes = [vp, i64, i32, i32, vp, ctypes.c_double, vp]
+        lib.oracle_rope_apply.restype = ctypes.c_int
         _lib = lib
     return _lib
 
@@ -211,3 +216,30 @@ def chunk_select(token_ids, vocab_size, block_size, chunk, k, sink, mode):
     if rc != 0:
         raise ValueError(f"oracle_chunk_select rejected its arguments (rc={rc})")
     return dict(sel_chunks=sel, prefix_idx=pidx, prefix_len=plen, score=score)
+
+
+def assemble_positions(prefix_idx, prefix_len, block_size, mode="sparse"):
+    """Position ids of the assembled Phase-1 inputs stored back to back (Appendix E); ``mode``
+    "sparse" (global positions kept) or "contiguous" (each input renumbered from 0)."""
+    pidx = np.ascontiguousarray(np.asarray(prefix_idx, dtype=np.int32))
+    plen = np.ascontiguousarray(np.asarray(prefix_len, dtype=np.int32))
+    B = plen.shape[0]
+    out = np.zeros(int(plen.sum()) + B * block_size, np.int32)
+    n = _load().oracle_assemble_positions(_ptr(pidx), _ptr(plen), B, block_size,
+                                          {"sparse": 0, "contiguous": 1}[mode], _ptr(out))
+    if n != out.shape[0]:
+        raise ValueError("oracle_assemble_positions rejected its arguments")
+    return out
+
+
+def rope_apply(X, positions, theta=500000.0):
+    """Rotary embedding (rotate-half pairing) of X [rows,H,d] bf16 at the given position ids.
+    Returns float64 [rows,H,d]."""
+    x = _bits(X)
+    rows, H, d = x.shape
+    pos = np.ascontiguousarray(np.asarray(positions, dtype=np.int32))
+    Y = np.zeros((rows, H, d), np.float64)
+    rc = _load().oracle_rope_apply(_ptr(x), rows, H, d, _ptr(pos), float(theta), _ptr(Y))
+    if rc != 0:
+        raise ValueError(f"oracle_rope_apply rejected its arguments (rc={rc})")
+    return Y

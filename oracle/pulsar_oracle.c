@@ -15,6 +15,8 @@
  *   oracle_lse_merge       Appendix H Eq. 12-13, applied iteratively
  *   oracle_chunk_select    Appendix C: the TF-IDF (Eq. 6), BM25 (Eq. 7), type-token (Eq. 8) and
  *                          Max-IDF (Eq. 9) chunk scores with the same top-k and prefix list
+ *   oracle_assemble_positions, oracle_rope_apply   Appendix E: position ids of the assembled
+ *                          inputs (sparse / contiguous) and the rotary embedding they feed
  *   oracle_generate_step   Algorithm 1 lines 11-16: append KV(q) to the generation shard,
  *                          attend to context + shard (causal within the shard)
  *
@@ -443,5 +445,51 @@ int oracle_chunk_select(const uint32_t *token_ids, int64_t L, int32_t vocab_size
         if (prefix_len) prefix_len[b] = b == 0 ? 0 : (int32_t)(sink + b * k * chunk);
     }
     free(df); free(last_block); free(score); free(taken);
+    return 0;
+}
+
+/*
+ * Position ids of the assembled Phase-1 inputs (Appendix E).  Input_i = [first prefix_len[i] entries
+ * of the prefix list | block i] (Eq. 4), the inputs stored back to back.
+ *   mode 0 (sparse, the paper's default): every token keeps its global position -- a prefix entry
+ *          its prefix_idx value, row r of block i the position i*block_size + r
+ *   mode 1 (contiguous): each input is renumbered 0 .. n_i - 1
+ * pos_out has sum_i (prefix_len[i] + block_size) entries.  Returns that count, or -1.
+ */
+int64_t oracle_assemble_positions(const int32_t *prefix_idx, const int32_t *prefix_len, int32_t n_blocks,
+                                  int32_t block_size, int32_t mode, int32_t *pos_out) {
+    if (n_blocks <= 0 || block_size <= 0 || (mode != 0 && mode != 1)) return -1;
+    int64_t at = 0;
+    for (int32_t i = 0; i < n_blocks; ++i) {
+        for (int32_t j = 0; j < prefix_len[i]; ++j) pos_out[at++] = mode == 0 ? prefix_idx[j] : j;
+        for (int32_t r = 0; r < block_size; ++r)
+            pos_out[at++] = mode == 0 ? i * block_size + r : prefix_len[i] + r;
+    }
+    return at;
+}
+
+/*
+ * Rotary position embedding with explicit position ids (Appendix E; the rotate-half pairing of
+ * the Llama family the paper runs on): for row n at position p = positions[n], head h and
+ * j < d/2, with angle = p * theta^(-2j/d):
+ *   y[j]       = x[j] cos(angle) - x[j + d/2] sin(angle)
+ *   y[j + d/2] = x[j + d/2] cos(angle) + x[j] sin(angle)
+ * X [rows, H, d] bf16 bits; Y [rows, H, d] float64 (not rounded).
+ */
+int oracle_rope_apply(const uint16_t *X, int64_t rows, int32_t H, int32_t d, const int32_t *positions,
+                      double theta, double *Y) {
+    if (rows < 0 || H <= 0 || d <= 0 || d % 2 != 0 || theta <= 0.0) return -1;
+    const int32_t half = d / 2;
+    for (int64_t n = 0; n < rows; ++n)
+        for (int32_t j = 0; j < half; ++j) {
+            const double angle = (double)positions[n] * pow(theta, -2.0 * (double)j / (double)d);
+            const double c = cos(angle), sn = sin(angle);
+            for (int32_t h = 0; h < H; ++h) {
+                const size_t base = ((size_t)n * H + h) * d;
+                const double a = bf16_to_double(X[base + j]), b = bf16_to_double(X[base + j + half]);
+                Y[base + j] = a * c - b * sn;
+                Y[base + j + half] = b * c + a * sn;
+            }
+        }
     return 0;
 }
