@@ -537,6 +537,15 @@ def run_extras(binding, w, dev, K_d, V_d, peaks):
     fl = 4 * w4.d * w4.Hq * pairs
     res["pulsar_assembled_all_rows"] = dict(ms=t["median_ms"], rows=cu[-1], tflop=fl / 1e12,
                                             tflops=fl / (t["median_ms"] * 1e-3) / 1e12)
+    # rotary embedding of the assembled 64K inputs at their sparse position ids (Appendix E): a stream
+    pos = binding.pulsar_assemble_positions(torch.from_numpy(pidx).to(dev), torch.from_numpy(plen).to(dev),
+                                            w4.n_blocks, w4.block_size, cu[-1], "sparse")
+    t = time_calls(lambda: (binding.pulsar_rope_apply(Qa, pos, out=Oa), binding.pulsar_rope_apply(Ka, pos, out=Ka)), 10)
+    rope_bytes = 2 * (Qa.numel() + Ka.numel()) * 2 + 2 * pos.numel() * 4
+    out["rope_sparse_positions_64k_assembled"] = dict(
+        ms=t["median_ms"], rows=cu[-1], bytes=rope_bytes, gbs=rope_bytes / (t["median_ms"] * 1e-3) / 1e9,
+        frac_of_measured_hbm=rope_bytes / (t["median_ms"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+        what="Q (32 heads) and K (8 heads) of all assembled inputs, read once and written once")
     res["flop_ratio_star_over_pulsar"] = res["star_anchor"]["tflop"] / res["pulsar"]["tflop"]
     res["time_ratio_star_over_pulsar"] = res["star_anchor"]["ms"] / res["pulsar"]["ms"]
     out["phase1_64k_prefix_comparison"] = res

@@ -59,6 +59,7 @@ typedef enum pulsar_status {
 #define PULSAR_DEV_BAD_PREFIX  0x2 /* prefix index outside [0, first row of its block) (row 0 used) */
 #define PULSAR_DEV_TIMEOUT     0x4 /* an mbarrier wait exceeded its bound (results invalid)   */
 #define PULSAR_DEV_BAD_LENGTH  0x8 /* prefix_len[i] outside [0, prefix_total] (clamped)       */
+#define PULSAR_DEV_BAD_POSITION 0x10 /* negative position id (0 used)                          */
 
 /* Static, human-readable name of a status code (host pointer, never NULL). */
 const char *pulsar_status_string(int32_t status);
@@ -405,6 +406,36 @@ int32_t pulsar_lse_merge(const float *part_O, const float *part_LSE, int32_t n_p
 int32_t pulsar_lse_merge_strided(const float *part_O, const float *part_LSE, int32_t n_parts,
                                  int64_t part_stride_O, int64_t part_stride_LSE, int64_t rows,
                                  int32_t d, void *O, int32_t out_is_f32, float *LSE, void *stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Position ids of the assembled Phase-1 inputs and rotary embedding (Appendix E).
+ *
+ * pulsar_assemble_positions: Input_i = [first prefix_len[i] entries of the prefix list | block i]
+ * (Eq. 4), the B inputs stored back to back (the layout pulsar_causal_varlen_attn takes).
+ *   PULSAR_POS_SPARSE      (the paper's default) every token keeps its global position: a prefix
+ *                          entry its prefix_idx value, row r of block i the position i*block_size+r
+ *   PULSAR_POS_CONTIGUOUS  each input is renumbered 0 .. n_i - 1
+ *   pos_out  out [sum_i (prefix_len[i] + block_size)] int32 device; writes beyond pos_capacity
+ *            entries are dropped.  A prefix_len outside [0, prefix_total] sets PULSAR_DEV_BAD_LENGTH.
+ *
+ * pulsar_rope_apply: rotary embedding with explicit position ids, rotate-half pairing (element j
+ * with element j + d/2), angle = position * theta^(-2j/d):
+ *   y[j] = x[j] cos - x[j+d/2] sin,   y[j+d/2] = x[j+d/2] cos + x[j] sin.
+ *   X in, Y out [rows, H, d] bf16 device (Y may be X); positions [rows] int32 device, >= 0 (a
+ *   negative id sets PULSAR_DEV_BAD_POSITION and counts as 0).  The angle is formed in float64
+ *   and reduced before the float32 sine and cosine, products in float32, result rounded to bf16.
+ *   Requirements: d % 16 == 0, d <= 256 (else PULSAR_ERR_SHAPE); theta > 0.
+ * ------------------------------------------------------------------------------------------ */
+enum { PULSAR_POS_SPARSE = 0, PULSAR_POS_CONTIGUOUS = 1 };
+
+int32_t pulsar_assemble_positions(const int32_t *prefix_idx, const int32_t *prefix_len,
+                                  int32_t prefix_total, int32_t n_blocks, int32_t block_size,
+                                  int32_t mode, int32_t *pos_out, int64_t pos_capacity,
+                                  int32_t *device_status, void *stream);
+
+int32_t pulsar_rope_apply(const uint16_t *X, uint16_t *Y, int64_t rows, int32_t H, int32_t d,
+                          const int32_t *positions, double theta,
+                          int32_t *device_status, void *stream);
 
 #ifdef __cplusplus
 }

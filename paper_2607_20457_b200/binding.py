@@ -22,7 +22,7 @@ STATUS_NAMES = {
     4: "PULSAR_ERR_WORKSPACE", 5: "PULSAR_ERR_UNSUPPORTED_DEVICE", 6: "PULSAR_ERR_CUDA",
     7: "PULSAR_ERR_TIMEOUT", 8: "PULSAR_ERR_DEVICE_CHECK",
 }
-DEV_BAD_TOKEN, DEV_BAD_PREFIX, DEV_TIMEOUT, DEV_BAD_LENGTH = 0x1, 0x2, 0x4, 0x8
+DEV_BAD_TOKEN, DEV_BAD_PREFIX, DEV_TIMEOUT, DEV_BAD_LENGTH, DEV_BAD_POSITION = 0x1, 0x2, 0x4, 0x8, 0x10
 
 EXPORTS = (
     "pulsar_status_string", "pulsar_abi_version", "pulsar_launch_count", "pulsar_wait_selftest",
@@ -34,6 +34,7 @@ EXPORTS = (
     "pulsar_phase2_choose_splits", "pulsar_phase2_workspace_bytes", "pulsar_phase2_attn",
     "pulsar_phase2_generate_workspace_bytes", "pulsar_phase2_generate_step",
     "pulsar_lse_merge", "pulsar_lse_merge_strided",
+    "pulsar_assemble_positions", "pulsar_rope_apply",
 )
 
 
@@ -113,6 +114,10 @@ def load_library(build_if_missing: bool = False):
     lib.pulsar_phase2_generate_step.restype = i32
     lib.pulsar_lse_merge.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp]
     lib.pulsar_lse_merge.restype = i32
+    lib.pulsar_assemble_positions.argtypes = [vp, vp, i32, i32, i32, i32, vp, i64, vp, vp]
+    lib.pulsar_assemble_positions.restype = i32
+    lib.pulsar_rope_apply.argtypes = [vp, vp, i64, i32, i32, vp, ctypes.c_double, vp, vp]
+    lib.pulsar_rope_apply.restype = i32
     _lib = lib
     return lib
 
@@ -448,3 +453,37 @@ def pulsar_phase1_attn_sharded(Q, K, V, block_size: int, K_prefix, V_prefix, pre
                                         workspace.numel(), _p(status), _stream())
     _check("pulsar_phase1_attn_sharded", rc)
     return O, LSE
+
+
+POSITION_MODES = {"sparse": 0, "contiguous": 1}
+
+
+def pulsar_assemble_positions(prefix_idx, prefix_len, n_blocks: int, block_size: int, total: int, mode="sparse",
+                              status=None):
+    """Position ids (CUDA int32 [total]) of the assembled Phase-1 inputs stored back to back;
+    ``total`` = sum_i (prefix_len[i] + block_size), which the caller knows from the layout."""
+    lib = load_library()
+    _need(prefix_len, torch.int32, "prefix_len")
+    _need(prefix_idx, torch.int32, "prefix_idx")
+    pos = torch.empty(max(total, 1), dtype=torch.int32, device=prefix_len.device)
+    n_pref = prefix_idx.numel()
+    rc = lib.pulsar_assemble_positions(_p(prefix_idx) if n_pref else None, _p(prefix_len), n_pref, n_blocks,
+                                       block_size, POSITION_MODES.get(mode, mode), _p(pos), total, _p(status),
+                                       _stream())
+    _check("pulsar_assemble_positions", rc)
+    return pos[:total]
+
+
+def pulsar_rope_apply(X, positions, theta: float = 500000.0, out=None, status=None):
+    """Rotary embedding of X [rows,H,d] CUDA bf16 at ``positions`` (CUDA int32 [rows]); rotate-half
+    pairing.  ``out`` may be X itself (in place)."""
+    lib = load_library()
+    _need(X, torch.bfloat16, "X")
+    _need(positions, torch.int32, "positions")
+    rows, H, d = X.shape
+    if positions.numel() != rows:
+        raise ValueError("one position id per row")
+    Y = torch.empty_like(X) if out is None else out
+    rc = lib.pulsar_rope_apply(_p(X), _p(Y), rows, H, d, _p(positions), float(theta), _p(status), _stream())
+    _check("pulsar_rope_apply", rc)
+    return Y
