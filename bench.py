@@ -509,7 +509,7 @@ def run_extras(binding, w, dev, K_d, V_d, peaks):
     nbytes = cm.phase2_hbm_bytes(1, w.L, w.Hq, w.Hkv, w.d, J + 1)
     out["phase2_generate_step_1tok"] = dict(ms=ms, context_parts=J, shard_rows=65, gbs=nbytes / (ms * 1e-3) / 1e9,
                                             frac_of_measured_hbm=nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                                            launches="2 copies + attention + merge")
+                                            launches="append + attention + merge")
     del flush
     w4 = W.CONFIGS["64k"]
     Q, K, V = (t.to(dev) for t in W.qkv(w4))

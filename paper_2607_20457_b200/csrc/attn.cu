@@ -50,6 +50,8 @@ struct AttnArgs {
     int n_ctx_parts;       // phase 2: parts of the context KV; part n_ctx_parts (if any) is the generation shard
     int gen_len;           // phase 2: rows of the generation shard that precede the new tokens
     int gen_total;         // phase 2: gen_len + new tokens (0 = no generation shard)
+    int quad;              // phase 2, at most 32 query rows per KV head: the rows are replicated into the four
+                           // lane quarters of the tile and each softmax warp takes one quarter of the keys
     int Hkv;
     int pairs;             // phase 1: query-tile pairs per block; phase 2: query-tile pairs per KV head
     int n_items;           // work items in total
@@ -89,6 +91,17 @@ gather_prefix_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V, c
     for (int v = threadIdx.x; v < row_vecs; v += blockDim.x) {
         Kp[dst + v] = K[src + v];
         Vp[dst + v] = V[src + v];
+    }
+}
+
+// KV(q) of the new tokens appended to the generation shard: one launch for both tensors.
+__global__ void __launch_bounds__(256)
+append_kv_kernel(const uint4* __restrict__ Knew, const uint4* __restrict__ Vnew, uint4* __restrict__ Kdst,
+                 uint4* __restrict__ Vdst, int vecs) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < vecs) {
+        Kdst[i] = Knew[i];
+        Vdst[i] = Vnew[i];
     }
 }
 
@@ -475,10 +488,21 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 ++q_use0;
                 if (!ok) break;
                 if (leader) mbar_expect_tx_a(bar0 + 8 * (SL::bQFull + 0), SL::kTileBytes);
+                if (a.quad) {
+                    // the same 32 rows four times, at rows 0, 32, 64, 96 of the tile (the box of the
+                    // tensor map is 32 rows here; 32 rows of a panel are 4096 bytes)
 #pragma unroll
-                for (int p = 0; p < SL::kPanels; ++p)
-                    if (leader) tma_load_3d_a(q_smem + p * kPanelBytes, &tmQ, bar0 + 8 * (SL::bQFull + 0), p * 64, it.head0,
-                                  it.token0_a);
+                    for (int c = 0; c < 4; ++c)
+#pragma unroll
+                        for (int p = 0; p < SL::kPanels; ++p)
+                            if (leader) tma_load_3d_a(q_smem + p * kPanelBytes + c * 4096, &tmQ, bar0 + 8 * (SL::bQFull + 0),
+                                          p * 64, it.head0, it.token0_a);
+                } else {
+#pragma unroll
+                    for (int p = 0; p < SL::kPanels; ++p)
+                        if (leader) tma_load_3d_a(q_smem + p * kPanelBytes, &tmQ, bar0 + 8 * (SL::bQFull + 0), p * 64, it.head0,
+                                      it.token0_a);
+                }
                 for (int t = 0; t < it.n_load && ok; ++t) {
                     __syncwarp();
                     const bool pref = t < it.n_pref_tiles;
@@ -681,6 +705,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             if (n == 0) continue;
             float m_used = -INFINITY, l_run = 0.f;
             const int my_row_in_block = (s ? it.row0_b : it.row0_a) + row;
+            const int row_t = a.quad ? lane : row;             // row as far as token and head are concerned
 
             for (int t = 0; t < n; ++t) {
                 // visible key columns of this tile for this row: [0, n_vis)
@@ -690,7 +715,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                     const int valid = it.pref_len - t * kTileN;
                     if (valid < kTileN) { n_vis = valid; masked = true; }
                     if (it.gen_base >= 0) {                   // generation shard: causal by token
-                        const int token = (s ? it.token0_b : it.token0_a) + row / a.pack;
+                        const int token = (s ? it.token0_b : it.token0_a) + row_t / a.pack;
                         n_vis = min(n_vis, it.gen_base + token + 1 - t * kTileN);
                         masked = true;
                     }
@@ -708,6 +733,73 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 ++s_cnt;
                 if (!ok) break;
                 tc_fence_after();
+
+                if (a.quad) {
+                    // Few query rows (decode): this warp's lane quarter holds a copy of the rows and
+                    // the warp takes keys [32q, 32q+32) of the tile only; the other keys get P = 0 in
+                    // its copy.  Each copy ends as a partial of its own, merged with the KV parts.
+                    const int q4 = warp & 3;
+                    uint32_t rq[32];
+                    tmem_ld32(tS + 32 * q4, rq);
+                    tmem_wait_ld();
+                    if (masked) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (32 * q4 + c >= n_vis) rq[c] = 0xff800000u;          // -inf
+                    }
+                    float mq = -INFINITY;
+#pragma unroll
+                    for (int c = 0; c < 32; c += 2) mq = max3(mq, __uint_as_float(rq[c]), __uint_as_float(rq[c + 1]));
+                    const float m_tile = mq * a.scale_log2;
+                    const bool need = m_tile > m_used + kRescaleThreshold;
+                    if (__any_sync(0xffffffffu, need)) {
+                        const float m_new = need ? m_tile : m_used;
+                        const float alpha = (m_new == -INFINITY) ? 1.f : ex2(m_used - m_new);
+                        l_run *= alpha;
+                        m_used = m_new;
+                        if (t > 0) {
+#pragma unroll
+                            for (int c0 = 0; c0 < D; c0 += 32) {
+                                uint32_t o[32];
+                                tmem_ld32(tO + c0, o);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                                tmem_st32(tO + c0, o);
+                            }
+                        }
+                    }
+                    const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
+                    uint32_t pk[16];
+                    float2 acc = make_float2(0.f, 0.f);
+                    const float2 sc = make_float2(a.scale_log2, a.scale_log2), nm = make_float2(neg_m, neg_m);
+#pragma unroll
+                    for (int c = 0; c < 32; c += 2) {
+                        const float2 x = __ffma2_rn(make_float2(__uint_as_float(rq[c]), __uint_as_float(rq[c + 1])), sc, nm);
+                        float2 pv;
+                        pv.x = ex2(x.x);
+                        pv.y = ex2(x.y);
+                        acc = __fadd2_rn(acc, pv);
+                        pk[c >> 1] = pack_bf16x2(pv.x, pv.y);
+                    }
+                    l_run += acc.x + acc.y;
+                    uint32_t zero[16];
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) zero[c] = 0u;
+#pragma unroll
+                    for (int qq = 0; qq < 4; ++qq) {
+                        if (qq == q4) tmem_st16(tS + 16 * qq, pk);          // P column c/2 holds keys c, c+1
+                        else tmem_st16(tS + 16 * qq, zero);
+                    }
+                    tmem_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive(bar_p);
+                        mbar_arrive(bar_p2);
+                    }
+                    continue;
+                }
 
                 uint32_t r[kTileN];
                 PULSAR_TMEM_LD32_AT(tS + 0, r, 0);
@@ -787,8 +879,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             if (!ok) break;
             tc_fence_after();
             {
-                const int token = (s ? it.token0_b : it.token0_a) + row / a.pack;
-                const int head = it.head0 + row % a.pack;
+                const int token = (s ? it.token0_b : it.token0_a) + row_t / a.pack;
+                const int head = it.head0 + row_t % a.pack;
+                const int part = a.quad ? it.part * 4 + (warp & 3) : it.part;
                 bool store = token < a.n_tokens;
                 if (a.mode != kModePhase2) store = store && my_row_in_block < it.main_len;
                 const float inv_l = l_run > 0.f ? 1.f / l_run : 0.f;
@@ -802,7 +895,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                     if (!store) continue;
                     if (a.part_O != nullptr) {
                         float4* dst = reinterpret_cast<float4*>(
-                            a.part_O + (static_cast<size_t>(it.part) * a.n_tokens * a.Hq + orow) * D + c0);
+                            a.part_O + (static_cast<size_t>(part) * a.n_tokens * a.Hq + orow) * D + c0);
 #pragma unroll
                         for (int c = 0; c < 32; c += 4)
                             dst[c >> 2] = make_float4(__uint_as_float(o[c]) * inv_l, __uint_as_float(o[c + 1]) * inv_l,
@@ -822,7 +915,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 }
                 if (store) {
                     if (a.part_O != nullptr)
-                        a.part_LSE[static_cast<size_t>(it.part) * a.n_tokens * a.Hq + orow] = lse;
+                        a.part_LSE[static_cast<size_t>(part) * a.n_tokens * a.Hq + orow] = lse;
                     else if (a.LSE != nullptr)
                         a.LSE[orow] = lse;
                 }
@@ -948,6 +1041,11 @@ int32_t choose_splits(int32_t nq, int64_t L, int32_t Hq, int32_t Hkv, int32_t d)
     }
     return static_cast<int32_t>(best);
 }
+
+// Decode shapes: all query rows of a KV head (tokens x heads per KV head) fit one quarter of a
+// tile, so the kernel works on four copies of them, one key quarter each; every copy is a partial
+// of its own (four times the partials, merged with the KV parts).
+inline bool phase2_quad(int32_t nq, int32_t g) { return nq * g <= 32; }
 
 // Keys per KV part: L / n_splits when that divides; otherwise the parts are whole 128-key tiles,
 // ceil(tiles / n_splits) each, the last one shorter.  0 if some part would be empty.
@@ -1187,6 +1285,7 @@ extern "C" size_t pulsar_phase2_workspace_bytes(int32_t nq, int32_t B, int32_t b
                                                 int32_t d, int32_t n_splits) {
     size_t a, b;
     if (plan_phase2(nq, B, block_size, Hq, Hkv, d, n_splits, a, b) != PULSAR_OK) return 0;
+    if (phase2_quad(nq, Hq / Hkv)) return 4 * (a + b);
     return n_splits == 1 ? 256 : a + b;
 }
 
@@ -1206,7 +1305,11 @@ extern "C" int32_t pulsar_phase2_attn(const uint16_t* Qq, int32_t nq, const uint
         (part_O && !aligned(part_O, 16)) || (part_LSE && !aligned(part_LSE, 4)) ||
         (workspace && !aligned(workspace, 256)))
         return PULSAR_ERR_ALIGNMENT;
-    const bool need_ws = n_splits > 1 && !user_parts;
+    const bool quad = !user_parts && phase2_quad(nq, Hq / Hkv);
+    const int copies = quad ? 4 : 1;
+    po_bytes *= copies;                                        // both stay multiples of 256
+    pl_bytes *= copies;
+    const bool need_ws = (n_splits > 1 || quad) && !user_parts;
     if (need_ws && (!workspace || workspace_bytes < po_bytes + pl_bytes)) return PULSAR_ERR_WORKSPACE;
     rc = check_device();
     if (rc != PULSAR_OK) return rc;
@@ -1215,11 +1318,12 @@ extern "C" int32_t pulsar_phase2_attn(const uint16_t* Qq, int32_t nq, const uint
     const int64_t L = static_cast<int64_t>(B) * block_size;
     const int g = Hq / Hkv;
     CUtensorMap tmQ, tmK, tmV;
-    if (!make_map_3d(&tmQ, Qq, nq, Hq, d, g, kTileM / g) || !make_map_2d(&tmK, Kb, L, static_cast<int64_t>(Hkv) * d) ||
+    if (!make_map_3d(&tmQ, Qq, nq, Hq, d, g, (quad ? 32 : kTileM) / g) ||
+        !make_map_2d(&tmK, Kb, L, static_cast<int64_t>(Hkv) * d) ||
         !make_map_2d(&tmV, Vb, L, static_cast<int64_t>(Hkv) * d))
         return PULSAR_ERR_CUDA;
 
-    const bool partial_out = n_splits > 1 || user_parts;
+    const bool partial_out = n_splits > 1 || user_parts || quad;
     float* pO = user_parts ? part_O : (need_ws ? static_cast<float*>(workspace) : nullptr);
     float* pL = user_parts ? part_LSE
                            : (need_ws ? reinterpret_cast<float*>(static_cast<char*>(workspace) + po_bytes) : nullptr);
@@ -1233,6 +1337,7 @@ extern "C" int32_t pulsar_phase2_attn(const uint16_t* Qq, int32_t nq, const uint
     a.split_len = static_cast<int>(phase2_split_len(L, n_splits));
     a.kv_len = static_cast<int>(L);
     a.n_ctx_parts = n_splits;
+    a.quad = quad ? 1 : 0;
     a.scale_log2 = (softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf(static_cast<float>(d))) * 1.4426950408889634f;
     a.O = O;
     a.LSE = LSE;
@@ -1248,7 +1353,7 @@ extern "C" int32_t pulsar_phase2_attn(const uint16_t* Qq, int32_t nq, const uint
                   : launch_attn<64>(tmQ, tmK, tmV, tmK, tmV, a, stream);
     if (rc != PULSAR_OK) return rc;
     if (partial_out)
-        return launch_lse_merge(pO, pL, n_splits, static_cast<int64_t>(nq) * Hq, d, O, LSE, stream);
+        return launch_lse_merge(pO, pL, n_splits * copies, static_cast<int64_t>(nq) * Hq, d, O, LSE, stream);
     return PULSAR_OK;
 }
 
@@ -1259,9 +1364,9 @@ extern "C" size_t pulsar_phase2_generate_workspace_bytes(int32_t n_new, int32_t 
                                                          int32_t Hkv, int32_t d, int32_t n_splits) {
     size_t a, b;
     if (plan_phase2(n_new, B, block_size, Hq, Hkv, d, n_splits, a, b) != PULSAR_OK) return 0;
-    // one more part than the context has: the generation shard
-    return round_up(static_cast<size_t>(n_splits + 1) * n_new * Hq * d * 4, 256) +
-           round_up(static_cast<size_t>(n_splits + 1) * n_new * Hq * 4, 256);
+    // one more part than the context has: the generation shard; four partials per part for decode shapes
+    const size_t parts = static_cast<size_t>(n_splits + 1) * (phase2_quad(n_new, Hq / Hkv) ? 4 : 1);
+    return round_up(parts * n_new * Hq * d * 4, 256) + round_up(parts * n_new * Hq * 4, 256);
 }
 
 extern "C" int32_t pulsar_phase2_generate_step(const uint16_t* Qnew, const uint16_t* Knew, const uint16_t* Vnew,
@@ -1282,8 +1387,10 @@ extern "C" int32_t pulsar_phase2_generate_step(const uint16_t* Qnew, const uint1
         !aligned(workspace, 256))
         return PULSAR_ERR_ALIGNMENT;
     const int n_parts = n_splits + 1;
-    const size_t po_bytes = round_up(static_cast<size_t>(n_parts) * n_new * Hq * d * 4, 256);
-    const size_t pl_bytes = round_up(static_cast<size_t>(n_parts) * n_new * Hq * 4, 256);
+    const bool quad = phase2_quad(n_new, Hq / Hkv);
+    const int copies = quad ? 4 : 1;
+    const size_t po_bytes = round_up(static_cast<size_t>(n_parts) * copies * n_new * Hq * d * 4, 256);
+    const size_t pl_bytes = round_up(static_cast<size_t>(n_parts) * copies * n_new * Hq * 4, 256);
     if (workspace_bytes < po_bytes + pl_bytes) return PULSAR_ERR_WORKSPACE;
     rc = check_device();
     if (rc != PULSAR_OK) return rc;
@@ -1293,7 +1400,7 @@ extern "C" int32_t pulsar_phase2_generate_step(const uint16_t* Qnew, const uint1
     const int g = Hq / Hkv;
     const size_t row_bytes = static_cast<size_t>(Hkv) * d * 2;
     CUtensorMap tmQ, tmK, tmV, tmKg, tmVg;
-    if (!make_map_3d(&tmQ, Qnew, n_new, Hq, d, g, kTileM / g) ||
+    if (!make_map_3d(&tmQ, Qnew, n_new, Hq, d, g, (quad ? 32 : kTileM) / g) ||
         !make_map_2d(&tmK, Kb, L, static_cast<int64_t>(Hkv) * d) ||
         !make_map_2d(&tmV, Vb, L, static_cast<int64_t>(Hkv) * d) ||
         !make_map_2d(&tmKg, Kgen, gen_capacity, static_cast<int64_t>(Hkv) * d) ||
@@ -1301,10 +1408,15 @@ extern "C" int32_t pulsar_phase2_generate_step(const uint16_t* Qnew, const uint1
         return PULSAR_ERR_CUDA;
 
     // append KV(q) to the generation shard (Algorithm 1 line 15), then attend
-    PULSAR_CUDA_OK(cudaMemcpyAsync(reinterpret_cast<char*>(Kgen) + gen_len * row_bytes, Knew, n_new * row_bytes,
-                                   cudaMemcpyDeviceToDevice, stream));
-    PULSAR_CUDA_OK(cudaMemcpyAsync(reinterpret_cast<char*>(Vgen) + gen_len * row_bytes, Vnew, n_new * row_bytes,
-                                   cudaMemcpyDeviceToDevice, stream));
+    {
+        const int vecs = static_cast<int>(n_new * row_bytes / 16);
+        append_kv_kernel<<<(vecs + 255) / 256, 256, 0, stream>>>(
+            reinterpret_cast<const uint4*>(Knew), reinterpret_cast<const uint4*>(Vnew),
+            reinterpret_cast<uint4*>(reinterpret_cast<char*>(Kgen) + gen_len * row_bytes),
+            reinterpret_cast<uint4*>(reinterpret_cast<char*>(Vgen) + gen_len * row_bytes), vecs);
+        PULSAR_CUDA_OK(cudaGetLastError());
+        count_launch();
+    }
 
     float* pO = static_cast<float*>(workspace);
     float* pL = reinterpret_cast<float*>(static_cast<char*>(workspace) + po_bytes);
@@ -1319,6 +1431,7 @@ extern "C" int32_t pulsar_phase2_generate_step(const uint16_t* Qnew, const uint1
     a.n_ctx_parts = n_splits;
     a.gen_len = gen_len;
     a.gen_total = gen_len + n_new;
+    a.quad = quad ? 1 : 0;
     a.scale_log2 = (softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf(static_cast<float>(d))) * 1.4426950408889634f;
     a.O = O;
     a.LSE = LSE;
@@ -1333,7 +1446,7 @@ extern "C" int32_t pulsar_phase2_generate_step(const uint16_t* Qnew, const uint1
     rc = d == 128 ? launch_attn<128>(tmQ, tmK, tmV, tmKg, tmVg, a, stream)
                   : launch_attn<64>(tmQ, tmK, tmV, tmKg, tmVg, a, stream);
     if (rc != PULSAR_OK) return rc;
-    return launch_lse_merge(pO, pL, n_parts, static_cast<int64_t>(n_new) * Hq, d, O, LSE, stream);
+    return launch_lse_merge(pO, pL, n_parts * copies, static_cast<int64_t>(n_new) * Hq, d, O, LSE, stream);
 }
 
 // =============================================================================================

@@ -19,12 +19,16 @@ lse_merge_kernel(const float* __restrict__ part_O, const float* __restrict__ par
     const int64_t row = idx / vec_per_row;
     const int v = static_cast<int>(idx - row * vec_per_row);
 
+    // The loads of a group of parts are independent: issue them together (a decode-shaped merge is
+    // a few CTAs whose run time is a chain of load latencies).
     float m = -INFINITY;
+#pragma unroll 8
     for (int j = 0; j < n_parts; ++j) m = fmaxf(m, part_LSE[static_cast<size_t>(j) * stride_L + row]);
 
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float denom = 0.f;
     if (m > -INFINITY) {
+#pragma unroll 8
         for (int j = 0; j < n_parts; ++j) {
             const float w = __expf(part_LSE[static_cast<size_t>(j) * stride_L + row] - m);
             const float4 o = *reinterpret_cast<const float4*>(part_O + static_cast<size_t>(j) * stride_O + row * d + v * 4);
@@ -45,11 +49,86 @@ lse_merge_kernel(const float* __restrict__ part_O, const float* __restrict__ par
     if (LSE != nullptr && v == 0) LSE[row] = (m > -INFINITY) ? m + logf(denom) : -INFINITY;
 }
 
+// The same merge for few output rows and many parts (decode shapes), where one thread per output
+// vector would run a long chain of load latencies on a handful of CTAs: kMergeLanes consecutive
+// lanes share an output vector, lane i takes parts i, i + kMergeLanes, ...; the maximum and the
+// sums are combined by butterfly shuffles (a fixed order, so the result is reproducible).
+constexpr int kMergeLanes = 8;
+
+template <bool kF32>
+__global__ void __launch_bounds__(256)
+lse_merge_lanes_kernel(const float* __restrict__ part_O, const float* __restrict__ part_LSE, int n_parts,
+                       int64_t stride_O, int64_t stride_L, int64_t rows, int d, void* __restrict__ O_,
+                       float* __restrict__ LSE) {
+    const int vec_per_row = d >> 2;
+    const int64_t tid = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const int sub = static_cast<int>(tid % kMergeLanes);
+    const int64_t idx = tid / kMergeLanes;
+    const bool valid = idx < rows * vec_per_row;
+    const int64_t row = valid ? idx / vec_per_row : 0;
+    const int v = valid ? static_cast<int>(idx - row * vec_per_row) : 0;
+
+    float m = -INFINITY;
+    if (valid) {
+#pragma unroll 4
+        for (int j = sub; j < n_parts; j += kMergeLanes) m = fmaxf(m, part_LSE[static_cast<size_t>(j) * stride_L + row]);
+    }
+#pragma unroll
+    for (int o = 1; o < kMergeLanes; o <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float denom = 0.f;
+    if (valid && m > -INFINITY) {
+#pragma unroll 4
+        for (int j = sub; j < n_parts; j += kMergeLanes) {
+            const float w = __expf(part_LSE[static_cast<size_t>(j) * stride_L + row] - m);
+            const float4 o = *reinterpret_cast<const float4*>(part_O + static_cast<size_t>(j) * stride_O + row * d + v * 4);
+            denom += w;
+            acc.x += w * o.x; acc.y += w * o.y; acc.z += w * o.z; acc.w += w * o.w;
+        }
+    }
+#pragma unroll
+    for (int o = 1; o < kMergeLanes; o <<= 1) {
+        denom += __shfl_xor_sync(0xffffffffu, denom, o);
+        acc.x += __shfl_xor_sync(0xffffffffu, acc.x, o);
+        acc.y += __shfl_xor_sync(0xffffffffu, acc.y, o);
+        acc.z += __shfl_xor_sync(0xffffffffu, acc.z, o);
+        acc.w += __shfl_xor_sync(0xffffffffu, acc.w, o);
+    }
+    if (!valid || sub != 0) return;
+    if (m > -INFINITY) {
+        const float inv = 1.f / denom;
+        acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+    }
+    if (kF32) {
+        *reinterpret_cast<float4*>(static_cast<float*>(O_) + row * d + v * 4) = acc;
+    } else {
+        uint2 packed;
+        packed.x = pack_bf16x2(acc.x, acc.y);
+        packed.y = pack_bf16x2(acc.z, acc.w);
+        *reinterpret_cast<uint2*>(static_cast<uint16_t*>(O_) + row * d + v * 4) = packed;
+    }
+    if (LSE != nullptr && v == 0) LSE[row] = (m > -INFINITY) ? m + logf(denom) : -INFINITY;
+}
+
 namespace {
 int32_t launch_merge(const float* part_O, const float* part_LSE, int32_t n_parts, int64_t stride_O, int64_t stride_L,
                      int64_t rows, int32_t d, void* O, bool f32, float* LSE, cudaStream_t stream) {
     if (rows == 0) return PULSAR_OK;
     const int64_t threads = rows * (d >> 2);
+    if (n_parts >= 2 * kMergeLanes && threads <= 64 * 1024) {
+        // few outputs, many parts: spread the parts of an output over lanes
+        const unsigned blocks = static_cast<unsigned>((threads * kMergeLanes + 255) / 256);
+        if (f32)
+            lse_merge_lanes_kernel<true><<<blocks, 256, 0, stream>>>(part_O, part_LSE, n_parts, stride_O, stride_L, rows,
+                                                                     d, O, LSE);
+        else
+            lse_merge_lanes_kernel<false><<<blocks, 256, 0, stream>>>(part_O, part_LSE, n_parts, stride_O, stride_L, rows,
+                                                                      d, O, LSE);
+        PULSAR_CUDA_OK(cudaGetLastError());
+        count_launch();
+        return PULSAR_OK;
+    }
     const int64_t blocks = (threads + 255) / 256;
     if (blocks > 0x7fffffffll) return PULSAR_ERR_SHAPE;
     if (f32)

@@ -86,6 +86,29 @@ def test_merge_entry_point_against_oracle_merge():
     assert torch.equal(O1, torch.from_numpy(pO[0].astype(np.float32)).to(DEV).to(torch.bfloat16))
 
 
+@pytest.mark.parametrize("J,rows,d", [(16, 32, 128), (72, 32, 128), (77, 5, 64), (23, 250, 128)])
+def test_merge_of_many_parts_into_few_rows(J, rows, d):
+    """Decode shapes take the merge that spreads the parts of an output over lanes."""
+    rng = np.random.default_rng(J)
+    pO = rng.standard_normal((J, rows, d)).astype(np.float32)
+    pL = (rng.standard_normal((J, rows)) * 4).astype(np.float32)
+    pL[J // 2, : rows // 2] = -np.inf
+    pL[:, -1] = -np.inf                                   # a row with no keys at all
+    Oref, Lref = oracle.lse_merge(pO.astype(np.float64), np.where(np.isinf(pL), -1e30, pL.astype(np.float64)))
+    out = torch.empty((rows, d), dtype=torch.float32, device=DEV)
+    lse = torch.empty(rows, dtype=torch.float32, device=DEV)
+    tO, tL = torch.from_numpy(pO).to(DEV), torch.from_numpy(pL).to(DEV)
+    binding.pulsar_lse_merge_strided(tO.view(-1), tL.view(-1), J, rows * d, rows, rows, d, out, lse)
+    torch.cuda.synchronize()
+    got, gl = out.cpu().numpy(), lse.cpu().numpy()
+    assert np.abs(got[:-1] - Oref[:-1]).max() < 5e-6 * max(1.0, np.abs(Oref).max())
+    assert np.abs(gl[:-1] - Lref[:-1]).max() < 1e-5
+    assert np.isneginf(gl[-1]) and (got[-1] == 0).all()
+    again = torch.empty_like(out)
+    binding.pulsar_lse_merge_strided(tO.view(-1), tL.view(-1), J, rows * d, rows, rows, d, again, lse)
+    assert torch.equal(again, out)                        # fixed combination order
+
+
 def test_phase1_then_phase2_chain_on_retained_kv():
     w = W.CONFIGS["tiny"]
     Q, K, V = W.qkv(w)
