@@ -540,7 +540,7 @@ def run_extras(binding, w, dev, K_d, V_d, peaks):
     # rotary embedding of the assembled 64K inputs at their sparse position ids (Appendix E): a stream
     pos = binding.pulsar_assemble_positions(torch.from_numpy(pidx).to(dev), torch.from_numpy(plen).to(dev),
                                             w4.n_blocks, w4.block_size, cu[-1], "sparse")
-    t = time_calls(lambda: (binding.pulsar_rope_apply(Qa, pos, out=Oa), binding.pulsar_rope_apply(Ka, pos, out=Ka)), 10)
+    t = time_calls(lambda: binding.pulsar_rope_apply_qk(Qa, Ka, pos, q_out=Oa, k_out=Ka), 10)
     rope_bytes = 2 * (Qa.numel() + Ka.numel()) * 2 + 2 * pos.numel() * 4
     out["rope_sparse_positions_64k_assembled"] = dict(
         ms=t["median_ms"], rows=cu[-1], bytes=rope_bytes, gbs=rope_bytes / (t["median_ms"] * 1e-3) / 1e9,

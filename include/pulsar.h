@@ -437,6 +437,13 @@ int32_t pulsar_rope_apply(const uint16_t *X, uint16_t *Y, int64_t rows, int32_t 
                           const int32_t *positions, double theta,
                           int32_t *device_status, void *stream);
 
+/* The same embedding for a query and a key tensor of the same rows in one launch (the rows' sines and
+ * cosines are formed once): Q [rows, Hq, d] -> Q_out, K [rows, Hkv, d] -> K_out (each may be in place). */
+int32_t pulsar_rope_apply_qk(const uint16_t *Q, uint16_t *Q_out, int32_t Hq,
+                             const uint16_t *K, uint16_t *K_out, int32_t Hkv,
+                             int64_t rows, int32_t d, const int32_t *positions, double theta,
+                             int32_t *device_status, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

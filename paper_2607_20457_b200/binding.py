@@ -34,7 +34,7 @@ EXPORTS = (
     "pulsar_phase2_choose_splits", "pulsar_phase2_workspace_bytes", "pulsar_phase2_attn",
     "pulsar_phase2_generate_workspace_bytes", "pulsar_phase2_generate_step",
     "pulsar_lse_merge", "pulsar_lse_merge_strided",
-    "pulsar_assemble_positions", "pulsar_rope_apply",
+    "pulsar_assemble_positions", "pulsar_rope_apply", "pulsar_rope_apply_qk",
 )
 
 
@@ -118,6 +118,8 @@ def load_library(build_if_missing: bool = False):
     lib.pulsar_assemble_positions.restype = i32
     lib.pulsar_rope_apply.argtypes = [vp, vp, i64, i32, i32, vp, ctypes.c_double, vp, vp]
     lib.pulsar_rope_apply.restype = i32
+    lib.pulsar_rope_apply_qk.argtypes = [vp, vp, i32, vp, vp, i32, i64, i32, vp, ctypes.c_double, vp, vp]
+    lib.pulsar_rope_apply_qk.restype = i32
     _lib = lib
     return lib
 
@@ -487,3 +489,21 @@ def pulsar_rope_apply(X, positions, theta: float = 500000.0, out=None, status=No
     rc = lib.pulsar_rope_apply(_p(X), _p(Y), rows, H, d, _p(positions), float(theta), _p(status), _stream())
     _check("pulsar_rope_apply", rc)
     return Y
+
+
+def pulsar_rope_apply_qk(Q, K, positions, theta: float = 500000.0, q_out=None, k_out=None, status=None):
+    """Rotary embedding of Q [rows,Hq,d] and K [rows,Hkv,d] (CUDA bf16) in one launch; the outputs
+    default to new tensors and may be the inputs themselves."""
+    lib = load_library()
+    _need(Q, torch.bfloat16, "Q")
+    _need(K, torch.bfloat16, "K")
+    _need(positions, torch.int32, "positions")
+    rows, Hq, d = Q.shape
+    if K.shape[0] != rows or K.shape[2] != d or positions.numel() != rows:
+        raise ValueError("Q, K and positions must cover the same rows and head size")
+    Qo = torch.empty_like(Q) if q_out is None else q_out
+    Ko = torch.empty_like(K) if k_out is None else k_out
+    rc = lib.pulsar_rope_apply_qk(_p(Q), _p(Qo), Hq, _p(K), _p(Ko), K.shape[1], rows, d, _p(positions), float(theta),
+                                  _p(status), _stream())
+    _check("pulsar_rope_apply_qk", rc)
+    return Qo, Ko

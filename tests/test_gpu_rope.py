@@ -64,6 +64,18 @@ def test_rope_in_place_and_sparse_positions_of_an_assembled_input():
     assert torch.equal(Xd, Y)
 
 
+def test_rope_qk_in_one_launch_equals_two():
+    g = torch.Generator().manual_seed(21)
+    rows = 1003
+    Q = torch.randn((rows, 32, 128), generator=g).bfloat16().to(DEV)
+    K = torch.randn((rows, 8, 128), generator=g).bfloat16().to(DEV)
+    pos = torch.randint(0, 131072, (rows,), generator=g, dtype=torch.int32).to(DEV)
+    Qo, Ko = binding.pulsar_rope_apply_qk(Q, K, pos)
+    assert torch.equal(Qo, binding.pulsar_rope_apply(Q, pos)) and torch.equal(Ko, binding.pulsar_rope_apply(K, pos))
+    binding.pulsar_rope_apply_qk(Q, K, pos, q_out=Q, k_out=K)              # in place
+    assert torch.equal(Q, Qo) and torch.equal(K, Ko)
+
+
 def test_rope_keeps_attention_scores_relative():
     """q at position m against k at position n gives the same logit as at (m+s, n+s): checked on the
     GPU results within bf16 rounding of the rotated vectors."""
