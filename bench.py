@@ -374,6 +374,10 @@ def run_gpu_blocks(args, w):
     lay = ShardLayout.make(w.n_blocks, world, w.block_size, w.chunk, w.k, w.sink, args.mapping)
     coll = TorchCollective() if world > 1 else SingleRankCollective()
     enc = ShardedContextEncoder(lay, rank, w.Hq, w.Hkv, w.d, w.vocab_size, dev, coll)
+    peers = None
+    if args.exchange == "fused":                      # Phase-2 partials read in place by the merge kernel
+        from paper_2607_20457_b200.sharding import LocalPeers, SymmetricMemoryPeers
+        peers = SymmetricMemoryPeers() if world > 1 else LocalPeers(1)
 
     # every rank generates the same sequence and keeps its own blocks (pinned host copies for e2e)
     ids = W.token_ids(w)
@@ -392,7 +396,10 @@ def run_gpu_blocks(args, w):
         if record: record[1].record()
         O1, _ = enc.phase1(t["Q"], t["K"], t["V"])
         if record: record[2].record()
-        O2, _ = enc.phase2(t["Qq"], t["K"], t["V"])
+        if peers is not None:
+            O2, _ = enc.phase2_fused(peers, t["Qq"], t["K"], t["V"])
+        else:
+            O2, _ = enc.phase2(t["Qq"], t["K"], t["V"])
         if record: record[3].record()
         return O1, O2
 
@@ -450,7 +457,7 @@ def run_gpu_blocks(args, w):
         data="synthetic",
         config=dict(workload=w.name, L=w.L, blocks=w.n_blocks, block_size=w.block_size, chunk=w.chunk, k=w.k,
                     sink=w.sink, vocab=w.vocab_size, Hq=w.Hq, Hkv=w.Hkv, d=w.d, phase2_query_rows=w.nq,
-                    shard="blocks", mapping=args.mapping, blocks_per_gpu=lay.n_local, rank0_blocks=mine,
+                    shard="blocks", mapping=args.mapping, phase2_exchange=args.exchange, blocks_per_gpu=lay.n_local, rank0_blocks=mine,
                     collectives_per_step="all_gather of summary K/V rows + all_gather of Phase-2 partials",
                     cache="inputs larger than the 126 MB L2; no flush needed"),
         parts=dict(select_us=sel_ms * 1e3, phase1_ms_slowest_rank=p1_ms, phase2_ms_slowest_rank=p2_ms,
@@ -562,6 +569,8 @@ def main():
     ap.add_argument("--shard", default="sequences", choices=["sequences", "blocks"],
                     help="sequences: every GPU encodes its own sequence; blocks: one sequence, blocks spread over GPUs")
     ap.add_argument("--mapping", default="zigzag", choices=list(cm.MAPPINGS), help="block-to-GPU mapping for --shard blocks")
+    ap.add_argument("--exchange", default="allgather", choices=["allgather", "fused"],
+                    help="--shard blocks: all-gather the Phase-2 partials, or let the merge kernel read them from peers")
     ap.add_argument("--no-extras", dest="extras", action="store_false")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--traffic-bytes", type=float, default=None,

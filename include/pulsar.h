@@ -407,6 +407,24 @@ int32_t pulsar_lse_merge_strided(const float *part_O, const float *part_LSE, int
                                  int64_t part_stride_O, int64_t part_stride_LSE, int64_t rows,
                                  int32_t d, void *O, int32_t out_is_f32, float *LSE, void *stream);
 
+/* The merge fused with the exchange that precedes it on several GPUs (Appendix H): instead of
+ * all-gathering every GPU's partial and merging all rows everywhere, GPU r merges only rows
+ * [row_begin, row_begin + rows) and reads that slice of every GPU's partial in place, through
+ * peer-mapped addresses, while it merges.  Each GPU then holds 1/H of the merged rows (the caller
+ * gathers the bf16 results if every GPU needs them all): H times fewer bytes cross NVLink than
+ * with the all-gather of partials.
+ *
+ *   part_bases  HOST array [n_parts] of DEVICE addresses (this GPU's own memory or peer-mapped
+ *               memory of other GPUs), each a buffer [rows_total*d float32 outputs | rows_total
+ *               float32 LSE]; n_parts <= 64.  The caller orders the launch after the writers of
+ *               those buffers (a barrier across the GPUs) and keeps them unchanged until it ends.
+ *   O           out [rows, d] (float32 if out_is_f32, else bf16), LSE out [rows] or NULL: the slice
+ * Only plain loads touch the part buffers (no TMA, no multicast).  Requirements as
+ * pulsar_lse_merge_strided; row_begin + rows <= rows_total. */
+int32_t pulsar_lse_merge_peers(const float *const *part_bases, int32_t n_parts, int64_t rows_total,
+                               int64_t row_begin, int64_t rows, int32_t d,
+                               void *O, int32_t out_is_f32, float *LSE, void *stream);
+
 /* ------------------------------------------------------------------------------------------
  * Position ids of the assembled Phase-1 inputs and rotary embedding (Appendix E).
  *

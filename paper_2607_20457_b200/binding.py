@@ -33,7 +33,7 @@ EXPORTS = (
     "pulsar_pack_summary_kv", "pulsar_gather_kv_rows", "pulsar_phase1_attn_sharded", "pulsar_causal_varlen_attn",
     "pulsar_phase2_choose_splits", "pulsar_phase2_workspace_bytes", "pulsar_phase2_attn",
     "pulsar_phase2_generate_workspace_bytes", "pulsar_phase2_generate_step",
-    "pulsar_lse_merge", "pulsar_lse_merge_strided",
+    "pulsar_lse_merge", "pulsar_lse_merge_strided", "pulsar_lse_merge_peers",
     "pulsar_assemble_positions", "pulsar_rope_apply", "pulsar_rope_apply_qk",
 )
 
@@ -114,6 +114,8 @@ def load_library(build_if_missing: bool = False):
     lib.pulsar_phase2_generate_step.restype = i32
     lib.pulsar_lse_merge.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp]
     lib.pulsar_lse_merge.restype = i32
+    lib.pulsar_lse_merge_peers.argtypes = [vp, i32, i64, i64, i64, i32, vp, i32, vp, vp]
+    lib.pulsar_lse_merge_peers.restype = i32
     lib.pulsar_assemble_positions.argtypes = [vp, vp, i32, i32, i32, i32, vp, i64, vp, vp]
     lib.pulsar_assemble_positions.restype = i32
     lib.pulsar_rope_apply.argtypes = [vp, vp, i64, i32, i32, vp, ctypes.c_double, vp, vp]
@@ -507,3 +509,16 @@ def pulsar_rope_apply_qk(Q, K, positions, theta: float = 500000.0, q_out=None, k
                                   _p(status), _stream())
     _check("pulsar_rope_apply_qk", rc)
     return Qo, Ko
+
+
+def pulsar_lse_merge_peers(part_ptrs, rows_total: int, row_begin: int, rows: int, d: int, out, lse_out=None):
+    """Merge rows [row_begin, row_begin+rows) of the partials at the device addresses ``part_ptrs``
+    (ints: this GPU's buffers or peer-mapped ones, each laid out [rows_total*d | rows_total] float32).
+    ``out`` [rows, d] float32 or bf16 on the current device."""
+    lib = load_library()
+    n = len(part_ptrs)
+    table = (ctypes.c_void_p * n)(*[ctypes.c_void_p(int(p)) for p in part_ptrs])
+    rc = lib.pulsar_lse_merge_peers(ctypes.cast(table, ctypes.c_void_p), n, rows_total, row_begin, rows, d, _p(out),
+                                    1 if out.dtype == torch.float32 else 0, _p(lse_out), _stream())
+    _check("pulsar_lse_merge_peers", rc)
+    return out, lse_out

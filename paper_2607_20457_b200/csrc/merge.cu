@@ -111,6 +111,56 @@ lse_merge_lanes_kernel(const float* __restrict__ part_O, const float* __restrict
     if (LSE != nullptr && v == 0) LSE[row] = (m > -INFINITY) ? m + logf(denom) : -INFINITY;
 }
 
+// The merge with every part at its own address: part j is the buffer parts[j], laid out
+// [rows_total * d outputs | rows_total LSE] like the Phase-2 exchange buffer of a GPU, and only rows
+// [row0, row0 + rows) are merged.  The addresses may be peer-mapped memory of other GPUs: the kernel
+// then pulls its slice of every GPU's partial over NVLink with plain loads while it merges (no copy
+// engine, no TMA, no multicast) -- the all-gather and the merge in one pass, each GPU reducing 1/H of
+// the rows.
+constexpr int kMaxMergePeers = 64;
+struct PartTable {
+    const float* base[kMaxMergePeers];
+};
+
+template <bool kF32>
+__global__ void __launch_bounds__(256)
+lse_merge_table_kernel(const __grid_constant__ PartTable parts, int n_parts, int64_t rows_total, int64_t row0,
+                       int64_t rows, int d, void* __restrict__ O_, float* __restrict__ LSE) {
+    const int vec_per_row = d >> 2;
+    const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (idx >= rows * vec_per_row) return;
+    const int64_t r = idx / vec_per_row;
+    const int v = static_cast<int>(idx - r * vec_per_row);
+    const int64_t row = row0 + r;
+    const int64_t lse_at = rows_total * d + row;
+
+    float m = -INFINITY;
+#pragma unroll 8
+    for (int j = 0; j < n_parts; ++j) m = fmaxf(m, parts.base[j][lse_at]);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float denom = 0.f;
+    if (m > -INFINITY) {
+#pragma unroll 8
+        for (int j = 0; j < n_parts; ++j) {
+            const float w = __expf(parts.base[j][lse_at] - m);
+            const float4 o = *reinterpret_cast<const float4*>(parts.base[j] + row * d + v * 4);
+            denom += w;
+            acc.x += w * o.x; acc.y += w * o.y; acc.z += w * o.z; acc.w += w * o.w;
+        }
+        const float inv = 1.f / denom;
+        acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+    }
+    if (kF32) {
+        *reinterpret_cast<float4*>(static_cast<float*>(O_) + r * d + v * 4) = acc;
+    } else {
+        uint2 packed;
+        packed.x = pack_bf16x2(acc.x, acc.y);
+        packed.y = pack_bf16x2(acc.z, acc.w);
+        *reinterpret_cast<uint2*>(static_cast<uint16_t*>(O_) + r * d + v * 4) = packed;
+    }
+    if (LSE != nullptr && v == 0) LSE[r] = (m > -INFINITY) ? m + logf(denom) : -INFINITY;
+}
+
 namespace {
 int32_t launch_merge(const float* part_O, const float* part_LSE, int32_t n_parts, int64_t stride_O, int64_t stride_L,
                      int64_t rows, int32_t d, void* O, bool f32, float* LSE, cudaStream_t stream) {
@@ -175,4 +225,36 @@ extern "C" int32_t pulsar_lse_merge_strided(const float* part_O, const float* pa
     if (rc != PULSAR_OK) return rc;
     return launch_merge(part_O, part_LSE, n_parts, part_stride_O, part_stride_LSE, rows, d, O, out_is_f32 != 0, LSE,
                         static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int32_t pulsar_lse_merge_peers(const float* const* part_bases_host, int32_t n_parts, int64_t rows_total,
+                                          int64_t row_begin, int64_t rows, int32_t d, void* O, int32_t out_is_f32,
+                                          float* LSE, void* stream) {
+    if (n_parts < 1 || n_parts > kMaxMergePeers || rows_total < 0 || row_begin < 0 || rows < 0 || d <= 0 ||
+        !part_bases_host)
+        return PULSAR_ERR_INVALID_ARG;
+    if (d % 4 != 0 || d > 1024 || row_begin + rows > rows_total) return PULSAR_ERR_SHAPE;
+    if (rows == 0) return PULSAR_OK;
+    if (!O) return PULSAR_ERR_INVALID_ARG;
+    PartTable t{};
+    for (int j = 0; j < n_parts; ++j) {
+        if (!part_bases_host[j]) return PULSAR_ERR_INVALID_ARG;
+        if (!aligned(part_bases_host[j], 16)) return PULSAR_ERR_ALIGNMENT;
+        t.base[j] = part_bases_host[j];
+    }
+    if (!aligned(O, out_is_f32 ? 16 : 8) || !aligned(LSE, 4)) return PULSAR_ERR_ALIGNMENT;
+    int32_t rc = check_device();
+    if (rc != PULSAR_OK) return rc;
+    const int64_t blocks = (rows * (d >> 2) + 255) / 256;
+    if (blocks > 0x7fffffffll) return PULSAR_ERR_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (out_is_f32)
+        lse_merge_table_kernel<true><<<static_cast<unsigned>(blocks), 256, 0, st>>>(t, n_parts, rows_total, row_begin, rows,
+                                                                                   d, O, LSE);
+    else
+        lse_merge_table_kernel<false><<<static_cast<unsigned>(blocks), 256, 0, st>>>(t, n_parts, rows_total, row_begin,
+                                                                                    rows, d, O, LSE);
+    PULSAR_CUDA_OK(cudaGetLastError());
+    count_launch();
+    return PULSAR_OK;
 }

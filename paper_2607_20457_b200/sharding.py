@@ -10,7 +10,10 @@ memory followed by a kernel that reads only local memory:
   ``pulsar_phase1_attn_sharded`` attends over the local blocks.
 * Phase 2: each rank attends the query to its retained KV (``pulsar_phase2_attn``), merges its
   own parts into one float32 partial (``pulsar_lse_merge_strided``); the partials (o_h, l_h) are
-  all-gathered and every rank merges the gathered set.
+  all-gathered and every rank merges the gathered set.  ``phase2_fused`` instead lets rank r merge
+  1/H of the rows straight out of every rank's peer-mapped partial (``pulsar_lse_merge_peers``:
+  the exchange and the merge in one kernel, H times fewer bytes over NVLink) and gathers the bf16
+  slices.
 
 All arithmetic is in the CUDA library; this module computes layouts on the host and calls the
 collective.  ``TorchCollective`` wraps ``torch.distributed``; a test can pass any object with
@@ -112,6 +115,49 @@ class SingleRankCollective:
         return send.unsqueeze(0)
 
 
+class LocalPeers:
+    """Peer buffers of ranks that live in one process on one GPU (tests): a registry of the
+    ranks' exchange buffers, whose device addresses every rank can read directly."""
+
+    def __init__(self, world: int):
+        self.world = world
+        self.buffers = [None] * world
+
+    def alloc(self, rank: int, nfloats: int, device) -> torch.Tensor:
+        self.buffers[rank] = torch.empty(nfloats, dtype=torch.float32, device=device)
+        return self.buffers[rank]
+
+    def ptrs(self):
+        return [b.data_ptr() for b in self.buffers]
+
+    def barrier(self):
+        pass                                  # the ranks run one after the other
+
+
+class SymmetricMemoryPeers:
+    """Peer buffers through ``torch.distributed._symmetric_memory``: every rank allocates the same
+    buffer, the rendezvous maps all of them into every process.  NOT RUN ON MORE THAN ONE GPU in
+    this build (none was available); the one-GPU tests cover the kernel through ``LocalPeers``."""
+
+    def __init__(self, group=None):
+        import torch.distributed as dist
+        import torch.distributed._symmetric_memory as symm_mem
+        self._symm, self.group = symm_mem, group if group is not None else dist.group.WORLD
+        self.world = dist.get_world_size(self.group)
+        self.handle = None
+
+    def alloc(self, rank: int, nfloats: int, device) -> torch.Tensor:
+        t = self._symm.empty(nfloats, dtype=torch.float32, device=device)
+        self.handle = self._symm.rendezvous(t, self.group)
+        return t
+
+    def ptrs(self):
+        return [int(p) for p in self.handle.buffer_ptrs]
+
+    def barrier(self):
+        self.handle.barrier()                 # a device-side barrier enqueued on the current stream
+
+
 class ShardedContextEncoder:
     """One rank's part of the sharded context encoding.  ``collective`` supplies all_gather."""
 
@@ -191,6 +237,59 @@ class ShardedContextEncoder:
         self.b.pulsar_lse_merge_strided(flat, flat[rows * self.d:], gathered.shape[0], stride, stride, rows, self.d,
                                         O.view(rows, self.d), LSE.view(rows))
         return O, LSE
+
+    # ---- Phase 2 with the exchange fused into the merge (each rank reduces 1/H of the rows) --------
+    def row_slice(self, nq: int):
+        """Rows of the [nq*Hq, d] result this rank merges: (first row, count)."""
+        rows = nq * self.Hq
+        per = (rows + self.lay.n_hosts - 1) // self.lay.n_hosts
+        begin = min(self.rank * per, rows)
+        return begin, min(per, rows - begin)
+
+    def phase2_local_into(self, peers, Qq, K, V, softmax_scale: float = 0.0, n_splits: int = 0):
+        """As phase2_local, with (o_h, l_h) written to this rank's peer-visible buffer."""
+        nq = Qq.shape[0]
+        if getattr(self, "_peer_buf_nq", None) != nq:
+            self._peer_buf = peers.alloc(self.rank, self.partial_stride(nq), self.dev)
+            self._peer_buf_nq = nq
+        lay, rows = self.lay, nq * self.Hq
+        J = n_splits or self.b.phase2_choose_splits(nq, lay.n_local, lay.block_size, self.Hq, self.Hkv, self.d)
+        _, _, pO, pL = self.b.pulsar_phase2_attn(Qq, K, V, lay.n_local, lay.block_size, softmax_scale, n_splits=J,
+                                                 want_partials=True, status=self.status)
+        send = self._peer_buf
+        self.b.pulsar_lse_merge_strided(pO.view(-1), pL.view(-1), J, rows * self.d, rows, rows, self.d,
+                                        send[: rows * self.d].view(rows, self.d), send[rows * self.d:])
+        return send
+
+    def phase2_merge_slice(self, peers, nq: int):
+        """This rank's slice of the merged result, read from every rank's buffer in place
+        (``pulsar_lse_merge_peers``).  Call after ``peers.barrier()``; returns (O bf16 [n,d], LSE [n],
+        first row)."""
+        rows = nq * self.Hq
+        begin, n = self.row_slice(nq)
+        O = torch.empty((max(n, 1), self.d), dtype=torch.bfloat16, device=self.dev)
+        LSE = torch.empty(max(n, 1), dtype=torch.float32, device=self.dev)
+        if n > 0:
+            self.b.pulsar_lse_merge_peers(peers.ptrs(), rows, begin, n, self.d, O, LSE)
+        return O[:n], LSE[:n], begin
+
+    def phase2_fused(self, peers, Qq, K, V, softmax_scale: float = 0.0, n_splits: int = 0):
+        """Phase 2 with the partial exchange fused into the merge; the bf16 slices are then gathered
+        with the collective so that every rank holds the whole result."""
+        nq = Qq.shape[0]
+        rows = nq * self.Hq
+        self.phase2_local_into(peers, Qq, K, V, softmax_scale, n_splits)
+        peers.barrier()                                     # stream-ordered: every buffer is complete before it is read
+        O, LSE, _ = self.phase2_merge_slice(peers, nq)
+        per = (rows + self.lay.n_hosts - 1) // self.lay.n_hosts
+        o_pad = torch.zeros((per, self.d), dtype=torch.bfloat16, device=self.dev)
+        l_pad = torch.zeros(per, dtype=torch.float32, device=self.dev)
+        o_pad[: O.shape[0]] = O
+        l_pad[: LSE.shape[0]] = LSE
+        Oall = self.coll.all_gather(o_pad).reshape(-1, self.d)[:rows].view(nq, self.Hq, self.d)
+        Lall = self.coll.all_gather(l_pad).reshape(-1)[:rows].view(nq, self.Hq)
+        peers.barrier()                                     # nobody overwrites its buffer while others still read
+        return Oall, Lall
 
     def phase2(self, Qq, K, V, softmax_scale: float = 0.0, n_splits: int = 0):
         send = self.phase2_local(Qq, K, V, softmax_scale, n_splits)

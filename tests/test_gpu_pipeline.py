@@ -45,12 +45,14 @@ def test_host_and_pipelined_steps_equal_the_device_step_and_the_oracle_selection
     assert int(enc.status.item()) == 0
 
 
-def test_bench_block_sharded_mode_runs_and_reports():
+@pytest.mark.parametrize("exchange", ["allgather", "fused"])
+def test_bench_block_sharded_mode_runs_and_reports(exchange):
     """`bench.py --shard blocks` at one rank: same contract line, strong scaling, clean status."""
     import json, os, subprocess, sys
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--workload", "tiny", "--shard", "blocks",
-                          "--steps", "3", "--warmup", "3"], capture_output=True, text=True, timeout=600)
+                          "--exchange", exchange, "--steps", "3", "--warmup", "3"], capture_output=True, text=True,
+                         timeout=600)
     assert out.returncode == 0, out.stderr[-2000:]
     line = json.loads(out.stdout.strip().splitlines()[-1])
     assert line["scaling"] == "strong" and line["config"]["shard"] == "blocks" and line["device_status"] == 0

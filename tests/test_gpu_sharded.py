@@ -127,3 +127,36 @@ def test_gather_rows_and_bad_index():
     idx[2] = 300
     binding.pulsar_gather_kv_rows(K, V, idx, Ko, Vo, status=st)
     assert int(st.item()) & 0x2 and torch.equal(Ko[2], K[0])
+
+
+@pytest.mark.parametrize("H,nq", [(1, 5), (2, 37), (4, 1), (4, 130)])
+def test_phase2_with_the_exchange_fused_into_the_merge(H, nq):
+    """Every rank merges its slice of the rows straight from all ranks' partial buffers (here all on
+    one GPU, addressed through a pointer table as peer memory would be)."""
+    from paper_2607_20457_b200.sharding import LocalPeers
+    w = W.CONFIGS["tiny"]
+    _, K, V = (t.to(DEV) for t in W.qkv(w))
+    Qq = W.phase2_query(w)
+    Qq = Qq.repeat((nq + Qq.shape[0] - 1) // Qq.shape[0], 1, 1)[:nq].contiguous().to(DEV)
+    lay, ranks = make_ranks(w, H, "zigzag")
+    peers = LocalPeers(H)
+    for h, r in enumerate(ranks):
+        rows = torch.from_numpy(lay.local_token_rows(h)).to(DEV)
+        r.phase2_local_into(peers, Qq, K[rows].contiguous(), V[rows].contiguous())
+    n_rows = nq * w.Hq
+    O = torch.empty((n_rows, w.d), dtype=torch.bfloat16, device=DEV)
+    LSE = torch.empty(n_rows, dtype=torch.float32, device=DEV)
+    covered = 0
+    for r in ranks:
+        o, lse, begin = r.phase2_merge_slice(peers, nq)
+        O[begin: begin + o.shape[0]] = o
+        LSE[begin: begin + o.shape[0]] = lse
+        covered += o.shape[0]
+    torch.cuda.synchronize()
+    assert covered == n_rows
+    O_ref, LSE_ref = oracle.phase2_attn(Qq.cpu(), K.cpu(), V.cpu(), w.n_blocks, w.block_size)
+    check_attention(O.view(nq, w.Hq, w.d), LSE.view(nq, w.Hq), O_ref, LSE_ref, f"fused exchange H={H} nq={nq}")
+    # and it is the all-gather path's result exactly (same parts, same order)
+    sends = torch.stack([p.clone() for p in peers.buffers])
+    O2, LSE2 = ranks[0].phase2_finish(sends, nq)
+    assert torch.equal(O2.view(n_rows, w.d), O) and torch.equal(LSE2.view(n_rows), LSE)
