@@ -136,8 +136,8 @@ class LocalPeers:
 
 class SymmetricMemoryPeers:
     """Peer buffers through ``torch.distributed._symmetric_memory``: every rank allocates the same
-    buffer, the rendezvous maps all of them into every process.  NOT RUN ON MORE THAN ONE GPU in
-    this build (none was available); the one-GPU tests cover the kernel through ``LocalPeers``."""
+    buffer, the rendezvous maps all of them into every process.  Exercised with one rank only (no
+    machine with several GPUs was available); the kernel itself is covered through ``LocalPeers``."""
 
     def __init__(self, group=None):
         import torch.distributed as dist

@@ -160,3 +160,39 @@ def test_phase2_with_the_exchange_fused_into_the_merge(H, nq):
     sends = torch.stack([p.clone() for p in peers.buffers])
     O2, LSE2 = ranks[0].phase2_finish(sends, nq)
     assert torch.equal(O2.view(n_rows, w.d), O) and torch.equal(LSE2.view(n_rows), LSE)
+
+
+_SYMM_WORLD1 = r"""
+import os, sys, torch, torch.distributed as dist
+os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(29650 + os.getpid() % 200), RANK="0", WORLD_SIZE="1")
+torch.cuda.set_device(0)
+dist.init_process_group("nccl", device_id=torch.device("cuda", 0))
+from paper_2607_20457_b200 import binding, workloads as W
+from paper_2607_20457_b200.sharding import ShardLayout, ShardedContextEncoder, SymmetricMemoryPeers, TorchCollective
+w = W.CONFIGS["tiny"]
+_, K, V = (t.cuda() for t in W.qkv(w))
+Qq = W.phase2_query(w).cuda()
+lay = ShardLayout.make(w.n_blocks, 1, w.block_size, w.chunk, w.k, w.sink, "zigzag")
+enc = ShardedContextEncoder(lay, 0, w.Hq, w.Hkv, w.d, w.vocab_size, "cuda:0", TorchCollective())
+peers = SymmetricMemoryPeers()
+O, LSE = enc.phase2_fused(peers, Qq, K, V)
+O2, LSE2 = enc.phase2(Qq, K, V)                      # NCCL all-gather path at world size 1
+O1, LSE1 = binding.pulsar_phase2_attn(Qq, K, V, w.n_blocks, w.block_size)
+torch.cuda.synchronize()
+assert torch.equal(O, O2) and torch.equal(LSE, LSE2)
+assert (O.float() - O1.float()).abs().max().item() < 1e-2 and (LSE - LSE1).abs().max().item() < 1e-3
+assert int(enc.status.item()) == 0
+dist.destroy_process_group()
+print("SYMM-OK")
+"""
+
+
+def test_symmetric_memory_and_nccl_plumbing_at_world_size_one():
+    """The rendezvous, the device-side barrier and the NCCL all-gather as one rank (the only
+    multi-process configuration a single GPU allows)."""
+    import os, subprocess, sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, PYTHONPATH=root + os.pathsep + os.environ.get("PYTHONPATH", ""))
+    out = subprocess.run([sys.executable, "-c", _SYMM_WORLD1], capture_output=True, text=True, timeout=600, env=env,
+                         cwd=root)
+    assert out.returncode == 0 and "SYMM-OK" in out.stdout, (out.stdout + out.stderr)[-3000:]
