@@ -153,3 +153,19 @@ def test_non_monotone_prefix_lengths():
     pidx = pidx.copy()
     pidx[:] = np.arange(len(pidx)) % 512                       # all entries lie in block 0
     print(run_phase1(w, Q, K, V, pidx, plen, what="non-monotone"))
+
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_logits_that_jump_far_above_the_running_maximum(d):
+    """Key magnitudes grow along the sequence in steps, some in the first and some in the second
+    half of a 128-key tile, so that later tiles hold logits tens of nats above everything seen
+    before: the kernel has to move its running maximum in the middle of a row, also after the first
+    half of a tile has already gone to the tensor cores."""
+    w = W.shrink(W.CONFIGS["tiny"], L=2048, block_size=1024, chunk=16, k=4, sink=64, Hq=4, Hkv=2, d=d)
+    Q, K, V = W.qkv(w, seed=31)
+    Kf = K.float()
+    for start, factor in ((200, 6.0), (330, 14.0), (520, 30.0), (1024 + 150, 8.0), (1024 + 600, 40.0), (1024 + 840, 90.0)):
+        Kf[start: start + 40] *= factor
+    K = Kf.bfloat16()
+    pidx, plen = W.first_k_prefix(w)
+    print(run_phase1(w, Q, K, V, pidx, plen, what=f"jumping logits d={d}"))
