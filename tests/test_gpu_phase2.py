@@ -39,6 +39,13 @@ def test_tiny_peaked():
     dict(L=768, block_size=192, Hq=8, Hkv=1, d=64, nq=17),        # g = 8, ragged rows
     dict(L=512, block_size=128, Hq=2, Hkv=2, d=128, nq=130),      # g = 1, more than one row tile
     dict(L=640, block_size=320, Hq=16, Hkv=1, d=64, nq=9),        # g = 16
+    # decode shapes: at most 32 query rows per KV head, each softmax warp takes a quarter of the keys
+    dict(L=640, block_size=320, Hq=16, Hkv=1, d=64, nq=2),        # g = 16, 32 rows
+    dict(L=900, block_size=300, Hq=8, Hkv=1, d=128, nq=3),        # g = 8, 24 rows, ragged keys
+    dict(L=512, block_size=256, Hq=2, Hkv=2, d=128, nq=32),       # g = 1, 32 rows
+    dict(L=512, block_size=256, Hq=2, Hkv=2, d=64, nq=33),        # g = 1, one row too many for that mode
+    dict(L=1152, block_size=384, Hq=4, Hkv=2, d=128, nq=16),      # g = 2, 32 rows
+    dict(L=90, block_size=45, Hq=4, Hkv=1, d=64, nq=5),           # fewer keys than one tile
 ])
 @pytest.mark.parametrize("n_splits", [1, 2])
 def test_small_shapes(shape, n_splits):
