@@ -57,7 +57,7 @@ class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
+              "clocks_event_reasons.sw_power_cap,power.draw.instant")
 
     def __init__(self, device_index: int):
         self.proc = None
@@ -81,7 +81,7 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
             out = ""
-        sm, mx, power, reasons = [], [], [], set()
+        sm, mx, power, instant, reasons = [], [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in out.strip().splitlines():
             f = [x.strip() for x in line.split(",")]
@@ -94,10 +94,14 @@ class ClockSampler:
             for n, v in zip(names, f[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
+            try:                                   # power.draw is a running average; this one is not
+                instant.append(float(f[7]))
+            except (IndexError, ValueError):
+                pass
         if not sm:
             return dict(sm_mhz=None, sm_max_mhz=None, reasons=["unsampled"])
-        return dict(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), power_w_max=max(power), samples=len(sm),
-                    reasons=sorted(reasons))
+        return dict(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), power_w_max=max(power),
+                    power_w_instant_max=max(instant) if instant else None, samples=len(sm), reasons=sorted(reasons))
 
 
 def dist_setup(n_gpus: int):
