@@ -104,3 +104,15 @@ def host_costs(pi, block_cost):
 def critical_path(pi, block_cost):
     """C_crit = max_h C_h (Eq. 15)."""
     return max(host_costs(pi, block_cost))
+
+
+# ---- position ids of the Phase-2 query (Appendix E) ---------------------------------------------
+def phase2_query_position_start(L: int, n_blocks: int, sink: int, sigma: int, mode: str = "sparse") -> int:
+    """First position id of the query tokens.  Sparse mode keeps global positions, so the query
+    follows the context at L.  In contiguous mode every Phase-1 input was renumbered from 0, and the
+    query starts just past the longest of them, n_{B-1} = L/B + sink + (B-1)*sigma (n_0 = L/B)."""
+    if mode == "sparse":
+        return L
+    if mode == "contiguous":
+        return max(paper_input_len(L, n_blocks, sink, sigma, i) for i in range(n_blocks))
+    raise ValueError(f"unknown position mode {mode!r}")

@@ -79,3 +79,10 @@ def test_config_sizes():
     star = [0] + [w4.block_size] * (w4.n_blocks - 1)
     ratio = cm.phase1_pairs(w4.block_size, star) / cm.phase1_pairs(w4.block_size, pl4)
     assert abs(ratio - 1.895) < 0.001
+
+
+def test_phase2_query_positions():
+    # the paper's 128K setting: B = 8 blocks of 16K, sink 64, sigma 512 -> longest input 16384 + 64 + 7*512
+    assert cm.phase2_query_position_start(131072, 8, 64, 512, "sparse") == 131072
+    assert cm.phase2_query_position_start(131072, 8, 64, 512, "contiguous") == 16384 + 64 + 3584
+    assert cm.phase2_query_position_start(4096, 1, 64, 512, "contiguous") == 4096      # one block: no prefix at all
