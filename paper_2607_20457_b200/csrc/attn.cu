@@ -11,7 +11,12 @@
 //            the block's own rows up to the diagonal tile (causal mask on that tile only).
 //   Phase 2: rows = (128/g tokens) x (the g query heads of one KV head); key tiles = one
 //            contiguous part of the retained KV, no mask; output is the fp32 partial (A_j, l_j)
-//            or, with a single part, the final bf16 result.
+//            or, with a single part, the final bf16 result.  With at most 32 such rows (decode)
+//            the rows are replicated into the four lane quarters of the tile and each softmax
+//            warp takes a quarter of the keys; the generation shard of Algorithm 1 l.11-16 is
+//            one more part, causal by token.
+//   Assembled inputs (Algorithm 1 l.8 as the paper runs it): sequences of any lengths packed back
+//            to back, every token a query, plain causal attention inside each.
 #include <cuda.h>
 
 #include "common.cuh"
