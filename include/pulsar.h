@@ -307,6 +307,18 @@ int32_t pulsar_causal_varlen_attn(const uint16_t *Q, const uint16_t *K, const ui
                                   void *workspace, size_t workspace_bytes,
                                   int32_t *device_status, void *stream);
 
+/* KV discard after the pass over assembled inputs (Section 3.1 "KV discard", Appendix F): the keys
+ * and values of the sink and summary tokens are dropped, the last block_size rows of every
+ * assembled input -- the block's own -- are kept, so that the retained cache holds every context
+ * token exactly once.
+ *   K, V        in  [total_rows, Hkv, d] bf16, the inputs packed as for pulsar_causal_varlen_attn
+ *   cu_seqlens  in  HOST pointer [n_seq + 1]; every input must be at least block_size rows long
+ *   K_ret, V_ret out [n_seq * block_size, Hkv, d] bf16
+ * Requirements (else PULSAR_ERR_SHAPE): 1 <= n_seq <= 64, Hkv*d*2 % 16 == 0. */
+int32_t pulsar_retain_block_kv(const uint16_t *K, const uint16_t *V, int64_t total_rows,
+                               const int32_t *cu_seqlens, int32_t n_seq, int32_t block_size,
+                               int32_t Hkv, int32_t d, uint16_t *K_ret, uint16_t *V_ret, void *stream);
+
 /* ------------------------------------------------------------------------------------------
  * Phase-2 query attention over the retained KV of all blocks, merged exactly (Section 3.2;
  * Algorithm 1 lines 12-13; Appendix H).

@@ -31,6 +31,7 @@ EXPORTS = (
     "pulsar_chunk_select_workspace_bytes", "pulsar_chunk_select",
     "pulsar_phase1_workspace_bytes", "pulsar_phase1_attn",
     "pulsar_pack_summary_kv", "pulsar_gather_kv_rows", "pulsar_phase1_attn_sharded", "pulsar_causal_varlen_attn",
+    "pulsar_retain_block_kv",
     "pulsar_phase2_choose_splits", "pulsar_phase2_workspace_bytes", "pulsar_phase2_attn",
     "pulsar_phase2_generate_workspace_bytes", "pulsar_phase2_generate_step",
     "pulsar_lse_merge", "pulsar_lse_merge_strided", "pulsar_lse_merge_peers",
@@ -116,6 +117,8 @@ def load_library(build_if_missing: bool = False):
     lib.pulsar_lse_merge.restype = i32
     lib.pulsar_lse_merge_peers.argtypes = [vp, i32, i64, i64, i64, i32, vp, i32, vp, vp]
     lib.pulsar_lse_merge_peers.restype = i32
+    lib.pulsar_retain_block_kv.argtypes = [vp, vp, i64, vp, i32, i32, i32, i32, vp, vp, vp]
+    lib.pulsar_retain_block_kv.restype = i32
     lib.pulsar_assemble_positions.argtypes = [vp, vp, i32, i32, i32, i32, vp, i64, vp, vp]
     lib.pulsar_assemble_positions.restype = i32
     lib.pulsar_rope_apply.argtypes = [vp, vp, i64, i32, i32, vp, ctypes.c_double, vp, vp]
@@ -522,3 +525,19 @@ def pulsar_lse_merge_peers(part_ptrs, rows_total: int, row_begin: int, rows: int
                                     1 if out.dtype == torch.float32 else 0, _p(lse_out), _stream())
     _check("pulsar_lse_merge_peers", rc)
     return out, lse_out
+
+
+def pulsar_retain_block_kv(K, V, cu_seqlens, block_size: int):
+    """The retained KV of assembled inputs: the last ``block_size`` rows of every input.  K, V
+    [total_rows,Hkv,d] CUDA bf16, cu_seqlens a host sequence.  Returns (K_ret, V_ret) [n_seq*block_size,Hkv,d]."""
+    lib = load_library()
+    _need(K, torch.bfloat16, "K")
+    _need(V, torch.bfloat16, "V")
+    cu = (ctypes.c_int32 * len(cu_seqlens))(*[int(x) for x in cu_seqlens])
+    n_seq = len(cu_seqlens) - 1
+    Kr = torch.empty((n_seq * block_size,) + tuple(K.shape[1:]), dtype=torch.bfloat16, device=K.device)
+    Vr = torch.empty_like(Kr)
+    rc = lib.pulsar_retain_block_kv(_p(K), _p(V), K.shape[0], ctypes.cast(cu, ctypes.c_void_p), n_seq, block_size,
+                                    K.shape[1], K.shape[2], _p(Kr), _p(Vr), _stream())
+    _check("pulsar_retain_block_kv", rc)
+    return Kr, Vr

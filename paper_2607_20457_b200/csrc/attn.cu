@@ -110,6 +110,24 @@ append_kv_kernel(const uint4* __restrict__ Knew, const uint4* __restrict__ Vnew,
     }
 }
 
+// KV discard (Section 3.1, Appendix F): of every assembled input only the last block_size rows -- the
+// block's own keys and values -- are kept.  first[j] = first kept row of input j.
+struct RetainTable {
+    int first[kMaxVarlenSeqs];
+};
+__global__ void __launch_bounds__(128)
+retain_block_kv_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V, const __grid_constant__ RetainTable tab,
+                       int block_size, int row_vecs, uint4* __restrict__ Kret, uint4* __restrict__ Vret) {
+    const int row = blockIdx.x;                              // retained row: input row / block_size, offset row % block_size
+    const int j = row / block_size;
+    const size_t src = static_cast<size_t>(tab.first[j] + (row - j * block_size)) * row_vecs;
+    const size_t dst = static_cast<size_t>(row) * row_vecs;
+    for (int v = threadIdx.x; v < row_vecs; v += blockDim.x) {
+        Kret[dst + v] = K[src + v];
+        Vret[dst + v] = V[src + v];
+    }
+}
+
 // Row gather without the prefix check: Kout[j] = K[idx[j]], Vout[j] = V[idx[j]].  An index outside
 // [0, rows_in) is reported and row 0 used.
 __global__ void __launch_bounds__(128)
@@ -1514,4 +1532,30 @@ extern "C" int32_t pulsar_causal_varlen_attn(const uint16_t* Q, const uint16_t* 
     a.status = device_status;
     return d == 128 ? launch_attn<128>(tmQ, tmK, tmV, tmK, tmV, a, stream, &vt)
                     : launch_attn<64>(tmQ, tmK, tmV, tmK, tmV, a, stream, &vt);
+}
+
+extern "C" int32_t pulsar_retain_block_kv(const uint16_t* K, const uint16_t* V, int64_t total_rows,
+                                          const int32_t* cu_seqlens_host, int32_t n_seq, int32_t block_size,
+                                          int32_t Hkv, int32_t d, uint16_t* K_ret, uint16_t* V_ret, void* stream) {
+    if (total_rows <= 0 || n_seq <= 0 || block_size <= 0 || Hkv <= 0 || d <= 0 || !cu_seqlens_host)
+        return PULSAR_ERR_INVALID_ARG;
+    if (n_seq > kMaxVarlenSeqs || total_rows >= (1ll << 31) || (static_cast<int64_t>(Hkv) * d * 2) % 16 != 0 ||
+        static_cast<int64_t>(n_seq) * block_size >= (1ll << 31))
+        return PULSAR_ERR_SHAPE;
+    if (cu_seqlens_host[0] != 0 || cu_seqlens_host[n_seq] != total_rows) return PULSAR_ERR_SHAPE;
+    RetainTable tab{};
+    for (int j = 0; j < n_seq; ++j) {
+        if (cu_seqlens_host[j + 1] - cu_seqlens_host[j] < block_size) return PULSAR_ERR_SHAPE;   // shorter than a block
+        tab.first[j] = cu_seqlens_host[j + 1] - block_size;
+    }
+    if (!K || !V || !K_ret || !V_ret) return PULSAR_ERR_INVALID_ARG;
+    if (!aligned(K, 16) || !aligned(V, 16) || !aligned(K_ret, 16) || !aligned(V_ret, 16)) return PULSAR_ERR_ALIGNMENT;
+    int32_t rc = check_device();
+    if (rc != PULSAR_OK) return rc;
+    retain_block_kv_kernel<<<n_seq * block_size, 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        reinterpret_cast<const uint4*>(K), reinterpret_cast<const uint4*>(V), tab, block_size, Hkv * d * 2 / 16,
+        reinterpret_cast<uint4*>(K_ret), reinterpret_cast<uint4*>(V_ret));
+    PULSAR_CUDA_OK(cudaGetLastError());
+    count_launch();
+    return PULSAR_OK;
 }

@@ -82,3 +82,28 @@ def test_bad_offsets_are_rejected_on_the_host():
         with pytest.raises(binding.PulsarError) as e:
             binding.pulsar_causal_varlen_attn(z, z, z, cu)
         assert e.value.status == 2
+
+
+def test_kv_discard_keeps_each_blocks_own_rows():
+    """Appendix F: after the pass over the assembled inputs only the last block_size rows of each are
+    kept -- the same rows a boolean mask that is true on the last block_size positions selects --
+    and the retained cache is the original K, V (every context token once)."""
+    w = W.CONFIGS["tiny"]
+    _, K, V = W.qkv(w)
+    pidx, plen = W.first_k_prefix(w)
+    rows, cu = [], [0]
+    for i in range(w.n_blocks):
+        rows += list(pidx[: plen[i]]) + list(range(i * w.block_size, (i + 1) * w.block_size))
+        cu.append(len(rows))
+    idx = torch.tensor(rows)
+    Ka, Va = K[idx].contiguous().to(DEV), V[idx].contiguous().to(DEV)
+    Kr, Vr = binding.pulsar_retain_block_kv(Ka, Va, cu, w.block_size)
+    torch.cuda.synchronize()
+    for i in range(w.n_blocks):
+        is_bi = torch.zeros(cu[i + 1] - cu[i], dtype=torch.bool)
+        is_bi[-w.block_size:] = True
+        seg = Ka[cu[i]: cu[i + 1]].cpu()[is_bi]
+        assert torch.equal(Kr[i * w.block_size: (i + 1) * w.block_size].cpu(), seg)
+    assert torch.equal(Kr.cpu(), K) and torch.equal(Vr.cpu(), V)
+    with pytest.raises(binding.PulsarError):
+        binding.pulsar_retain_block_kv(Ka, Va, cu, w.block_size + cu[1] + 1)       # longer than the first input
