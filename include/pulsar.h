@@ -340,6 +340,11 @@ int32_t pulsar_retain_block_kv(const uint16_t *K, const uint16_t *V, int64_t tot
  *   part_O      out [n_splits, nq, Hq, d] float32 or NULL (requires n_splits > 0)
  *   part_LSE    out [n_splits, nq, Hq]    float32 or NULL (both or neither)
  *
+ *   workspace   pulsar_phase2_workspace_bytes(...) bytes, 256-byte aligned: the partials when the
+ *               caller passes none.  Decode shapes (nq * Hq/Hkv <= 32, no caller partials) keep
+ *               four partials per part -- each softmax warp works on its own copy of the rows and
+ *               a quarter of every key tile -- and therefore need it even with a single part.
+ *
  * Requirements (else PULSAR_ERR_SHAPE): d in {64,128}; Hq % Hkv == 0; Hq/Hkv in {1,2,4,8,16};
  * nq >= 1.  pulsar_phase2_choose_splits returns the value used for n_splits == 0.
  * ------------------------------------------------------------------------------------------ */
