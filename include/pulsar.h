@@ -436,7 +436,7 @@ int32_t pulsar_lse_merge_strided(const float *part_O, const float *part_LSE, int
  *               float32 LSE]; n_parts <= 64.  The caller orders the launch after the writers of
  *               those buffers (a barrier across the GPUs) and keeps them unchanged until it ends.
  *   O           out [rows, d] (float32 if out_is_f32, else bf16), LSE out [rows] or NULL: the slice
- * Only plain loads touch the part buffers (no TMA, no multicast).  Requirements as
+ * Only plain loads touch the part buffers (no TMA).  Requirements as
  * pulsar_lse_merge_strided; row_begin + rows <= rows_total. */
 int32_t pulsar_lse_merge_peers(const float *const *part_bases, int32_t n_parts, int64_t rows_total,
                                int64_t row_begin, int64_t rows, int32_t d,

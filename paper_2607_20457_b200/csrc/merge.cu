@@ -118,7 +118,7 @@ lse_merge_lanes_kernel(const float* __restrict__ part_O, const float* __restrict
 // [rows_total * d outputs | rows_total LSE] like the Phase-2 exchange buffer of a GPU, and only rows
 // [row0, row0 + rows) are merged.  The addresses may be peer-mapped memory of other GPUs: the kernel
 // then pulls its slice of every GPU's partial over NVLink with plain loads while it merges (no copy
-// engine, no TMA, no multicast) -- the all-gather and the merge in one pass, each GPU reducing 1/H of
+// engine, no TMA) -- the all-gather and the merge in one pass, each GPU reducing 1/H of
 // the rows.
 constexpr int kMaxMergePeers = 64;
 struct PartTable {
