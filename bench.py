@@ -557,6 +557,23 @@ def run_extras(binding, w, dev, K_d, V_d, peaks):
         ms=t["median_ms"], rows=cu[-1], bytes=rope_bytes, gbs=rope_bytes / (t["median_ms"] * 1e-3) / 1e9,
         frac_of_measured_hbm=rope_bytes / (t["median_ms"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
         what="Q (32 heads) and K (8 heads) of all assembled inputs, read once and written once")
+    # whole steps at the small configurations, launched call by call and replayed as one CUDA graph
+    from paper_2607_20457_b200.pipeline import ContextEncoder
+    graph_res = {}
+    for name in ("tiny", "16k"):
+        ws_ = W.CONFIGS[name]
+        enc_s = ContextEncoder(ws_, dev)
+        sl = enc_s.slots[0]
+        sl["ids"].copy_(torch.from_numpy(W.token_ids(ws_).view(np.int32)))
+        for nm, t_ in zip(("Q", "K", "V"), W.qkv(ws_)):
+            sl[nm].copy_(t_)
+        sl["Qq"].copy_(W.phase2_query(ws_))
+        eager = time_calls(lambda: enc_s.step_device(sl["ids"], sl["Q"], sl["K"], sl["V"], sl["Qq"]), 20)
+        graph, _ = enc_s.capture_step()
+        replay = time_calls(graph.replay, 20)
+        graph_res[name] = dict(call_by_call_ms=eager["median_ms"], graph_replay_ms=replay["median_ms"])
+        del graph, enc_s
+    out["step_as_cuda_graph"] = graph_res
     res["flop_ratio_star_over_pulsar"] = res["star_anchor"]["tflop"] / res["pulsar"]["tflop"]
     res["time_ratio_star_over_pulsar"] = res["star_anchor"]["ms"] / res["pulsar"]["ms"]
     out["phase1_64k_prefix_comparison"] = res

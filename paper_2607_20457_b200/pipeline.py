@@ -6,7 +6,8 @@ already resident on the GPU.  ``step_host`` takes pinned host tensors, copies th
 in, runs the same three C-ABI calls and copies every result back to pinned host
 memory.  ``run_host_pipelined`` does that for a sequence of steps with two buffer
 sets and three streams, so that one step's copies overlap its neighbours'
-compute (PCIe is full duplex).  All arithmetic happens in the library's kernels.
+compute (PCIe is full duplex).  ``capture_step`` records a step as a CUDA graph.  All
+arithmetic happens in the library's kernels.
 """
 from __future__ import annotations
 
@@ -76,6 +77,23 @@ class ContextEncoder:
         if record:
             record[3].record()
         return dict(sel=sel, O1=O1, LSE1=LSE1, O2=O2, LSE2=LSE2, prefix_idx=sel["prefix_idx"])
+
+    def capture_step(self, slot_index: int = 0):
+        """The three calls of a step captured once as a CUDA graph on the slot's own device buffers
+        (fill ``slots[i]["ids" | "Q" | "K" | "V" | "Qq"]``, then ``graph.replay()``): one launch from
+        the host instead of nine, which matters when a step is shorter than the host's launch cadence.
+        Returns (graph, results); the results are the slot's output tensors."""
+        slot = self.slots[slot_index]
+        args = (slot["ids"], slot["Q"], slot["K"], slot["V"], slot["Qq"])
+        side = torch.cuda.Stream(device=self.dev)                 # a first run outside the capture: library
+        side.wait_stream(torch.cuda.current_stream(self.dev))     # load, kernel attributes, driver entry point
+        with torch.cuda.stream(side):
+            self.step_device(*args, slot=slot)
+        torch.cuda.current_stream(self.dev).wait_stream(side)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            res = self.step_device(*args, slot=slot)
+        return graph, res
 
     def host_buffers(self):
         """Pinned host buffers for the host-side entry points: inputs and outputs."""

@@ -57,3 +57,33 @@ def test_bench_block_sharded_mode_runs_and_reports(exchange):
     line = json.loads(out.stdout.strip().splitlines()[-1])
     assert line["scaling"] == "strong" and line["config"]["shard"] == "blocks" and line["device_status"] == 0
     assert line["value"] > 0 and line["gpu_launches"] > 0 and line["e2e"]["h2d_bytes_per_step"] > 0
+
+
+def test_step_captured_as_a_cuda_graph_replays_to_the_same_results():
+    w = W.CONFIGS["tiny"]
+    enc = ContextEncoder(w, DEV)
+    slot = enc.slots[0]
+    ids = W.needle_ids(w)
+    Q, K, V = W.qkv(w)
+    slot["ids"].copy_(torch.from_numpy(ids.view(np.int32)))
+    slot["Q"].copy_(Q); slot["K"].copy_(K); slot["V"].copy_(V); slot["Qq"].copy_(W.phase2_query(w))
+    eager = {k: v.clone() for k, v in enc.step_device(slot["ids"], slot["Q"], slot["K"], slot["V"], slot["Qq"]).items()
+             if k != "sel"}
+    graph, res = enc.capture_step()
+    for k in eager:
+        res[k].zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    for k in eager:
+        assert torch.equal(res[k], eager[k]), k
+    # new inputs in the same buffers, replayed: equals an eager run on them
+    Q2, K2, V2 = W.qkv(w, seed=77)
+    slot["Q"].copy_(Q2); slot["K"].copy_(K2); slot["V"].copy_(V2)
+    graph.replay()
+    torch.cuda.synchronize()
+    got = {k: res[k].clone() for k in eager}
+    again = enc.step_device(slot["ids"], slot["Q"], slot["K"], slot["V"], slot["Qq"])
+    torch.cuda.synchronize()
+    for k in eager:
+        assert torch.equal(got[k], again[k]), k
+    assert int(enc.status.item()) == 0
