@@ -99,3 +99,25 @@ def test_negative_position_and_bad_shapes():
     assert int(st.item()) & binding.DEV_BAD_POSITION and torch.equal(Y[1], X[1])     # counted as position 0
     with pytest.raises(binding.PulsarError):
         binding.pulsar_rope_apply(torch.randn((4, 2, 24), device=DEV).bfloat16(), pos, 10000.0)
+
+
+def test_rope_full_size_rows_sampled_against_the_oracle():
+    """131,072 rows of 32 + 8 heads in one launch (the shape the bench times), 1500 rows checked."""
+    rows = 131072
+    g = torch.Generator().manual_seed(4)
+    Q = torch.randn((rows, 32, 128), generator=g, dtype=torch.bfloat16)
+    K = torch.randn((rows, 8, 128), generator=g, dtype=torch.bfloat16)
+    pos = np.arange(rows, dtype=np.int32)                       # sparse mode of an unassembled sequence: global positions
+    st = binding.new_status(DEV)
+    Qo, Ko = binding.pulsar_rope_apply_qk(Q.to(DEV), K.to(DEV), torch.from_numpy(pos).to(DEV), status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    pick = np.unique(np.concatenate([np.arange(8), np.arange(rows - 8, rows),
+                                     np.random.default_rng(0).integers(0, rows, size=1500)]))
+    for X, Y in ((Q, Qo), (K, Ko)):
+        ref = oracle.rope_apply(X[pick], pos[pick], 500000.0)
+        x = X[pick].double().numpy()
+        mag = np.abs(x[..., :64]) + np.abs(x[..., 64:])
+        bound = 2.0 ** -8 * np.concatenate([mag, mag], axis=-1) + 1e-6
+        err = np.abs(Y[torch.from_numpy(pick).to(DEV)].double().cpu().numpy() - ref)
+        assert (err <= bound).all(), float((err / bound).max())
