@@ -196,3 +196,16 @@ def test_symmetric_memory_and_nccl_plumbing_at_world_size_one():
     out = subprocess.run([sys.executable, "-c", _SYMM_WORLD1], capture_output=True, text=True, timeout=600, env=env,
                          cwd=root)
     assert out.returncode == 0 and "SYMM-OK" in out.stdout, (out.stdout + out.stderr)[-3000:]
+
+
+def test_phase1_sharded_at_the_128k_configuration_equals_the_unsharded_call():
+    """Eight ranks with two blocks each (zigzag), run in turn: bit-identical to pulsar_phase1_attn, whose
+    output at this configuration is checked against the oracle in test_gpu_phase1.py."""
+    w = W.CONFIGS["128k"]
+    ids = W.token_ids(w)
+    Q, K, V = (t.to(DEV) for t in W.qkv(w))
+    O, LSE = sharded_phase1(w, 8, "zigzag", ids, Q, K, V)
+    sel = binding.pulsar_maxidf_select(to_dev_ids(ids, DEV), w.vocab_size, w.block_size, w.chunk, w.k, w.sink)
+    O1, LSE1, _, _ = binding.pulsar_phase1_attn(Q, K, V, w.block_size, sel["prefix_idx"], sel["prefix_len"])
+    torch.cuda.synchronize()
+    assert torch.equal(O, O1) and torch.equal(LSE, LSE1)
