@@ -376,7 +376,8 @@ int32_t pulsar_phase2_attn(const uint16_t *Qq, int32_t nq,
  *   Qnew        in  [n_new, Hq, d] bf16       Knew, Vnew  in [n_new, Hkv, d] bf16
  *   Kblocks, Vblocks in [B*block_size, Hkv, d] bf16 (retained context KV)
  *   Kgen, Vgen  in/out [gen_capacity, Hkv, d] bf16: rows [0, gen_len) hold the earlier query /
- *               generated tokens; rows [gen_len, gen_len + n_new) are written by this call
+ *               generated tokens; rows [gen_len, gen_len + n_new) are written by this call;
+ *               rows from gen_len + n_new on are never read (they may hold anything, NaN included)
  *   n_splits    parts of the context KV: 0 = library's choice, else as in pulsar_phase2_attn
  *   O           out [n_new, Hq, d] bf16       LSE out [n_new, Hq] float32 or NULL
  *

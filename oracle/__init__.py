@@ -95,10 +95,12 @@ def num_threads() -> int:
 def maxidf_select(token_ids, vocab_size, block_size, chunk, k, sink):
     """Max-IDF summary selection.  Returns a dict with ``sel_chunks`` [B,k],
     ``prefix_idx`` [sink+(B-1)*k*chunk], ``prefix_len`` [B], ``df`` [V] (uint32),
-    ``idf`` [V] and ``score`` [B, block_size/chunk] (float64)."""
+    ``idf`` [V] and ``score`` [B, C] (float64), B = ceil(L/block_size) blocks of
+    C = ceil(block_size/chunk) chunk slots.  Where a block has fewer than k chunks the
+    row of ``sel_chunks`` ends in -1; unused entries of ``prefix_idx`` are -1."""
     ids = np.ascontiguousarray(np.asarray(token_ids, dtype=np.uint32))
     L = ids.shape[0]
-    B, C = L // block_size, block_size // chunk
+    B, C = -(-L // block_size), -(-block_size // chunk)
     sel = np.zeros((B, k), np.int32)
     pidx = np.zeros(sink + max(B - 1, 0) * k * chunk, np.int32)
     plen = np.zeros(B, np.int32)

@@ -57,10 +57,23 @@ static double bf16_to_double(uint16_t h) {
  * score(chunk) = max over its tokens of IDF                (Eq. 2 / Eq. 9)
  * Sigma_b = the k best chunks of block b, in positional order (Alg. 1 l.6)
  * prefix  = [sink | Sigma_0 | ... | Sigma_{B-2}], block i uses its first
- *           prefix_len[i] = sink + i*k*chunk entries (0 for i = 0) (Eq. 4, 14)
+ *           prefix_len[i] entries: 0 for i = 0, else sink + the tokens of
+ *           Sigma_0 .. Sigma_{i-1}, which is sink + i*k*chunk when every selected
+ *           chunk is a whole one (Eq. 4, Eq. 14)
  *
- * Outputs (any may be NULL): sel_chunks [B*k], prefix_idx [sink+(B-1)*k*chunk],
- * prefix_len [B], df_out [vocab], idf_out [vocab], score_out [B*C].
+ * Lengths that do not divide (the paper cuts the tokenised context "into blocks
+ * of size" n_b and each block into chunks of m tokens, and says no more; the
+ * reading taken): the B = ceil(L / n_b) blocks are consecutive runs of n_b
+ * tokens, the last one holding the L - (B-1) n_b tokens that remain; a block of
+ * len tokens has ceil(len / m) chunks, the last one holding the tokens that
+ * remain and scored on those; a block with fewer than k chunks contributes all
+ * of them; the sink is the first min(sink, |B_0|) tokens.
+ *
+ * C = ceil(block_size / chunk) chunk slots per block.  Outputs (any may be NULL):
+ * sel_chunks [B*k] (a block's chosen chunks ascending, then -1 up to k),
+ * prefix_idx [sink+(B-1)*k*chunk] (entries past the last used one are -1),
+ * prefix_len [B], df_out [vocab], idf_out [vocab], score_out [B*C] (-inf for a
+ * slot without a chunk).
  * Returns 0, or -1 on a shape that the definition does not cover.
  */
 int oracle_maxidf_select(const uint32_t *token_ids, int64_t L, int32_t vocab_size,
@@ -68,9 +81,8 @@ int oracle_maxidf_select(const uint32_t *token_ids, int64_t L, int32_t vocab_siz
                          int32_t *sel_chunks, int32_t *prefix_idx, int32_t *prefix_len,
                          uint32_t *df_out, double *idf_out, double *score_out) {
     if (L <= 0 || block_size <= 0 || chunk <= 0 || vocab_size <= 0) return -1;
-    if (L % block_size != 0 || block_size % chunk != 0) return -1;
-    const int64_t B = L / block_size;
-    const int64_t C = block_size / chunk;
+    const int64_t B = (L + block_size - 1) / block_size;
+    const int64_t C = (block_size + chunk - 1) / chunk;
     if (k < 0 || k > C || sink < 0 || sink > block_size) return -1;
     for (int64_t p = 0; p < L; ++p)
         if (token_ids[p] >= (uint32_t)vocab_size) return -1;
@@ -84,23 +96,30 @@ int oracle_maxidf_select(const uint32_t *token_ids, int64_t L, int32_t vocab_siz
 
     /* document frequency: a block counts once however often the token occurs */
     for (int64_t t = 0; t < vocab_size; ++t) last_block[t] = -1;
-    for (int64_t b = 0; b < B; ++b)
-        for (int64_t p = b * block_size; p < (b + 1) * block_size; ++p) {
-            uint32_t t = token_ids[p];
-            if (last_block[t] != b) { last_block[t] = b; df[t] += 1; }
-        }
+    for (int64_t p = 0; p < L; ++p) {
+        const int64_t b = p / block_size;
+        uint32_t t = token_ids[p];
+        if (last_block[t] != b) { last_block[t] = b; df[t] += 1; }
+    }
     for (int64_t t = 0; t < vocab_size; ++t) {
         uint32_t f = df[t] > 1 ? df[t] : 1;
         idf[t] = log((double)B / (double)f);
     }
 
-    if (prefix_idx) for (int32_t j = 0; j < sink; ++j) prefix_idx[j] = j;
+    const int64_t cap = sink + (B - 1) * (int64_t)k * chunk;      /* room in prefix_idx */
+    const int64_t len0 = L < block_size ? L : block_size;
+    int64_t used = sink < len0 ? sink : len0;                     /* entries written so far */
+    if (prefix_idx) for (int64_t j = 0; j < used; ++j) prefix_idx[j] = (int32_t)j;
 
     for (int64_t b = 0; b < B; ++b) {
+        const int64_t lo = b * block_size;
+        const int64_t hi = lo + block_size < L ? lo + block_size : L;
+        const int64_t Cb = (hi - lo + chunk - 1) / chunk;         /* chunks this block has */
+        if (prefix_len) prefix_len[b] = b == 0 ? 0 : (int32_t)used;
         for (int64_t c = 0; c < C; ++c) {
             double s = -INFINITY;
-            for (int64_t p = 0; p < chunk; ++p) {
-                double v = idf[token_ids[b * block_size + c * chunk + p]];
+            for (int64_t p = lo + c * chunk; p < lo + (c + 1) * chunk && p < hi; ++p) {
+                double v = idf[token_ids[p]];
                 if (v > s) s = v;
             }
             score[c] = s;
@@ -109,25 +128,28 @@ int oracle_maxidf_select(const uint32_t *token_ids, int64_t L, int32_t vocab_siz
         /* top-k: take the best remaining chunk k times; a strict comparison
            scanning upward leaves equal scores to the lower index */
         memset(taken, 0, (size_t)C);
-        for (int32_t j = 0; j < k; ++j) {
+        for (int32_t j = 0; j < k && j < Cb; ++j) {
             int64_t best = -1;
-            for (int64_t c = 0; c < C; ++c)
+            for (int64_t c = 0; c < Cb; ++c)
                 if (!taken[c] && (best < 0 || score[c] > score[best])) best = c;
             if (best >= 0) taken[best] = 1;
         }
         /* positional order */
         int32_t j = 0;
-        for (int64_t c = 0; c < C; ++c) {
+        for (int64_t c = 0; c < Cb; ++c) {
             if (!taken[c]) continue;
             if (sel_chunks) sel_chunks[b * k + j] = (int32_t)c;
-            if (prefix_idx && b < B - 1)
-                for (int64_t p = 0; p < chunk; ++p)
-                    prefix_idx[sink + (b * k + j) * chunk + p] =
-                        (int32_t)(b * block_size + c * chunk + p);
+            if (b < B - 1)
+                for (int64_t p = lo + c * chunk; p < lo + (c + 1) * chunk && p < hi; ++p) {
+                    if (prefix_idx) prefix_idx[used] = (int32_t)p;
+                    ++used;
+                }
             ++j;
         }
-        if (prefix_len) prefix_len[b] = b == 0 ? 0 : (int32_t)(sink + b * k * chunk);
+        for (; j < k; ++j)
+            if (sel_chunks) sel_chunks[b * k + j] = -1;
     }
+    if (prefix_idx) for (int64_t j = used; j < cap; ++j) prefix_idx[j] = -1;
 
     if (df_out) memcpy(df_out, df, (size_t)vocab_size * sizeof(uint32_t));
     if (idf_out) memcpy(idf_out, idf, (size_t)vocab_size * sizeof(double));
@@ -186,8 +208,8 @@ int oracle_phase1_attn(const uint16_t *Q, const uint16_t *K, const uint16_t *V,
                        const int32_t *prefix_idx, const int32_t *prefix_len,
                        int32_t prefix_total, double scale,
                        const int64_t *rows, int64_t n_rows, double *O, double *LSE) {
-    if (L <= 0 || block_size <= 0 || L % block_size || Hkv <= 0 || Hq % Hkv || d <= 0) return -1;
-    const int64_t B = L / block_size;
+    if (L <= 0 || block_size <= 0 || Hkv <= 0 || Hq % Hkv || d <= 0) return -1;
+    const int64_t B = (L + block_size - 1) / block_size;      /* the last block may be shorter */
     for (int64_t i = 0; i < B; ++i) {
         if (prefix_len[i] < 0 || prefix_len[i] > prefix_total) return -1;
         for (int32_t j = 0; j < prefix_len[i]; ++j)

@@ -1426,8 +1426,11 @@ extern "C" int32_t pulsar_phase2_generate_step(const uint16_t* Qnew, const uint1
     if (!make_map_3d(&tmQ, Qnew, n_new, Hq, d, g, (quad ? 32 : kTileM) / g) ||
         !make_map_2d(&tmK, Kb, L, static_cast<int64_t>(Hkv) * d) ||
         !make_map_2d(&tmV, Vb, L, static_cast<int64_t>(Hkv) * d) ||
-        !make_map_2d(&tmKg, Kgen, gen_capacity, static_cast<int64_t>(Hkv) * d) ||
-        !make_map_2d(&tmVg, Vgen, gen_capacity, static_cast<int64_t>(Hkv) * d))
+        // The shard's maps end at its live rows: TMA zero-fills the rest of the last key tile, so
+        // whatever the unwritten rows [gen_len + n_new, gen_capacity) hold (NaN patterns of an
+        // uninitialised cache included) never reaches the PV product as 0 * NaN.
+        !make_map_2d(&tmKg, Kgen, static_cast<int64_t>(gen_len) + n_new, static_cast<int64_t>(Hkv) * d) ||
+        !make_map_2d(&tmVg, Vgen, static_cast<int64_t>(gen_len) + n_new, static_cast<int64_t>(Hkv) * d))
         return PULSAR_ERR_CUDA;
 
     // append KV(q) to the generation shard (Algorithm 1 line 15), then attend

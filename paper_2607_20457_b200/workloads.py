@@ -34,11 +34,11 @@ class Workload:
 
     @property
     def n_blocks(self) -> int:
-        return self.L // self.block_size
+        return -(-self.L // self.block_size)            # the last block may be shorter
 
     @property
     def chunks_per_block(self) -> int:
-        return self.block_size // self.chunk
+        return -(-self.block_size // self.chunk)        # the last chunk of a block may be shorter
 
     @property
     def sigma(self) -> int:
@@ -167,10 +167,11 @@ def sample_rows(w: Workload, per_block: int = 64, seed: int = 11) -> np.ndarray:
     rng = np.random.default_rng(seed)
     rows = []
     for b in range(w.n_blocks):
-        lo = b * w.block_size
-        fixed = list(range(lo, lo + 4)) + list(range(lo + w.block_size - 4, lo + w.block_size))
-        extra = rng.choice(np.arange(lo + 4, lo + w.block_size - 4),
-                           size=max(per_block - 8, 0), replace=False).tolist()
+        lo, hi = b * w.block_size, min((b + 1) * w.block_size, w.L)
+        fixed = list(range(lo, min(lo + 4, hi))) + list(range(max(hi - 4, lo), hi))
+        inner = np.arange(lo + 4, hi - 4)
+        extra = rng.choice(inner, size=min(max(per_block - 8, 0), len(inner)), replace=False).tolist() \
+            if len(inner) else []
         rows.extend(sorted(set(fixed + extra)))
     return np.asarray(rows, np.int64)
 

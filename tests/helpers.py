@@ -3,9 +3,10 @@ import numpy as np
 import torch
 
 # Tolerances stated by the benchmark spec: bf16 inputs, fp32 accumulation.
-# The 1e-2 bound on O is stated for N(0,1) inputs, whose outputs stay below 1 in magnitude.
-# Peaked test inputs produce outputs of magnitude up to ~4, where bf16 output rounding alone is
-# 2^-9 relative; there the bound scales with the largest reference magnitude.
+# The bound on O is element-wise: |dO| <= 1e-2 wherever |O_ref| <= 1 and 1e-2 * |O_ref| for the
+# larger elements (the output is rounded to bf16, whose half-ulp is 2^-9 relative: 0.0156 for an
+# element of magnitude 4, which an absolute 1e-2 could not admit).  No element borrows slack from
+# another: a small output next to a large one is still held to 1e-2.
 TOL_O_MAXABS = 1e-2
 TOL_LSE_ABS = 1e-3
 TOL_O_REL_L2 = 1e-2     # per (row set, head): guards against a kernel that ignores keys when |O| is tiny
@@ -29,6 +30,8 @@ def check_attention(O_gpu, LSE_gpu, O_ref, LSE_ref, what=""):
         msg += f" max|dLSE|={le:.3e}"
         assert le <= TOL_LSE_ABS, msg
     assert np.isfinite(o).all(), msg + " (non-finite output)"
-    assert max_abs <= TOL_O_MAXABS * max(1.0, float(np.abs(O_ref).max())), msg
+    bound = TOL_O_MAXABS * np.maximum(1.0, np.abs(O_ref))
+    worst = float((err / bound).max())
+    assert worst <= 1.0, msg + f" (worst element at {worst:.2f} of its bound)"
     assert rel <= TOL_O_REL_L2, msg
     return msg

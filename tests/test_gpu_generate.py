@@ -11,12 +11,12 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-def run_steps(w, steps, cap, q_scale=1.0, n_splits=0):
+def run_steps(w, steps, cap, q_scale=1.0, n_splits=0, shard_fill=0.0):
     _, K, V = W.qkv(w)
     Kd, Vd = K.to(DEV), V.to(DEV)
     gen = torch.Generator().manual_seed(21)
     Kgen_o = np.zeros((cap, w.Hkv, w.d), np.uint16); Vgen_o = np.zeros_like(Kgen_o)
-    Kgen_d = torch.zeros(cap, w.Hkv, w.d, dtype=torch.bfloat16, device=DEV); Vgen_d = torch.zeros_like(Kgen_d)
+    Kgen_d = torch.full((cap, w.Hkv, w.d), shard_fill, dtype=torch.bfloat16, device=DEV); Vgen_d = Kgen_d.clone()
     status = binding.new_status(DEV)
     gen_len = 0
     for n_new in steps:
@@ -45,6 +45,15 @@ def test_shard_longer_than_one_key_tile_and_peaked_logits():
     # 150 + 140 rows: the shard spans three key tiles, the new tokens two query tiles
     w = W.shrink(W.CONFIGS["tiny"], L=2048, block_size=512, Hq=8, Hkv=2, d=128)
     run_steps(w, [150, 140, 1], cap=320, q_scale=3.0, n_splits=4)
+
+
+def test_unwritten_shard_rows_may_hold_anything():
+    """The rows of the generation shard past the live ones belong to nobody yet (a cache taken from
+    an uninitialised allocation): filled with NaN they must not reach the result, neither while the
+    shard is shorter than one key tile nor when its last tile is partial."""
+    w = W.shrink(W.CONFIGS["tiny"], L=2048, block_size=512, Hq=8, Hkv=2, d=128)
+    run_steps(w, [5, 1, 130, 1], cap=512, shard_fill=float("nan"))
+    run_steps(W.CONFIGS["tiny"], [1, 1], cap=200, shard_fill=float("nan"))
 
 
 def test_16k_config_query_of_64_then_decode():

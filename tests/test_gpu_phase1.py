@@ -88,8 +88,11 @@ def test_poisoned_invisible_rows_do_not_leak():
 
 @pytest.mark.parametrize("name", ["16k", "32k", "64k", "128k"])
 def test_full_size_configs_on_sampled_rows(name):
+    """Each configuration with the prefix its own token ids select (the 32K ids carry injected rare
+    tokens; at 128K the selection leaves "the first k chunks" in some blocks)."""
     w = W.CONFIGS[name]
-    pidx, plen = W.first_k_prefix(w)
+    sel = oracle.maxidf_select(W.token_ids(w), w.vocab_size, w.block_size, w.chunk, w.k, w.sink)
+    pidx, plen = sel["prefix_idx"], sel["prefix_len"]
     Q, K, V = W.qkv(w)
     rows = W.sample_rows(w, per_block=16 if w.L > 40000 else 32)
     print(run_phase1(w, Q, K, V, pidx, plen, rows=rows, what=name))

@@ -11,14 +11,31 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-def run_phase2(w, Qq, K, V, n_splits=0, what="", scale=0.0):
+def run_phase2(w, Qq, K, V, n_splits=0, what="", scale=0.0, rows=None):
+    """The GPU always runs the whole query; ``rows`` limits the oracle (and the comparison) to some
+    query rows -- every query row is an independent softmax, so a subset is a query of its own."""
     status = binding.new_status(DEV)
     O, LSE = binding.pulsar_phase2_attn(Qq.to(DEV), K.to(DEV), V.to(DEV), w.n_blocks, w.block_size,
                                         softmax_scale=scale, n_splits=n_splits, status=status)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
+    if rows is not None:
+        idx = torch.as_tensor(np.asarray(rows))
+        Qq, O, LSE = Qq[idx].contiguous(), O[idx.to(DEV)], LSE[idx.to(DEV)]
     Oref, Lref = oracle.phase2_attn(Qq, K, V, w.n_blocks, w.block_size, scale=scale)
     return check_attention(O, LSE, Oref, Lref, what)
+
+
+def tile_edge_rows(nq, g, per_tile=2):
+    """Query tokens at the first and last row of row tiles (128 rows = 128/g tokens x g heads) and of
+    tile pairs, spread over the query, plus the last token."""
+    tok = 128 // g
+    tiles = -(-nq // tok)
+    pick = sorted(set([0, 1, tiles // 2, tiles - 2, tiles - 1]) & set(range(tiles)))
+    rows = []
+    for t in pick:
+        rows += [t * tok, min(nq, (t + 1) * tok) - 1]
+    return sorted(set(rows + [nq - 1]))
 
 
 @pytest.mark.parametrize("n_splits", [0, 1, 4, 32])
@@ -66,12 +83,29 @@ def test_per_block_partials_match_oracle_partials():
     check_attention(O, LSE, Oref, Lref, "merged")
 
 
-@pytest.mark.parametrize("name,nq", [("16k", None), ("128k", 64), ("128k", 1)])
+@pytest.mark.parametrize("name,nq", [("16k", None), ("32k", None), ("64k", None), ("128k", 64), ("128k", 1)])
 def test_full_size_kv(name, nq):
+    """Each configuration's own query (16K and 32K: 64 rows, 64K: 128 rows) and decode-sized
+    queries at 128K, library-chosen split, every query row checked."""
     w = W.CONFIGS[name]
     _, K, V = W.qkv(w)
     Qq = W.phase2_query(w, nq=nq)
     print(run_phase2(w, Qq, K, V, 0, what=f"{name} nq={Qq.shape[0]}"))
+
+
+@pytest.mark.parametrize("n_splits", [0, 9])
+def test_128k_config_own_query(n_splits):
+    """The 128K configuration's own Phase-2 call -- 8 queries x 64 tokens = 512 rows, i.e. 16 row
+    tiles (8 pairs) per KV head -- with the split the library picks (the launch the benchmark
+    times) and with 9 parts (1024 key tiles in runs of 114, the last one shorter).  The oracle runs
+    on the first and last tokens of several row tiles."""
+    w = W.CONFIGS["128k"]
+    assert w.nq == 512
+    J = n_splits or binding.phase2_choose_splits(w.nq, w.n_blocks, w.block_size, w.Hq, w.Hkv, w.d)
+    assert J > 1
+    _, K, V = W.qkv(w)
+    rows = tile_edge_rows(w.nq, w.Hq // w.Hkv)
+    print(run_phase2(w, W.phase2_query(w), K, V, n_splits, what=f"128k nq=512 J={J} rows={rows}", rows=rows))
 
 
 def test_merge_entry_point_against_oracle_merge():

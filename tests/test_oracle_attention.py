@@ -65,6 +65,33 @@ def test_phase1_equals_dense_attention_with_multiplicity_mask(q_scale):
     assert M.max() == 2
 
 
+def test_phase1_with_a_short_last_block_and_short_chunks():
+    """L = 230 in blocks of 64 (the last one holds 38 tokens) and chunks of 7 (the last chunk of a
+    block holds 1 token): the dense multiplicity-matrix attention again, and the short block with an
+    empty prefix equals library causal attention over its 38 rows."""
+    w = small_workload(L=230, chunk=7, k=3, sink=10)
+    assert w.n_blocks == 4 and w.L - 3 * w.block_size == 38
+    ids = np.random.default_rng(4).integers(0, 40, size=w.L).astype(np.uint32)
+    ids[63] = 41                                              # block 0's one-token chunk holds a unique id
+    sel = oracle.maxidf_select(ids, w.vocab_size, w.block_size, w.chunk, w.k, w.sink)
+    assert 9 in sel["sel_chunks"][0] and sel["prefix_len"][1] == w.sink + 2 * 7 + 1
+    Q, K, V = W.qkv(w, q_scale=2.0)
+    pidx, plen = sel["prefix_idx"], sel["prefix_len"]
+    O, LSE = oracle.phase1_attn(Q, K, V, w.block_size, pidx, plen)
+    Od, Ld, _ = dense_multiplicity_attention(Q, K, V, w, pidx, plen, 1.0 / np.sqrt(w.d))
+    np.testing.assert_allclose(O, Od, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(LSE, Ld, rtol=0, atol=1e-12)
+    # the short block alone
+    lo = 3 * w.block_size
+    Ob, _ = oracle.phase1_attn(Q, K, V, w.block_size, pidx, np.zeros(4, np.int32), rows=np.arange(lo, w.L))
+    g = w.Hq // w.Hkv
+    q = Q[lo:].to(torch.float64).permute(1, 0, 2)[None]
+    k = K[lo:].to(torch.float64).repeat_interleave(g, dim=1).permute(1, 0, 2)[None]
+    v = V[lo:].to(torch.float64).repeat_interleave(g, dim=1).permute(1, 0, 2)[None]
+    ref = torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True)[0]
+    np.testing.assert_allclose(Ob, ref.permute(1, 0, 2).numpy(), rtol=0, atol=1e-12)
+
+
 def test_block0_is_plain_causal_attention_library_routine():
     w = small_workload()
     Q, K, V = W.qkv(w)

@@ -138,9 +138,77 @@ def test_integer_and_float_ranking_agree():
 def test_rejects_shapes_outside_the_definition():
     ids = np.zeros(64, np.uint32)
     with pytest.raises(ValueError):
-        oracle.maxidf_select(ids, 8, 24, 4, 1, 0)       # L not a multiple of the block
-    with pytest.raises(ValueError):
         oracle.maxidf_select(ids, 8, 32, 4, 9, 0)       # k above chunks per block
+    with pytest.raises(ValueError):
+        oracle.maxidf_select(ids, 8, 32, 4, 2, 33)      # sink longer than a block
+    with pytest.raises(ValueError):
+        oracle.chunk_select(ids, 8, 24, 4, 1, 0, "bm25")   # the other scores keep whole blocks
+
+
+# ---- lengths that do not divide ---------------------------------------------------------------
+def ragged_reference(ids, nb, m, k, sink, V):
+    """The selection on a sequence whose length need not divide, by a route of its own: Python
+    slices cut the blocks and chunks (a slice simply ends where the data ends), df by set
+    membership, the k best chunks by sorting on (-score, index)."""
+    L = len(ids)
+    blocks = [ids[s: s + nb].tolist() for s in range(0, L, nb)]
+    B = len(blocks)
+    df = {t: sum(1 for blk in blocks if t in blk) for t in set(ids.tolist())}
+    sel, prefix, plen = [], list(range(min(sink, len(blocks[0])))), []
+    for b, blk in enumerate(blocks):
+        plen.append(0 if b == 0 else len(prefix))
+        chunks = [blk[s: s + m] for s in range(0, len(blk), m)]
+        score = [max(math.log(B / max(df[t], 1)) for t in ch) for ch in chunks]
+        best = sorted(sorted(range(len(chunks)), key=lambda c: (-score[c], c))[:k])
+        sel.append(best + [-1] * (k - len(best)))
+        if b < B - 1:
+            for c in best:
+                prefix += list(range(b * nb + c * m, b * nb + c * m + len(chunks[c])))
+    cap = sink + (B - 1) * k * m
+    return np.asarray(sel), np.asarray(prefix + [-1] * (cap - len(prefix))), np.asarray(plen)
+
+
+@pytest.mark.parametrize("L,nb,m,k,sink", [
+    (50, 16, 5, 2, 3),      # short last block (2 tokens) and a one-token last chunk in every block
+    (61, 20, 4, 3, 6),      # chunks divide the block, the last block holds 1 token: fewer chunks than k
+    (64, 16, 4, 2, 4),      # everything divides: the reading changes nothing
+    (47, 12, 5, 3, 12),     # sink = the whole first block; last block 11 tokens
+    (9, 16, 4, 2, 12),      # one block shorter than the block size and than the sink
+    (100, 33, 7, 5, 0),     # five chunks per block, all taken; no sink
+])
+@pytest.mark.parametrize("seed", range(3))
+def test_lengths_that_do_not_divide(L, nb, m, k, sink, seed):
+    V = 14
+    ids = np.random.default_rng(100 + seed).integers(0, V, size=L).astype(np.uint32)
+    r = oracle.maxidf_select(ids, V, nb, m, k, sink)
+    sel, prefix, plen = ragged_reference(ids, nb, m, k, sink, V)
+    np.testing.assert_array_equal(r["sel_chunks"], sel)
+    np.testing.assert_array_equal(r["prefix_idx"], prefix)
+    np.testing.assert_array_equal(r["prefix_len"], plen)
+
+
+def test_a_short_last_chunk_can_win_and_shortens_the_prefix():
+    # blocks of 10 tokens in chunks of 4: the third chunk of a block has 2 tokens.  Block 0's short
+    # chunk holds the only token that is unique to the block, so it is selected (Appendix C.5) and
+    # contributes its 2 tokens: block 1's prefix is sink + 4 + 2, not sink + 2*4 (Eq. 14 with whole chunks).
+    ids = np.zeros(30, np.uint32)
+    ids[9] = 7
+    r = oracle.maxidf_select(ids, 8, 10, 4, 2, 1)
+    assert r["sel_chunks"].tolist() == [[0, 2], [0, 1], [0, 1]]
+    assert r["prefix_len"].tolist() == [0, 1 + 4 + 2, 1 + 6 + 8]
+    assert r["prefix_idx"].tolist() == [0, 0, 1, 2, 3, 8, 9, 10, 11, 12, 13, 14, 15, 16, 17, -1, -1]
+    assert r["df"][7] == 1 and r["df"][0] == 3
+    assert r["score"][0, 2] == math.log(3.0) and r["score"][0, 0] == 0.0
+
+
+def test_short_last_block_counts_as_a_block():
+    # N is the number of blocks, the short one included: 3 blocks of 8, 8 and 2 tokens
+    ids = np.asarray([1] * 8 + [1] * 8 + [1, 2], np.uint32)
+    r = oracle.maxidf_select(ids, 4, 8, 4, 1, 0)
+    assert r["df"].tolist() == [0, 3, 1, 0]
+    assert r["idf"][2] == math.log(3.0) and r["idf"][1] == 0.0
+    assert r["sel_chunks"].tolist() == [[0], [0], [0]]
+    assert r["score"][2].tolist() == [math.log(3.0), -math.inf]
 
 
 # ---- the other scoring heuristics of Appendix C -------------------------------------------------
