@@ -82,25 +82,34 @@ int32_t pulsar_wait_selftest(int32_t *device_status, uint64_t limit_ns, int32_t 
 /* ------------------------------------------------------------------------------------------
  * Max-IDF summary selection (Section 3.1; Algorithm 1 lines 3 and 6; Appendix C.1, C.5).
  *
- * The L context tokens form B = L / block_size logical blocks.  df(t) = number of blocks in
- * which token t occurs; IDF(t) = ln(B / max(df(t),1)) (Eq. 3); each block is cut into
- * C = block_size / chunk chunks scored by the largest IDF among their tokens (Eq. 2); the k
- * best chunks of a block, equal scores going to the lower chunk index, listed in positional
+ * The L context tokens form B = ceil(L / block_size) logical blocks.  df(t) = number of blocks
+ * in which token t occurs; IDF(t) = ln(B / max(df(t),1)) (Eq. 3); each block is cut into
+ * C = ceil(block_size / chunk) chunks scored by the largest IDF among their tokens (Eq. 2); the
+ * k best chunks of a block, equal scores going to the lower chunk index, listed in positional
  * order, are its summary Sigma_b.  The prefix list is [0..sink-1 | Sigma_0 | ... | Sigma_{B-2}]
  * as global token positions; block i attends to its first prefix_len[i] entries, with
  * prefix_len[0] = 0 and prefix_len[i] = sink + i*k*chunk (Eq. 4, Eq. 14).  Ranking is done on
  * the integer df (IDF is strictly decreasing in df), so the result is exact.
  *
+ * Lengths that do not divide (the paper cuts the context "into blocks" and the blocks into
+ * chunks of `chunk` tokens and is silent on remainders; this is the reading taken): the last
+ * block holds the L - (B-1)*block_size tokens that remain; the last chunk of a block holds the
+ * tokens that remain and is scored on those; a block with fewer than k chunks contributes all
+ * of them; the sink is the first min(sink, L) tokens.  A summary that includes a short chunk
+ * has fewer than k*chunk tokens, so in general prefix_len[i] = sink + the tokens of
+ * Sigma_0 .. Sigma_{i-1}; that is Eq. 14's sink + i*k*chunk whenever chunk divides block_size.
+ *
  *   token_ids   in  [L] uint32, each < vocab_size
- *   sel_chunks  out [B*k] int32: chunk indices within the block, ascending, for every block
- *   prefix_idx  out [sink + (B-1)*k*chunk] int32
+ *   sel_chunks  out [B*k] int32: a block's chunk indices, ascending, then -1 up to k entries
+ *   prefix_idx  out [sink + (B-1)*k*chunk] int32; entries past prefix_len[B-1] (and past the
+ *               sink when B = 1) are -1
  *   prefix_len  out [B] int32
  *   df_out      out [vocab_size] uint32, or NULL
  *   idf_out     out [vocab_size] float32 (natural log), or NULL
  *
- * Requirements (else PULSAR_ERR_SHAPE): L % block_size == 0, block_size % chunk == 0,
- * 0 <= k <= C, 0 <= sink <= block_size, B <= 65535, vocab_size <= 1,800,000 (one block's
- * presence bitmap must fit in shared memory), C <= 32768.
+ * Requirements (else PULSAR_ERR_SHAPE): 0 <= k <= C, 0 <= sink <= block_size, B <= 65533,
+ * L < 2^31, vocab_size <= 1,800,000 (one block's presence bitmap must fit in shared memory),
+ * C <= 32768.
  * ------------------------------------------------------------------------------------------ */
 size_t pulsar_maxidf_select_workspace_bytes(int64_t L, int32_t vocab_size, int32_t block_size,
                                             int32_t chunk, int32_t k, int32_t sink);
@@ -191,6 +200,7 @@ int32_t pulsar_maxidf_select_noalloc(const uint32_t *token_ids, int64_t L, int32
 /* ------------------------------------------------------------------------------------------
  * Phase-1 prefix-block attention (Eq. 1 over the assembled input of Eq. 4; Alg. 1 l.7-8).
  *
+ * The L rows form B = ceil(L / block_size) blocks; the last one holds the rows that remain.
  * For block i, row r (global position p = i*block_size + r) and query head h, the keys are
  * rows prefix_idx[0 .. prefix_len[i]) followed by rows i*block_size .. p of K (KV head
  * h / (Hq/Hkv)); the prefix is fully visible, the block causal; a row listed twice counts
@@ -202,12 +212,13 @@ int32_t pulsar_maxidf_select_noalloc(const uint32_t *token_ids, int64_t L, int32
  * prefix_len = {0, block_size, block_size, ...}.
  *
  *   Q           in  [L, Hq, d] bf16         K, V   in [L, Hkv, d] bf16
- *   prefix_idx  in  [prefix_total] int32    prefix_len in [B] int32, B = L / block_size
+ *   prefix_idx  in  [prefix_total] int32    prefix_len in [B] int32
+ *               (entries of prefix_idx that no block's prefix_len reaches are not read)
  *   softmax_scale   <= 0 selects 1/sqrt(d)
  *   O           out [L, Hq, d] bf16         LSE    out [L, Hq] float32 (natural log) or NULL
- *   K_ret,V_ret out [L, Hkv, d] bf16 (= [B, block_size, Hkv, d]) or NULL
+ *   K_ret,V_ret out [L, Hkv, d] bf16 (block i = rows [i*block_size, ...)) or NULL
  *
- * Requirements (else PULSAR_ERR_SHAPE): d in {64, 128}; Hq % Hkv == 0; L % block_size == 0;
+ * Requirements (else PULSAR_ERR_SHAPE): d in {64, 128}; Hq % Hkv == 0; B <= 65535;
  * prefix_total >= 0; L < 2^31.  Arithmetic: bf16 operands, fp32 accumulation on the tensor
  * cores, probabilities rounded to bf16 before the PV product, bf16 output.
  * ------------------------------------------------------------------------------------------ */
@@ -330,7 +341,10 @@ int32_t pulsar_retain_block_kv(const uint16_t *K, const uint16_t *V, int64_t tot
  * O = sum_j e^{l_j - l} A_j, which equals one softmax over the concatenated keys.
  *
  *   Qq          in  [nq, Hq, d] bf16 (a batch of queries is flattened into nq rows)
- *   Kblocks, Vblocks in [B, block_size, Hkv, d] bf16 (the retained rows, i.e. [L, Hkv, d])
+ *   Kblocks, Vblocks in [B, block_size, Hkv, d] bf16 (the retained rows, i.e. [L, Hkv, d]).
+ *               Only the product L = B*block_size matters here (the parts below are the
+ *               library's, not the blocks'): the retained KV of a sequence whose last block is
+ *               short is passed as B = 1, block_size = L.
  *   n_splits    number of KV parts: 0 = let the library choose, otherwise >= 1.  If n_splits
  *               divides the B*block_size keys, every part has that many keys (n_splits == B
  *               gives the per-block (A_h, l_h) of Algorithm 1 line 12); if not, the parts are

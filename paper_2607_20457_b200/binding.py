@@ -174,12 +174,13 @@ def pulsar_maxidf_select(token_ids: torch.Tensor, vocab_size: int, block_size: i
                          sink: int, want_df: bool = False, want_idf: bool = False, workspace=None,
                          status=None, out=None):
     """Max-IDF summary selection.  ``token_ids``: CUDA int32 [L] holding the uint32 ids.
-    Returns a dict of CUDA tensors: sel_chunks [B,k], prefix_idx, prefix_len [B] (+ df, idf)."""
+    Returns a dict of CUDA tensors: sel_chunks [B,k], prefix_idx, prefix_len [B] (+ df, idf),
+    B = ceil(L / block_size)."""
     lib = load_library()
     _need(token_ids, torch.int32, "token_ids")
     L = token_ids.numel()
     dev = token_ids.device
-    B = L // block_size if block_size > 0 else 0
+    B = -(-L // block_size) if block_size > 0 else 0          # the last block may be shorter
     if out is not None:                  # (sel_buf, prefix_idx, prefix_len) preallocated by the caller
         sel_buf, pidx, plen = out
     else:

@@ -58,7 +58,9 @@ struct AttnArgs {
     int quad;              // phase 2, at most 32 query rows per KV head: the rows are replicated into the four
                            // lane quarters of the tile and each softmax warp takes one quarter of the keys
     int Hkv;
-    int pairs;             // phase 1: query-tile pairs per block; phase 2: query-tile pairs per KV head
+    int pairs;             // phase 1: query-tile pairs per full block; phase 2: query-tile pairs per KV head
+    int last_len;          // phase 1: tokens of the last block (block_size unless the sequence ends inside it)
+    int pairs_last;        // phase 1: query-tile pairs of the last block
     int n_items;           // work items in total
     int n_blocks;          // phase 1
     int32_t* counter;      // phase 1: work counter (zeroed before the launch); null = fixed round order
@@ -81,17 +83,21 @@ gather_prefix_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V, c
     const int j = blockIdx.x;
     __shared__ int s_src;
     if (threadIdx.x == 0) {
-        int64_t limit = L;
+        int64_t limit = -1;                 // stays -1 when no block uses entry j (the list may be shorter than its buffer)
         for (int i = 0; i < n_blocks; ++i)
             if (prefix_len[i] > j) { limit = static_cast<int64_t>(i) * block_size; break; }
-        int src = prefix_idx[j];
-        if (src < 0 || src >= limit) {
-            report(status, PULSAR_DEV_BAD_PREFIX);
-            src = 0;
+        int src = -1;
+        if (limit >= 0) {
+            src = prefix_idx[j];
+            if (src < 0 || src >= limit) {
+                report(status, PULSAR_DEV_BAD_PREFIX);
+                src = 0;
+            }
         }
         s_src = src;
     }
     __syncthreads();
+    if (s_src < 0) return;
     const size_t src = static_cast<size_t>(s_src) * row_vecs, dst = static_cast<size_t>(j) * row_vecs;
     for (int v = threadIdx.x; v < row_vecs; v += blockDim.x) {
         Kp[dst + v] = K[src + v];
@@ -301,14 +307,24 @@ __device__ __forceinline__ void decode_item(const AttnArgs& a, const VarlenTable
         // from the last tile pair (most causal tiles) down; the heads of one (block, pair) are
         // adjacent.  CTAs that run at the same time therefore read the same K/V rows (L2 hits),
         // and the costliest items are handed out first.
+        // The last block may be shorter than the others: it then has fewer tile pairs.
         const int rank = idx / a.Hq;
-        const int combo = (a.n_blocks - 1 - rank / a.pairs) * a.pairs + (a.pairs - 1 - rank % a.pairs);
-        it.head0 = idx - (idx / a.Hq) * a.Hq;
+        it.head0 = idx - rank * a.Hq;
         it.kvh = it.head0 / a.g;
         it.part = 0;
-        const int blk = combo / a.pairs, pair = combo - blk * a.pairs;
+        int blk, pair, len;
+        if (rank < a.pairs_last) {
+            blk = a.n_blocks - 1;
+            pair = a.pairs_last - 1 - rank;
+            len = a.last_len;
+        } else {
+            const int r2 = rank - a.pairs_last;
+            blk = a.n_blocks - 2 - r2 / a.pairs;
+            pair = a.pairs - 1 - r2 % a.pairs;
+            len = a.block_size;
+        }
         const int qt0 = 2 * pair;
-        it.has1 = (qt0 + 1 < a.tiles_per_block) ? 1 : 0;
+        it.has1 = (qt0 + 1 < (len + kTileM - 1) / kTileM) ? 1 : 0;
         it.row0_a = qt0 * kTileM;
         it.row0_b = (qt0 + 1) * kTileM;
         it.token0_a = blk * a.block_size + it.row0_a;
@@ -319,7 +335,7 @@ __device__ __forceinline__ void decode_item(const AttnArgs& a, const VarlenTable
         it.pref_len = pl;
         it.n_pref_tiles = (pl + kTileN - 1) / kTileN;
         it.main_row0 = blk * a.block_size;
-        it.main_len = a.block_size;
+        it.main_len = len;
         it.gen_base = -1;
         it.n_tiles_a = it.n_pref_tiles + qt0 + 1;
         it.n_tiles_b = it.has1 ? it.n_pref_tiles + qt0 + 2 : 0;
@@ -1021,22 +1037,31 @@ int32_t launch_attn(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMa
 
 struct Phase1Plan {
     int n_blocks, tiles_per_block, pairs_per_block;
+    int last_len, pairs_last;                 // the last block: its tokens and its tile pairs
+    int n_items;
     size_t pref_rows, pref_bytes, total;
 };
 
+// whole_only: the entry point takes only sequences made of whole blocks.
 int32_t plan_phase1(int64_t L, int32_t Hq, int32_t Hkv, int32_t d, int32_t block_size, int32_t prefix_total,
-                    Phase1Plan& p) {
+                    Phase1Plan& p, bool whole_only = false) {
     if (L <= 0 || Hq <= 0 || Hkv <= 0 || block_size <= 0 || prefix_total < 0) return PULSAR_ERR_INVALID_ARG;
-    if ((d != 64 && d != 128) || Hq % Hkv != 0 || L % block_size != 0 || L >= (1ll << 31)) return PULSAR_ERR_SHAPE;
-    if (L / block_size > 65535 || Hq > 65535) return PULSAR_ERR_SHAPE;
+    if ((d != 64 && d != 128) || Hq % Hkv != 0 || L >= (1ll << 31)) return PULSAR_ERR_SHAPE;
+    if (whole_only && L % block_size != 0) return PULSAR_ERR_SHAPE;
+    const int64_t B = (L + block_size - 1) / block_size;       // the last block holds the tokens that remain
+    if (B > 65535 || Hq > 65535) return PULSAR_ERR_SHAPE;
     if (prefix_total > (1 << 30)) return PULSAR_ERR_SHAPE;
-    p.n_blocks = static_cast<int>(L / block_size);
+    p.n_blocks = static_cast<int>(B);
     p.tiles_per_block = (block_size + kTileM - 1) / kTileM;
     p.pref_rows = static_cast<size_t>(prefix_total > 0 ? prefix_total : 1);
     p.pairs_per_block = (p.tiles_per_block + 1) / 2;
+    p.last_len = static_cast<int>(L - (B - 1) * block_size);
+    p.pairs_last = ((p.last_len + kTileM - 1) / kTileM + 1) / 2;
     p.pref_bytes = round_up(p.pref_rows * Hkv * d * 2, 256);
     p.total = 2 * p.pref_bytes + 256;                        // gathered prefix K, V and the work counter
-    if (static_cast<int64_t>(p.n_blocks) * p.pairs_per_block * Hq >= (1ll << 31)) return PULSAR_ERR_SHAPE;
+    const int64_t items = ((B - 1) * p.pairs_per_block + p.pairs_last) * Hq;
+    if (items >= (1ll << 31)) return PULSAR_ERR_SHAPE;
+    p.n_items = static_cast<int>(items);
     return PULSAR_OK;
 }
 
@@ -1142,7 +1167,9 @@ extern "C" int32_t pulsar_phase1_attn(const uint16_t* Q, const uint16_t* K, cons
     a.mode = kModePhase1;
     a.Hkv = Hkv;
     a.pairs = p.pairs_per_block;
-    a.n_items = p.n_blocks * p.pairs_per_block * Hq;
+    a.last_len = p.last_len;
+    a.pairs_last = p.pairs_last;
+    a.n_items = p.n_items;
     a.n_blocks = p.n_blocks;
     a.counter = counter;
     a.n_tokens = static_cast<int>(L);
@@ -1227,7 +1254,7 @@ extern "C" int32_t pulsar_phase1_attn_sharded(const uint16_t* Q, const uint16_t*
                                               float softmax_scale, uint16_t* O, float* LSE, void* workspace,
                                               size_t workspace_bytes, int32_t* device_status, void* stream_) {
     Phase1Plan p;
-    int32_t rc = plan_phase1(L_local, Hq, Hkv, d, block_size, prefix_total, p);
+    int32_t rc = plan_phase1(L_local, Hq, Hkv, d, block_size, prefix_total, p, /*whole_only=*/true);
     if (rc != PULSAR_OK) return rc;
     if (!Q || !K || !V || !O || !prefix_len_local || !workspace || (prefix_total > 0 && (!K_prefix || !V_prefix)))
         return PULSAR_ERR_INVALID_ARG;
@@ -1257,7 +1284,9 @@ extern "C" int32_t pulsar_phase1_attn_sharded(const uint16_t* Q, const uint16_t*
     a.mode = kModePhase1;
     a.Hkv = Hkv;
     a.pairs = p.pairs_per_block;
-    a.n_items = p.n_blocks * p.pairs_per_block * Hq;
+    a.last_len = p.last_len;
+    a.pairs_last = p.pairs_last;
+    a.n_items = p.n_items;
     a.n_blocks = p.n_blocks;
     a.counter = counter;
     a.n_tokens = static_cast<int>(L_local);

@@ -29,14 +29,15 @@ constexpr int kTopkThreads = 256;
 constexpr size_t kMaxDynSmem = 227 * 1024;
 
 __global__ void __launch_bounds__(kPresenceThreads)
-presence_kernel(const uint32_t* __restrict__ ids, int block_size, int vocab_size, int words,
+presence_kernel(const uint32_t* __restrict__ ids, int64_t L, int block_size, int vocab_size, int words,
                 uint32_t* __restrict__ bitmaps, int32_t* status) {
     extern __shared__ uint32_t bits[];
     const int b = blockIdx.x;
     for (int w = threadIdx.x; w < words; w += blockDim.x) bits[w] = 0u;
     __syncthreads();
     const uint32_t* blk = ids + static_cast<size_t>(b) * block_size;
-    for (int i = threadIdx.x; i < block_size; i += blockDim.x) {
+    const int len = static_cast<int>(min(static_cast<int64_t>(block_size), L - static_cast<int64_t>(b) * block_size));
+    for (int i = threadIdx.x; i < len; i += blockDim.x) {
         const uint32_t t = blk[i];
         if (t < static_cast<uint32_t>(vocab_size)) atomicOr(&bits[t >> 5], 1u << (t & 31));
         else report(status, PULSAR_DEV_BAD_TOKEN);
@@ -82,56 +83,123 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int& 
     return base + incl - v;
 }
 
-// level[b*C + c] = min over the chunk's tokens of df (ids outside the vocabulary rank last).
+// level[b*C + c] = min over the chunk's tokens of df.  Slot c of block b covers the tokens
+// [b*block_size + c*chunk, +chunk) that lie inside the block and the sequence: the last chunk of
+// a block may be shorter, and a slot past the end of a short last block holds no chunk at all.
+// Ranks: a chunk whose ids all lie outside the vocabulary gets `worst` (after every real df), a
+// slot without a chunk worst + 1 (never selected).
 __global__ void __launch_bounds__(256)
-chunk_level_kernel(const uint32_t* __restrict__ ids, const uint16_t* __restrict__ df_table, int n_chunks_total,
-                   int chunk, int vocab_size, int worst, uint16_t* __restrict__ level) {
+chunk_level_kernel(const uint32_t* __restrict__ ids, const uint16_t* __restrict__ df_table, int64_t L,
+                   int block_size, int chunks_per_block, int n_slots_total, int chunk, int vocab_size, int worst,
+                   uint16_t* __restrict__ level) {
     const int lane = threadIdx.x & 31;
-    const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (c >= n_chunks_total) return;
-    const uint32_t* tok = ids + static_cast<size_t>(c) * chunk;
-    int mn = worst;
-    for (int p = lane; p < chunk; p += 32) {
-        const uint32_t t = tok[p];
+    const int slot = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (slot >= n_slots_total) return;
+    const int b = slot / chunks_per_block, c = slot - b * chunks_per_block;
+    const int64_t lo = static_cast<int64_t>(b) * block_size;
+    const int64_t block_end = min(lo + block_size, L);
+    const int64_t start = lo + static_cast<int64_t>(c) * chunk;
+    const int len = static_cast<int>(max(static_cast<int64_t>(0), min(static_cast<int64_t>(chunk), block_end - start)));
+    int mn = len > 0 ? worst : worst + 1;
+    for (int p = lane; p < len; p += 32) {
+        const uint32_t t = ids[start + p];
         if (t < static_cast<uint32_t>(vocab_size)) mn = min(mn, static_cast<int>(df_table[t]));
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, o));
-    if (lane == 0) level[c] = static_cast<uint16_t>(mn);
+    if (lane == 0) level[slot] = static_cast<uint16_t>(mn);
 }
 
-// Block b's part of the prefix list (Eq. 4): its k chosen chunks (ascending, in shared memory)
-// as global token positions, the sink entries (written by block 0) and prefix_len[b].
-__device__ __forceinline__ void write_block_prefix(int b, int n_blocks, int block_size, int chunk, int k, int sink,
-                                                   const int* chosen, int32_t* __restrict__ prefix_idx,
+// Where a block's part of the prefix list goes and how long it is when lengths do not divide.
+struct PrefixGeometry {
+    int k_b;          // chunks this block contributes: min(k, chunks it has)
+    int sink_eff;     // min(sink, tokens of block 0)
+    int tail;         // tokens of the last chunk slot of a full block (= chunk when chunk divides block_size)
+    int cap;          // entries of prefix_idx: sink + (n_blocks - 1) * k * chunk
+};
+
+__device__ __forceinline__ PrefixGeometry prefix_geometry(int b, int n_blocks, int64_t L, int block_size, int chunk,
+                                                          int k, int sink) {
+    PrefixGeometry g;
+    const int64_t lo = static_cast<int64_t>(b) * block_size;
+    const int len_b = static_cast<int>(min(static_cast<int64_t>(block_size), L - lo));
+    const int chunks_b = (len_b + chunk - 1) / chunk;
+    g.k_b = min(k, chunks_b);
+    g.sink_eff = static_cast<int>(min(static_cast<int64_t>(sink), min(static_cast<int64_t>(block_size), L)));
+    const int C = (block_size + chunk - 1) / chunk;
+    g.tail = block_size - (C - 1) * chunk;
+    g.cap = sink + (n_blocks - 1) * k * chunk;
+    return g;
+}
+
+// Block b's part of the prefix list (Eq. 4): its chosen chunks (ascending, in shared memory) as
+// global token positions starting at entry `offset`, the sink entries (written by block 0), the
+// unused entries at the end (-1, written by the last block) and prefix_len[b] = offset (0 for
+// block 0).  Only the last chosen chunk can be a short one (the last slot of the block), so the
+// block's entries are the leading ones of k_b * chunk: those whose position lies inside the block.
+__device__ __forceinline__ void write_block_prefix(int b, int n_blocks, int block_size, int chunk, int k,
+                                                   const PrefixGeometry& g, int offset, const int* chosen,
+                                                   int32_t* __restrict__ sel_chunks, int32_t* __restrict__ prefix_idx,
                                                    int32_t* __restrict__ prefix_len) {
-    const int sigma = k * chunk;
+    for (int j = g.k_b + threadIdx.x; j < k; j += blockDim.x) sel_chunks[static_cast<size_t>(b) * k + j] = -1;
     if (b < n_blocks - 1) {
-        int32_t* dst = prefix_idx + sink + static_cast<size_t>(b) * sigma;
-        for (int i = threadIdx.x; i < sigma; i += blockDim.x) {
+        int32_t* dst = prefix_idx + offset;
+        const int n = g.k_b * chunk;
+        for (int i = threadIdx.x; i < n; i += blockDim.x) {
             const int j = i / chunk, p = i - j * chunk;
-            dst[i] = b * block_size + chosen[j] * chunk + p;
+            const int pos = chosen[j] * chunk + p;
+            if (pos < block_size) dst[i] = b * block_size + pos;
         }
+    } else {
+        for (int i = offset + threadIdx.x; i < g.cap; i += blockDim.x) prefix_idx[i] = -1;
     }
     if (b == 0)
-        for (int i = threadIdx.x; i < sink; i += blockDim.x) prefix_idx[i] = i;
-    if (threadIdx.x == 0) prefix_len[b] = b == 0 ? 0 : sink + b * sigma;
+        for (int i = threadIdx.x; i < g.sink_eff; i += blockDim.x) prefix_idx[i] = i;
+    if (threadIdx.x == 0) prefix_len[b] = b == 0 ? 0 : offset;
+}
+
+// Entry of prefix_idx at which block b's summary starts: the sink plus the tokens of the
+// summaries of blocks 0..b-1.  Those blocks are full ones; each contributes k chunks of `chunk`
+// tokens, except that a block which selected its last chunk slot contributes only that slot's
+// `tail` tokens for it.  The last slot (index C-1) is selected iff fewer than k of the other slots
+// rank at or before it, i.e. have a level <= its own (they all have a lower index).  Only needed
+// when chunk does not divide block_size; one warp per earlier block.
+__device__ __forceinline__ int prefix_offset(int b, const uint16_t* __restrict__ level_all, int C, int chunk, int k,
+                                             const PrefixGeometry& g, int* s_short) {
+    if (g.tail == chunk || k == 0 || b == 0) return g.sink_eff + b * k * chunk;
+    if (threadIdx.x == 0) *s_short = 0;
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    for (int j = warp; j < b; j += n_warps) {
+        const uint16_t* lv = level_all + static_cast<size_t>(j) * C;
+        const int last = lv[C - 1];
+        int before = 0;
+        for (int c = lane; c < C - 1; c += 32) before += (lv[c] <= last) ? 1 : 0;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
+        if (lane == 0 && before < k) atomicAdd(s_short, 1);
+    }
+    __syncthreads();
+    return g.sink_eff + b * k * chunk - *s_short * (chunk - g.tail);
 }
 
 __global__ void __launch_bounds__(kTopkThreads)
-topk_kernel(const uint16_t* __restrict__ level_all, int n_blocks, int block_size, int chunk, int k, int sink,
-            int32_t* __restrict__ sel_chunks, int32_t* __restrict__ prefix_idx, int32_t* __restrict__ prefix_len) {
+topk_kernel(const uint16_t* __restrict__ level_all, int n_blocks, int64_t L, int block_size, int chunk, int k_all,
+            int sink, int32_t* __restrict__ sel_chunks, int32_t* __restrict__ prefix_idx,
+            int32_t* __restrict__ prefix_len) {
     extern __shared__ int smem[];
-    const int C = block_size / chunk;
+    const int C = (block_size + chunk - 1) / chunk;
     int* level = smem;                       // [C]   min df of the chunk
-    int* hist = level + C;                   // [n_blocks + 2]
-    int* chosen = hist + n_blocks + 2;       // [k]   selected chunk ids, ascending
+    int* hist = level + C;                   // [n_blocks + 3]
+    int* chosen = hist + n_blocks + 3;       // [k]   selected chunk ids, ascending
     __shared__ int warp_sums[kTopkThreads / 32];
-    __shared__ int s_threshold, s_need;
+    __shared__ int s_threshold, s_need, s_short;
 
     const int b = blockIdx.x;
+    const PrefixGeometry geo = prefix_geometry(b, n_blocks, L, block_size, chunk, k_all, sink);
+    const int k = geo.k_b;                   // a short last block may have fewer than k_all chunks
 
-    for (int i = threadIdx.x; i < n_blocks + 2; i += blockDim.x) hist[i] = 0;
+    for (int i = threadIdx.x; i < n_blocks + 3; i += blockDim.x) hist[i] = 0;
     __syncthreads();
     for (int c = threadIdx.x; c < C; c += blockDim.x) {
         const int lv = level_all[static_cast<size_t>(b) * C + c];
@@ -157,7 +225,7 @@ topk_kernel(const uint16_t* __restrict__ level_all, int n_blocks, int block_size
     int at_T_before = 0, taken_before = 0;
     for (int c0 = 0; c0 < C; c0 += kTopkThreads) {
         const int c = c0 + threadIdx.x;
-        const int lv = c < C ? level[c] : n_blocks + 2;
+        const int lv = c < C ? level[c] : n_blocks + 3;
         const int is_T = (lv == T) ? 1 : 0;
         int tot_T;
         const int rank_T = at_T_before + block_exclusive_scan(is_T, warp_sums, tot_T);
@@ -166,14 +234,15 @@ topk_kernel(const uint16_t* __restrict__ level_all, int n_blocks, int block_size
         const int pos = taken_before + block_exclusive_scan(take, warp_sums, tot_take);
         if (take && pos < k) {
             chosen[pos] = c;
-            sel_chunks[static_cast<size_t>(b) * k + pos] = c;
+            sel_chunks[static_cast<size_t>(b) * k_all + pos] = c;
         }
         at_T_before += tot_T;
         taken_before += tot_take;
     }
     __syncthreads();
 
-    write_block_prefix(b, n_blocks, block_size, chunk, k, sink, chosen, prefix_idx, prefix_len);
+    const int offset = prefix_offset(b, level_all, C, chunk, k_all, geo, &s_short);
+    write_block_prefix(b, n_blocks, block_size, chunk, k_all, geo, offset, chosen, sel_chunks, prefix_idx, prefix_len);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -270,7 +339,11 @@ topk_score_kernel(const double* __restrict__ score_all, int n_blocks, int block_
         taken_before += tot;
     }
     __syncthreads();
-    write_block_prefix(b, n_blocks, block_size, chunk, k, sink, chosen, prefix_idx, prefix_len);
+    // this entry point takes whole blocks and chunks only: every summary has k * chunk tokens
+    const PrefixGeometry geo = prefix_geometry(b, n_blocks, static_cast<int64_t>(n_blocks) * block_size, block_size,
+                                               chunk, k, sink);
+    write_block_prefix(b, n_blocks, block_size, chunk, k, geo, sink + b * k * chunk, chosen, sel_chunks, prefix_idx,
+                       prefix_len);
 }
 
 struct SelectPlan {
@@ -279,18 +352,21 @@ struct SelectPlan {
     size_t presence_smem, topk_smem;
 };
 
+// whole_only: the entry point takes only lengths that divide (L by block_size, block_size by chunk).
 int32_t plan_select(int64_t L, int32_t vocab_size, int32_t block_size, int32_t chunk, int32_t k, int32_t sink,
-                    SelectPlan& p) {
+                    SelectPlan& p, bool whole_only = false) {
     if (L <= 0 || vocab_size <= 0 || block_size <= 0 || chunk <= 0 || k < 0 || sink < 0) return PULSAR_ERR_INVALID_ARG;
-    if (L % block_size != 0 || block_size % chunk != 0) return PULSAR_ERR_SHAPE;
+    if (whole_only && (L % block_size != 0 || block_size % chunk != 0)) return PULSAR_ERR_SHAPE;
     if (L >= (1ll << 31)) return PULSAR_ERR_SHAPE;
-    const int64_t B = L / block_size;
-    p.C = block_size / chunk;
-    if (B > 65535 || k > p.C || sink > block_size || p.C > 32768) return PULSAR_ERR_SHAPE;
+    const int64_t B = (L + block_size - 1) / block_size;
+    p.C = (block_size + chunk - 1) / chunk;
+    // chunk levels are 16-bit: the real df values 0..B and the two ranks after them, B + 1 and B + 2
+    if (B > 65533 || k > p.C || sink > block_size || p.C > 32768) return PULSAR_ERR_SHAPE;
+    if (sink + (B - 1) * static_cast<int64_t>(k) * chunk >= (1ll << 31)) return PULSAR_ERR_SHAPE;
     p.n_blocks = static_cast<int>(B);
     p.words = (vocab_size + 31) / 32;
     p.presence_smem = static_cast<size_t>(p.words) * 4;
-    p.topk_smem = (static_cast<size_t>(p.C) + p.n_blocks + 2 + k) * 4;
+    p.topk_smem = (static_cast<size_t>(p.C) + p.n_blocks + 3 + k) * 4;
     if (p.presence_smem > kMaxDynSmem || p.topk_smem > kMaxDynSmem) return PULSAR_ERR_SHAPE;
     p.bitmap_bytes = round_up(static_cast<size_t>(p.n_blocks) * p.words * 4, 256);
     p.df_bytes = round_up(static_cast<size_t>(vocab_size) * 2, 256);
@@ -340,7 +416,7 @@ extern "C" int32_t pulsar_maxidf_select(const uint32_t* token_ids, int64_t L, in
                                             static_cast<int>(p.topk_smem)));
 
     presence_kernel<<<p.n_blocks, kPresenceThreads, p.presence_smem, stream>>>(
-        token_ids, block_size, vocab_size, p.words, bitmaps, device_status);
+        token_ids, L, block_size, vocab_size, p.words, bitmaps, device_status);
     PULSAR_CUDA_OK(cudaGetLastError());
     count_launch();
     df_idf_kernel<<<(vocab_size + 255) / 256, 256, 0, stream>>>(bitmaps, p.n_blocks, p.words, vocab_size, df_table,
@@ -348,11 +424,12 @@ extern "C" int32_t pulsar_maxidf_select(const uint32_t* token_ids, int64_t L, in
     PULSAR_CUDA_OK(cudaGetLastError());
     count_launch();
     const int n_chunks_total = p.n_blocks * p.C;
-    chunk_level_kernel<<<(n_chunks_total + 7) / 8, 256, 0, stream>>>(token_ids, df_table, n_chunks_total, chunk,
-                                                                     vocab_size, p.n_blocks + 1, level);
+    chunk_level_kernel<<<(n_chunks_total + 7) / 8, 256, 0, stream>>>(token_ids, df_table, L, block_size, p.C,
+                                                                     n_chunks_total, chunk, vocab_size,
+                                                                     p.n_blocks + 1, level);
     PULSAR_CUDA_OK(cudaGetLastError());
     count_launch();
-    topk_kernel<<<p.n_blocks, kTopkThreads, p.topk_smem, stream>>>(level, p.n_blocks, block_size, chunk, k, sink,
+    topk_kernel<<<p.n_blocks, kTopkThreads, p.topk_smem, stream>>>(level, p.n_blocks, L, block_size, chunk, k, sink,
                                                                    sel_chunks, prefix_idx, prefix_len);
     PULSAR_CUDA_OK(cudaGetLastError());
     count_launch();
@@ -370,7 +447,7 @@ struct ScorePlan {
 int32_t plan_score(int64_t L, int32_t vocab_size, int32_t block_size, int32_t chunk, int32_t k, int32_t sink,
                    int32_t mode, ScorePlan& p) {
     if (mode < PULSAR_SCORE_MAX_IDF || mode > PULSAR_SCORE_TYPE_TOKEN) return PULSAR_ERR_INVALID_ARG;
-    int32_t rc = plan_select(L, vocab_size, block_size, chunk, k, sink, p.base);
+    int32_t rc = plan_select(L, vocab_size, block_size, chunk, k, sink, p.base, /*whole_only=*/true);
     if (rc != PULSAR_OK) return rc;
     if (p.base.n_blocks > kMaxScoreBlocks || chunk > kMaxScoreChunk || p.base.C > kMaxScoreChunksPerBlock)
         return PULSAR_ERR_SHAPE;
@@ -428,7 +505,7 @@ extern "C" int32_t pulsar_chunk_select(const uint32_t* token_ids, int64_t L, int
     if (b.presence_smem > 48 * 1024)
         PULSAR_CUDA_OK(cudaFuncSetAttribute(presence_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             static_cast<int>(b.presence_smem)));
-    presence_kernel<<<b.n_blocks, kPresenceThreads, b.presence_smem, stream>>>(token_ids, block_size, vocab_size,
+    presence_kernel<<<b.n_blocks, kPresenceThreads, b.presence_smem, stream>>>(token_ids, L, block_size, vocab_size,
                                                                                b.words, bitmaps, device_status);
     PULSAR_CUDA_OK(cudaGetLastError());
     count_launch();

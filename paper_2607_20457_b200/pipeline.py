@@ -31,9 +31,11 @@ class ContextEncoder:
             binding.maxidf_select_workspace_bytes(w.L, w.vocab_size, w.block_size, w.chunk, w.k, w.sink), dev)
         self.ws_p1 = binding._workspace(
             binding.phase1_workspace_bytes(w.L, w.Hq, w.Hkv, w.d, w.block_size, w.prefix_total), dev)
-        self.n_splits = phase2_splits or binding.phase2_choose_splits(w.nq, B, w.block_size, w.Hq, w.Hkv, w.d)
+        # Phase 2 only needs the number of retained rows: a sequence that ends inside a block is one run of L rows
+        self.kv_shape = (B, w.block_size) if w.L % w.block_size == 0 else (1, w.L)
+        self.n_splits = phase2_splits or binding.phase2_choose_splits(w.nq, *self.kv_shape, w.Hq, w.Hkv, w.d)
         self.ws_p2 = binding._workspace(
-            binding.phase2_workspace_bytes(w.nq, B, w.block_size, w.Hq, w.Hkv, w.d, self.n_splits), dev)
+            binding.phase2_workspace_bytes(w.nq, *self.kv_shape, w.Hq, w.Hkv, w.d, self.n_splits), dev)
         self.slots = [self._new_slot() for _ in range(slots)]
 
     def _new_slot(self):
@@ -71,7 +73,7 @@ class ContextEncoder:
             workspace=self.ws_p1, status=self.status)
         if record:
             record[2].record()
-        O2, LSE2 = binding.pulsar_phase2_attn(Qq, K_ret, V_ret, w.n_blocks, w.block_size, n_splits=self.n_splits,
+        O2, LSE2 = binding.pulsar_phase2_attn(Qq, K_ret, V_ret, *self.kv_shape, n_splits=self.n_splits,
                                               out=slot["O2"], lse_out=slot["LSE2"], workspace=self.ws_p2,
                                               status=self.status)
         if record:

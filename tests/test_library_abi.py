@@ -45,17 +45,21 @@ def test_workspace_sizes(lib):
     # phase 2: fp32 partials for the chosen number of parts
     assert binding.phase2_workspace_bytes(512, 16, 8192, 32, 8, 128, 4) == 4 * 512 * 32 * 129 * 4
     assert binding.phase2_workspace_bytes(512, 16, 8192, 32, 8, 128, 1) == 256
+    # a sequence that ends inside a block: ceil(100/64) = 2 blocks of ceil(64/8) = 8 chunk slots
+    assert binding.maxidf_select_workspace_bytes(100, 128, 64, 8, 1, 0) == 3 * 256
     # shapes the kernels do not cover give 0
-    assert binding.maxidf_select_workspace_bytes(100, 128, 64, 8, 1, 0) == 0
+    assert binding.maxidf_select_workspace_bytes(128, 128, 64, 8, 9, 0) == 0
+    assert lib.pulsar_chunk_select_workspace_bytes(100, 128, 64, 8, 1, 0, 2) == 0     # other scores: whole blocks only
     assert binding.phase1_workspace_bytes(4096, 4, 1, 96, 1024, 0) == 0
 
 
 def test_host_validation_launches_nothing(lib):
     null = None
     one = ctypes.c_void_p(256)          # never dereferenced: validation fails first
-    # selection: L not a multiple of the block, k above chunks per block
-    assert lib.pulsar_maxidf_select(one, 100, 128, 64, 8, 1, 0, one, one, one, null, null, one, 1 << 20, null, null) == 2
+    # selection: k above chunks per block, sink above the block, more blocks than the 16-bit levels cover
     assert lib.pulsar_maxidf_select(one, 128, 128, 64, 8, 9, 0, one, one, one, null, null, one, 1 << 20, null, null) == 2
+    assert lib.pulsar_maxidf_select(one, 128, 128, 64, 8, 1, 65, one, one, one, null, null, one, 1 << 20, null, null) == 2
+    assert lib.pulsar_maxidf_select(one, 65534, 128, 1, 1, 1, 0, one, one, one, null, null, one, 1 << 30, null, null) == 2
     # NULL data pointer, misaligned pointer, workspace too small
     assert lib.pulsar_maxidf_select(null, 128, 128, 64, 8, 1, 0, one, one, one, null, null, one, 1 << 20, null, null) == 1
     assert lib.pulsar_maxidf_select(ctypes.c_void_p(260), 128, 128, 64, 8, 1, 0, one, one, one, null, null, one, 1 << 20, null, null) == 3
