@@ -23,8 +23,10 @@
 
 namespace pulsar {
 
+// after_attention: the merge follows the attention launch that wrote the partials and may be
+// scheduled while that launch drains (it waits for it before it reads).
 int32_t launch_lse_merge(const float* part_O, const float* part_LSE, int32_t n_parts, int64_t rows, int32_t d,
-                         uint16_t* O, float* LSE, cudaStream_t stream);
+                         uint16_t* O, float* LSE, cudaStream_t stream, bool after_attention = false);
 
 namespace {
 
@@ -55,6 +57,8 @@ struct AttnArgs {
     int n_ctx_parts;       // phase 2: parts of the context KV; part n_ctx_parts (if any) is the generation shard
     int gen_len;           // phase 2: rows of the generation shard that precede the new tokens
     int gen_total;         // phase 2: gen_len + new tokens (0 = no generation shard)
+    int loader_waits;      // the launch before this one wrote rows the loader reads (the appended shard rows) and this
+                           // launch was allowed to start beside it: the loader waits for it first
     int quad;              // phase 2, at most 32 query rows per KV head: the rows are replicated into the four
                            // lane quarters of the tile and each softmax warp takes one quarter of the keys
     int Hkv;
@@ -105,10 +109,13 @@ gather_prefix_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V, c
     }
 }
 
-// KV(q) of the new tokens appended to the generation shard: one launch for both tensors.
+// KV(q) of the new tokens appended to the generation shard: one launch for both tensors.  The
+// attention launch that follows may start beside it; its loader waits for this grid before it
+// reads the shard.
 __global__ void __launch_bounds__(256)
 append_kv_kernel(const uint4* __restrict__ Knew, const uint4* __restrict__ Vnew, uint4* __restrict__ Kdst,
                  uint4* __restrict__ Vdst, int vecs) {
+    grid_launch_dependents();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < vecs) {
         Kdst[i] = Knew[i];
@@ -418,7 +425,9 @@ __device__ __forceinline__ float exp_row128(const uint32_t (&r)[kTileN], float s
     return (acc0.x + acc0.y) + (acc1.x + acc1.y);
 }
 
-template <int D>
+// kQuad: the decode-shaped instance (AttnArgs::quad); a separate instantiation keeps its code out
+// of the Phase-1 kernel's register allocation.
+template <int D, bool kQuad>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
             const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmKp,
@@ -434,6 +443,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SL::kAbort);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // The launch that follows (the merge of this launch's partials, if any) may be scheduled as
+    // SMs become free; it waits for this grid to finish before it reads anything.
+    grid_launch_dependents();
 
     if (tid == 0) {
         *abort_flag = 0;
@@ -491,6 +503,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             uint32_t q_use0 = 0, q_use1 = 0;
             bool ok = true;
             volatile int* item_q = reinterpret_cast<volatile int*>(smem + SL::kItemQ);
+            if (a.loader_waits) grid_dependency_wait();
             for (uint32_t seq = 0; ok; ++seq) {
                 // Reconverge once per iteration: every barrier is waited on at most once per
                 // iteration, so a lane that is still polling can never be more than one phase behind
@@ -527,7 +540,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 ++q_use0;
                 if (!ok) break;
                 if (leader) mbar_expect_tx_a(bar0 + 8 * (SL::bQFull + 0), SL::kTileBytes);
-                if (a.quad) {
+                if (kQuad) {
                     // the same 32 rows four times, at rows 0, 32, 64, 96 of the tile (the box of the
                     // tensor map is 32 rows here; 32 rows of a panel are 4096 bytes)
 #pragma unroll
@@ -744,7 +757,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             if (n == 0) continue;
             float m_used = -INFINITY, l_run = 0.f;
             const int my_row_in_block = (s ? it.row0_b : it.row0_a) + row;
-            const int row_t = a.quad ? lane : row;             // row as far as token and head are concerned
+            const int row_t = kQuad ? lane : row;             // row as far as token and head are concerned
 
             for (int t = 0; t < n; ++t) {
                 // visible key columns of this tile for this row: [0, n_vis)
@@ -773,7 +786,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 if (!ok) break;
                 tc_fence_after();
 
-                if (a.quad) {
+                if (kQuad) {
                     // Few query rows (decode): this warp's lane quarter holds a copy of the rows and
                     // the warp takes keys [32q, 32q+32) of the tile only; the other keys get P = 0 in
                     // its copy.  Each copy ends as a partial of its own, merged with the KV parts.
@@ -920,7 +933,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             {
                 const int token = (s ? it.token0_b : it.token0_a) + row_t / a.pack;
                 const int head = it.head0 + row_t % a.pack;
-                const int part = a.quad ? it.part * 4 + (warp & 3) : it.part;
+                const int part = kQuad ? it.part * 4 + (warp & 3) : it.part;
                 bool store = token < a.n_tokens;
                 if (a.mode != kModePhase2) store = store && my_row_in_block < it.main_len;
                 const float inv_l = l_run > 0.f ? 1.f / l_run : 0.f;
@@ -1018,18 +1031,33 @@ bool make_map_2d(CUtensorMap* m, const void* base, int64_t rows, int64_t width) 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// overlap_prior: launch with programmatic stream serialization, i.e. the kernel may start while the
+// launch before it on the stream is still running (that launch must be this library's append
+// kernel, which releases its dependent at once); the loader then waits for it before its first
+// load (AttnArgs::loader_waits).
 template <int D>
 int32_t launch_attn(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& v, const CUtensorMap& kp,
                     const CUtensorMap& vp, const AttnArgs& a, cudaStream_t stream,
-                    const VarlenTable* table = nullptr) {
+                    const VarlenTable* table = nullptr, bool overlap_prior = false) {
     constexpr int smem = SmemLayout<D>::kDynBytes;
     // The opt-in to more than 48 KB of dynamic shared memory is a per-device function attribute;
     // setting it on every launch keeps multi-device processes correct and costs well under a microsecond.
-    PULSAR_CUDA_OK(cudaFuncSetAttribute(attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    auto kernel = a.quad ? attn_kernel<D, true> : attn_kernel<D, false>;
+    PULSAR_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     const int grid = a.n_items < sm_count() ? a.n_items : sm_count();     // one persistent CTA per SM
     if (grid <= 0) return PULSAR_OK;
     static const VarlenTable kNoTable{};
-    attn_kernel<D><<<grid, kAttnThreads, smem, stream>>>(q, k, v, kp, vp, a, table ? *table : kNoTable);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.blockDim = dim3(kAttnThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap_prior ? 1 : 0;
+    PULSAR_CUDA_OK(cudaLaunchKernelEx(&cfg, kernel, q, k, v, kp, vp, a, table ? *table : kNoTable));
     PULSAR_CUDA_OK(cudaGetLastError());
     count_launch();
     return PULSAR_OK;
@@ -1405,7 +1433,7 @@ extern "C" int32_t pulsar_phase2_attn(const uint16_t* Qq, int32_t nq, const uint
                   : launch_attn<64>(tmQ, tmK, tmV, tmK, tmV, a, stream);
     if (rc != PULSAR_OK) return rc;
     if (partial_out)
-        return launch_lse_merge(pO, pL, n_splits * copies, static_cast<int64_t>(nq) * Hq, d, O, LSE, stream);
+        return launch_lse_merge(pO, pL, n_splits * copies, static_cast<int64_t>(nq) * Hq, d, O, LSE, stream, true);
     return PULSAR_OK;
 }
 
@@ -1498,10 +1526,11 @@ extern "C" int32_t pulsar_phase2_generate_step(const uint16_t* Qnew, const uint1
     a.Hkv = Hkv;
     a.pairs = (row_tiles + 1) / 2;
     a.n_items = a.pairs * Hkv * n_parts;
-    rc = d == 128 ? launch_attn<128>(tmQ, tmK, tmV, tmKg, tmVg, a, stream)
-                  : launch_attn<64>(tmQ, tmK, tmV, tmKg, tmVg, a, stream);
+    a.loader_waits = 1;                                // the shard rows are written by the append launch
+    rc = d == 128 ? launch_attn<128>(tmQ, tmK, tmV, tmKg, tmVg, a, stream, nullptr, true)
+                  : launch_attn<64>(tmQ, tmK, tmV, tmKg, tmVg, a, stream, nullptr, true);
     if (rc != PULSAR_OK) return rc;
-    return launch_lse_merge(pO, pL, n_parts * copies, static_cast<int64_t>(n_new) * Hq, d, O, LSE, stream);
+    return launch_lse_merge(pO, pL, n_parts * copies, static_cast<int64_t>(n_new) * Hq, d, O, LSE, stream, true);
 }
 
 // =============================================================================================

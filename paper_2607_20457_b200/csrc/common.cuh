@@ -54,6 +54,15 @@ __device__ __forceinline__ bool elect_one() {
     return pred != 0;
 }
 
+// ---- programmatic dependent launch ----------------------------------------------------------
+// In a kernel launched with the programmatic-stream-serialization attribute: wait until the
+// kernel launched before it has finished and its writes are visible.  Without the attribute
+// (an ordinary launch) the instruction returns at once.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// In the kernel launched first: allow the dependent kernel to start (its own waits still hold it
+// back where it needs this kernel's results).
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- mbarrier ---------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));

@@ -13,6 +13,7 @@ __global__ void __launch_bounds__(256)
 lse_merge_kernel(const float* __restrict__ part_O, const float* __restrict__ part_LSE, int n_parts,
                  int64_t stride_O, int64_t stride_L, int64_t rows, int d, void* __restrict__ O_,
                  float* __restrict__ LSE) {
+    grid_dependency_wait();        // launched beside the attention kernel that writes the partials: wait for it
     const int vec_per_row = d >> 2;
     const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (idx >= rows * vec_per_row) return;
@@ -50,48 +51,77 @@ lse_merge_kernel(const float* __restrict__ part_O, const float* __restrict__ par
 }
 
 // The same merge for few output rows and many parts (decode shapes), where one thread per output
-// vector would run a long chain of load latencies on a handful of CTAs: kMergeLanes consecutive
-// lanes share an output vector, lane i takes parts i, i + kMergeLanes, ...; the maximum and the
-// sums are combined by butterfly shuffles (a fixed order, so the result is reproducible).
-constexpr int kMergeLanes = 8;
+// vector would run a long chain of load latencies on a handful of CTAs: kLanes consecutive lanes
+// share an output vector, lane i takes parts i, i + kLanes, ...; the maximum and the sums are
+// combined by butterfly shuffles (a fixed order, so the result is reproducible).  A lane issues
+// the loads of all its parts -- the l_j and the output vectors, which do not depend on them --
+// before it uses any (up to kMaxInFlight parts at a time), so the kernel lasts about one memory
+// round trip however many parts there are.
+constexpr int kMergeLanes = 8;          // moderate part counts
+constexpr int kMergeLanesWide = 32;     // decode shapes: 4 partials per KV part, dozens of parts
 // Outputs (rows x d/4) up to which the lane form is used.  Measured: 72 parts into 32 or 256 rows 3.5 us
 // faster than one thread per output; 16 parts into 2048 rows 2.6 us and 64 parts into 1024 rows 6 us slower.
 constexpr int64_t kMergeLanesMaxThreads = 8192;
+// ... and up to which a whole warp shares an output vector.  Measured at 72 parts: 32 rows (1024 outputs)
+// 3 us faster than with 8 lanes, 256 rows (8192 outputs) no faster.
+constexpr int64_t kMergeWideMaxThreads = 1024;
 
-template <bool kF32>
+template <bool kF32, int kLanes>
 __global__ void __launch_bounds__(256)
 lse_merge_lanes_kernel(const float* __restrict__ part_O, const float* __restrict__ part_LSE, int n_parts,
                        int64_t stride_O, int64_t stride_L, int64_t rows, int d, void* __restrict__ O_,
                        float* __restrict__ LSE) {
+    grid_dependency_wait();        // launched beside the attention kernel that writes the partials: wait for it
+    constexpr int kMaxInFlight = 4;
     const int vec_per_row = d >> 2;
     const int64_t tid = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-    const int sub = static_cast<int>(tid % kMergeLanes);
-    const int64_t idx = tid / kMergeLanes;
+    const int sub = static_cast<int>(tid % kLanes);
+    const int64_t idx = tid / kLanes;
     const bool valid = idx < rows * vec_per_row;
     const int64_t row = valid ? idx / vec_per_row : 0;
     const int v = valid ? static_cast<int>(idx - row * vec_per_row) : 0;
 
-    float m = -INFINITY;
-    if (valid) {
-#pragma unroll 4
-        for (int j = sub; j < n_parts; j += kMergeLanes) m = fmaxf(m, part_LSE[static_cast<size_t>(j) * stride_L + row]);
-    }
-#pragma unroll
-    for (int o = 1; o < kMergeLanes; o <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-
+    // running maximum, weight sum and weighted sum over this lane's parts (ascending part order)
+    float m = -INFINITY, denom = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    float denom = 0.f;
-    if (valid && m > -INFINITY) {
-#pragma unroll 4
-        for (int j = sub; j < n_parts; j += kMergeLanes) {
-            const float w = __expf(part_LSE[static_cast<size_t>(j) * stride_L + row] - m);
-            const float4 o = *reinterpret_cast<const float4*>(part_O + static_cast<size_t>(j) * stride_O + row * d + v * 4);
-            denom += w;
-            acc.x += w * o.x; acc.y += w * o.y; acc.z += w * o.z; acc.w += w * o.w;
+    if (valid) {
+        for (int j0 = sub; j0 < n_parts; j0 += kLanes * kMaxInFlight) {
+            float l[kMaxInFlight];
+            float4 o[kMaxInFlight];
+#pragma unroll
+            for (int b = 0; b < kMaxInFlight; ++b) {
+                const int j = j0 + b * kLanes;
+                const int jc = j < n_parts ? j : j0;                 // a slot past the end repeats a load and weighs nothing
+                l[b] = part_LSE[static_cast<size_t>(jc) * stride_L + row];
+                o[b] = *reinterpret_cast<const float4*>(part_O + static_cast<size_t>(jc) * stride_O + row * d + v * 4);
+                if (j >= n_parts) l[b] = -INFINITY;
+            }
+            float m_new = m;
+#pragma unroll
+            for (int b = 0; b < kMaxInFlight; ++b) m_new = fmaxf(m_new, l[b]);
+            if (m_new > -INFINITY) {
+                const float keep = (m == -INFINITY) ? 0.f : __expf(m - m_new);
+                denom *= keep;
+                acc.x *= keep; acc.y *= keep; acc.z *= keep; acc.w *= keep;
+#pragma unroll
+                for (int b = 0; b < kMaxInFlight; ++b) {
+                    const float w = (l[b] == -INFINITY) ? 0.f : __expf(l[b] - m_new);
+                    denom += w;
+                    acc.x += w * o[b].x; acc.y += w * o[b].y; acc.z += w * o[b].z; acc.w += w * o[b].w;
+                }
+                m = m_new;
+            }
         }
     }
+    // bring the lanes to the common maximum, then add them up
+    float m_all = m;
 #pragma unroll
-    for (int o = 1; o < kMergeLanes; o <<= 1) {
+    for (int o = 1; o < kLanes; o <<= 1) m_all = fmaxf(m_all, __shfl_xor_sync(0xffffffffu, m_all, o));
+    const float mine = (m == -INFINITY) ? 0.f : __expf(m - m_all);
+    denom *= mine;
+    acc.x *= mine; acc.y *= mine; acc.z *= mine; acc.w *= mine;
+#pragma unroll
+    for (int o = 1; o < kLanes; o <<= 1) {
         denom += __shfl_xor_sync(0xffffffffu, denom, o);
         acc.x += __shfl_xor_sync(0xffffffffu, acc.x, o);
         acc.y += __shfl_xor_sync(0xffffffffu, acc.y, o);
@@ -99,7 +129,7 @@ lse_merge_lanes_kernel(const float* __restrict__ part_O, const float* __restrict
         acc.w += __shfl_xor_sync(0xffffffffu, acc.w, o);
     }
     if (!valid || sub != 0) return;
-    if (m > -INFINITY) {
+    if (m_all > -INFINITY) {
         const float inv = 1.f / denom;
         acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
     }
@@ -111,7 +141,7 @@ lse_merge_lanes_kernel(const float* __restrict__ part_O, const float* __restrict
         packed.y = pack_bf16x2(acc.z, acc.w);
         *reinterpret_cast<uint2*>(static_cast<uint16_t*>(O_) + row * d + v * 4) = packed;
     }
-    if (LSE != nullptr && v == 0) LSE[row] = (m > -INFINITY) ? m + logf(denom) : -INFINITY;
+    if (LSE != nullptr && v == 0) LSE[row] = (m_all > -INFINITY) ? m_all + logf(denom) : -INFINITY;
 }
 
 // The merge with every part at its own address: part j is the buffer parts[j], laid out
@@ -165,40 +195,56 @@ lse_merge_table_kernel(const __grid_constant__ PartTable parts, int n_parts, int
 }
 
 namespace {
+// Launch with or without programmatic stream serialization (see launch_lse_merge).
+template <typename Kernel, typename... Args>
+cudaError_t launch_maybe_dependent(Kernel kernel, unsigned blocks, cudaStream_t stream, bool dependent, Args... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(blocks);
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 int32_t launch_merge(const float* part_O, const float* part_LSE, int32_t n_parts, int64_t stride_O, int64_t stride_L,
-                     int64_t rows, int32_t d, void* O, bool f32, float* LSE, cudaStream_t stream) {
+                     int64_t rows, int32_t d, void* O, bool f32, float* LSE, cudaStream_t stream,
+                     bool dependent = false) {
     if (rows == 0) return PULSAR_OK;
     const int64_t threads = rows * (d >> 2);
     if (n_parts >= 2 * kMergeLanes && threads <= kMergeLanesMaxThreads) {
         // few outputs, many parts: spread the parts of an output over lanes
-        const unsigned blocks = static_cast<unsigned>((threads * kMergeLanes + 255) / 256);
-        if (f32)
-            lse_merge_lanes_kernel<true><<<blocks, 256, 0, stream>>>(part_O, part_LSE, n_parts, stride_O, stride_L, rows,
-                                                                     d, O, LSE);
-        else
-            lse_merge_lanes_kernel<false><<<blocks, 256, 0, stream>>>(part_O, part_LSE, n_parts, stride_O, stride_L, rows,
-                                                                      d, O, LSE);
+        const bool wide = n_parts >= 2 * kMergeLanesWide && threads <= kMergeWideMaxThreads;
+        const int lanes = wide ? kMergeLanesWide : kMergeLanes;
+        const unsigned blocks = static_cast<unsigned>((threads * lanes + 255) / 256);
+        auto kernel = wide ? (f32 ? lse_merge_lanes_kernel<true, kMergeLanesWide> : lse_merge_lanes_kernel<false, kMergeLanesWide>)
+                           : (f32 ? lse_merge_lanes_kernel<true, kMergeLanes> : lse_merge_lanes_kernel<false, kMergeLanes>);
+        PULSAR_CUDA_OK(launch_maybe_dependent(kernel, blocks, stream, dependent, part_O, part_LSE, static_cast<int>(n_parts),
+                                              stride_O, stride_L, rows, static_cast<int>(d), O, LSE));
         PULSAR_CUDA_OK(cudaGetLastError());
         count_launch();
         return PULSAR_OK;
     }
     const int64_t blocks = (threads + 255) / 256;
     if (blocks > 0x7fffffffll) return PULSAR_ERR_SHAPE;
-    if (f32)
-        lse_merge_kernel<true><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(part_O, part_LSE, n_parts, stride_O,
-                                                                                 stride_L, rows, d, O, LSE);
-    else
-        lse_merge_kernel<false><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(part_O, part_LSE, n_parts, stride_O,
-                                                                                  stride_L, rows, d, O, LSE);
+    auto kernel = f32 ? lse_merge_kernel<true> : lse_merge_kernel<false>;
+    PULSAR_CUDA_OK(launch_maybe_dependent(kernel, static_cast<unsigned>(blocks), stream, dependent, part_O, part_LSE,
+                                          static_cast<int>(n_parts), stride_O, stride_L, rows, static_cast<int>(d), O, LSE));
     PULSAR_CUDA_OK(cudaGetLastError());
     count_launch();
     return PULSAR_OK;
 }
 }  // namespace
 
+// after_attention: launched right behind the attention kernel that writes the partials, with
+// programmatic stream serialization: its CTAs are placed as that kernel's CTAs leave and wait
+// (grid_dependency_wait) until it has finished, so no launch gap separates the two.
 int32_t launch_lse_merge(const float* part_O, const float* part_LSE, int32_t n_parts, int64_t rows, int32_t d,
-                         uint16_t* O, float* LSE, cudaStream_t stream) {
-    return launch_merge(part_O, part_LSE, n_parts, rows * d, rows, rows, d, O, false, LSE, stream);
+                         uint16_t* O, float* LSE, cudaStream_t stream, bool after_attention) {
+    return launch_merge(part_O, part_LSE, n_parts, rows * d, rows, rows, d, O, false, LSE, stream, after_attention);
 }
 
 }  // namespace pulsar
@@ -213,7 +259,7 @@ extern "C" int32_t pulsar_lse_merge(const float* part_O, const float* part_LSE, 
     if (!aligned(part_O, 16) || !aligned(part_LSE, 4) || !aligned(O, 8)) return PULSAR_ERR_ALIGNMENT;
     int32_t rc = check_device();
     if (rc != PULSAR_OK) return rc;
-    return launch_lse_merge(part_O, part_LSE, n_parts, rows, d, O, LSE, static_cast<cudaStream_t>(stream));
+    return launch_lse_merge(part_O, part_LSE, n_parts, rows, d, O, LSE, static_cast<cudaStream_t>(stream), false);
 }
 
 extern "C" int32_t pulsar_lse_merge_strided(const float* part_O, const float* part_LSE, int32_t n_parts,
