@@ -36,14 +36,56 @@ from paper_2607_20457_b200 import workloads as W
 
 METRIC = "context_tokens_per_s_per_layer"
 UNIT = "tokens/s"
-# DRAM bytes (read + write) of one Phase-1 attention launch at the 128K workload, from a
-# single-pass ncu capture of this bench command (summary: profiles/bench_128k_launch_list.md).
-PHASE1_DRAM_TRAFFIC_128K = 2.32e9 + 1.08e9
+# Measured DRAM bytes of the dominant kernel, per workload: a small JSON written by
+# `bench.py --traffic-from-ncu-csv <csv>` from an ncu capture of dram__bytes_read.sum and
+# dram__bytes_write.sum of this bench command.  Absent or for another workload: traffic is null.
+TRAFFIC_JSON = os.path.join(os.path.dirname(os.path.abspath(__file__)), "profiles", "phase1_attn_dram_traffic.json")
 
 
 # --------------------------------------------------------------------------------------------
 # helpers
 # --------------------------------------------------------------------------------------------
+def load_traffic(workload: str):
+    """DRAM bytes (read + write) per Phase-1 attention launch at ``workload`` from the tracked
+    capture, or None."""
+    try:
+        rec = json.load(open(TRAFFIC_JSON)).get(workload)
+        return float(rec["dram_bytes_read"] + rec["dram_bytes_write"]) if rec else None
+    except (OSError, ValueError, KeyError, TypeError):
+        return None
+
+
+def traffic_from_ncu_csv(path: str, workload: str):
+    """Reads an ncu --csv log holding dram__bytes_read.sum and dram__bytes_write.sum of the bench's
+    kernels, takes the Phase-1 attention launches (the attention kernel launches with the larger
+    DRAM reads: Phase 2 reads K and V once), and records their per-launch median in TRAFFIC_JSON."""
+    import csv
+    rows = [r for r in csv.reader(open(path, errors="replace")) if len(r) > 10]
+    head = next(r for r in rows if "Metric Name" in r)
+    ix = {n: head.index(n) for n in ("ID", "Kernel Name", "Metric Name", "Metric Unit", "Metric Value")}
+    unit = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}
+    per_launch = {}
+    for r in rows:
+        if r is head or "attn_kernel" not in r[ix["Kernel Name"]] or not r[ix["Metric Name"]].startswith("dram__bytes_"):
+            continue
+        val = float(r[ix["Metric Value"]].replace(",", "")) * unit.get(r[ix["Metric Unit"]], 1.0)
+        per_launch.setdefault(r[ix["ID"]], {})[r[ix["Metric Name"]]] = val
+    launches = [v for v in per_launch.values() if len(v) == 2]
+    if not launches:
+        raise SystemExit(f"{path}: no attention launches with both DRAM metrics")
+    big = max(v["dram__bytes_read.sum"] for v in launches)
+    p1 = [v for v in launches if v["dram__bytes_read.sum"] > 0.5 * big]
+    rec = {}
+    if os.path.exists(TRAFFIC_JSON):
+        rec = json.load(open(TRAFFIC_JSON))
+    rec[workload] = dict(kernel="attn_kernel (Phase 1)", launches=len(p1),
+                         dram_bytes_read=statistics.median(v["dram__bytes_read.sum"] for v in p1),
+                         dram_bytes_write=statistics.median(v["dram__bytes_write.sum"] for v in p1),
+                         source=os.path.basename(path))
+    json.dump(rec, open(TRAFFIC_JSON, "w"), indent=1, sort_keys=True)
+    print(json.dumps(rec[workload]))
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -143,29 +185,67 @@ def max_over_ranks(value: float, world: int, device) -> float:
 # --------------------------------------------------------------------------------------------
 def oracle_sample(w, ids, Q, K, V, Qq, rows_per_block=40, p2_rows=20):
     """Times the float64 oracle, as it stands, on a bounded sample of the workload and scales
-    the three parts to one full step by exact work counts.  Returns a dict."""
+    the three parts to one full step by exact work counts.  Every Phase-1 / Phase-2 call of the
+    oracle first widens all of K and V to float (a fixed cost that does not grow with the rows
+    asked for); it is timed on its own -- a call that asks for no rows -- and counted once per
+    call of the full step instead of being scaled with the rows.  Returns a dict with the timing
+    and the oracle's outputs on the sample."""
     import oracle
     t0 = time.perf_counter()
     sel = oracle.maxidf_select(ids, w.vocab_size, w.block_size, w.chunk, w.k, w.sink)
     t_sel = time.perf_counter() - t0
     pidx, plen = sel["prefix_idx"], sel["prefix_len"]
+    t0 = time.perf_counter()
+    oracle.phase1_attn(Q, K, V, w.block_size, pidx, plen, rows=np.zeros(0, np.int64))
+    t_fixed = time.perf_counter() - t0
     rows = W.sample_rows(w, per_block=rows_per_block)
     t0 = time.perf_counter()
-    oracle.phase1_attn(Q, K, V, w.block_size, pidx, plen, rows=rows)
+    O1, L1 = oracle.phase1_attn(Q, K, V, w.block_size, pidx, plen, rows=rows)
     t_p1 = time.perf_counter() - t0
     sample_pairs = int(sum(int(plen[r // w.block_size]) + (r % w.block_size) + 1 for r in rows))
     total_pairs = cm.phase1_pairs(w.block_size, plen)
     n2 = min(p2_rows, w.nq)
+    q_rows = np.unique(np.linspace(0, w.nq - 1, n2).round().astype(np.int64))
+    n2 = len(q_rows)
     t0 = time.perf_counter()
-    oracle.phase2_attn(Qq[:n2], K, V, w.n_blocks, w.block_size)
+    O2, L2 = oracle.phase2_attn(Qq[torch.from_numpy(q_rows)].contiguous(), K, V, 1, w.L)
     t_p2 = time.perf_counter() - t0
-    est_step = t_sel + t_p1 * total_pairs / sample_pairs + t_p2 * w.nq / n2
+    fixed = min(t_fixed, t_p1, t_p2)
+    est_step = (t_sel + fixed + (t_p1 - fixed) * total_pairs / sample_pairs + fixed + (t_p2 - fixed) * w.nq / n2)
     return dict(
-        value=w.L / est_step, seconds_measured=t_sel + t_p1 + t_p2, est_step_seconds=est_step,
-        cores=oracle.num_threads(),
+        value=w.L / est_step, seconds_measured=t_sel + t_fixed + t_p1 + t_p2, est_step_seconds=est_step,
+        fixed_seconds=fixed, cores=oracle.num_threads(),
         sample=(f"selection in full ({t_sel:.3f}s); Phase 1 on {len(rows)} sampled query positions x all heads "
                 f"({sample_pairs} of {total_pairs} (q,k) pairs per head, {t_p1:.2f}s); Phase 2 on {n2} of {w.nq} "
-                f"query rows ({t_p2:.2f}s); each part scaled to the full step by its exact work count"))
+                f"query rows ({t_p2:.2f}s); each part scaled to the full step by its exact work count after taking "
+                f"out the oracle's fixed cost per call (widening K and V: {fixed:.2f}s, counted once per call)"),
+        outputs=dict(sel=sel, rows=rows, O1=O1, L1=L1, q_rows=q_rows, O2=O2, L2=L2))
+
+
+def parity_of_last_step(slot, ref):
+    """Compares the GPU results of the last timed step with the oracle's outputs on the sample the
+    CPU baseline computed anyway: selection bit for bit, attention outputs element-wise
+    (|dO| <= 1e-2 * max(1, |O_ref|)) and |dLSE| <= 1e-3."""
+    sel_buf, pidx, plen = slot["sel"]
+    sel = ref["sel"]
+    n_sel, n_pref = sel["sel_chunks"].size, sel["prefix_idx"].size
+    exact = (np.array_equal(sel_buf[:n_sel].cpu().numpy(), sel["sel_chunks"].reshape(-1)) and
+             np.array_equal(pidx[:n_pref].cpu().numpy(), sel["prefix_idx"]) and
+             np.array_equal(plen[: sel["prefix_len"].size].cpu().numpy(), sel["prefix_len"]))
+
+    def errs(O, L, Oref, Lref):
+        o = O.float().cpu().numpy().astype(np.float64)
+        e = np.abs(o - Oref)
+        return float(e.max()), float((e / (1e-2 * np.maximum(1.0, np.abs(Oref)))).max()), \
+            float(np.abs(L.cpu().numpy().astype(np.float64) - Lref).max())
+    r1 = torch.from_numpy(ref["rows"]).to(slot["O1"].device)
+    r2 = torch.from_numpy(ref["q_rows"]).to(slot["O2"].device)
+    d1, w1, l1 = errs(slot["O1"][r1], slot["LSE1"][r1], ref["O1"], ref["L1"])
+    d2, w2, l2 = errs(slot["O2"][r2], slot["LSE2"][r2], ref["O2"], ref["L2"])
+    return {"selection_exact": bool(exact), "phase1_max_abs_dO": d1, "phase1_max_abs_dLSE": l1,
+            "phase2_max_abs_dO": d2, "phase2_max_abs_dLSE": l2, "phase1_rows": int(len(ref["rows"])),
+            "phase2_rows": int(len(ref["q_rows"])),
+            "pass": bool(exact and w1 <= 1.0 and w2 <= 1.0 and l1 <= 1e-3 and l2 <= 1e-3)}
 
 
 def run_reference(args, w):
@@ -179,7 +259,7 @@ def run_reference(args, w):
     oracle.build()
     times, last = [], None
     for i in range(args.warmup + args.steps):
-        last = oracle_sample(w, ids, Q, K, V, Qq, rows_per_block=2, p2_rows=1)
+        last = oracle_sample(w, ids, Q, K, V, Qq)      # the same sample as the GPU arm's cpu_baseline leg
         if i >= args.warmup:
             times.append(last["est_step_seconds"])
     est = statistics.mean(times)
@@ -190,7 +270,8 @@ def run_reference(args, w):
         dtype="f64", data="synthetic",
         config=dict(workload=w.name, L=w.L, blocks=w.n_blocks, block_size=w.block_size, chunk=w.chunk, k=w.k,
                     sink=w.sink, Hq=w.Hq, Hkv=w.Hkv, d=w.d, phase2_query_rows=w.nq),
-        cpu_baseline=dict(value=value, unit=UNIT, cores=last["cores"], kind="oracle", sample=last["sample"]),
+        cpu_baseline=dict(value=value, unit=UNIT, cores=last["cores"], kind="oracle", sample=last["sample"],
+                          fixed_seconds=last["fixed_seconds"]),
         e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
         gpu_launches=0,
         note="float64 CPU oracle; each step is a bounded sample scaled to a full step by exact work counts")
@@ -336,8 +417,9 @@ def run_gpu(args, w):
                       peak_source=f"{peaks['source']} sustained bf16 (kernel timed inside a long step)",
                       algorithmic_flops_per_launch=p1_flops,
                       algorithmic_hbm_bytes_per_launch=cm.phase1_hbm_bytes(wl.L, wl.Hq, wl.Hkv, wl.d),
-                      traffic=args.traffic_bytes if args.traffic_bytes is not None else
-                      (PHASE1_DRAM_TRAFFIC_128K if wl.name == "128k" else None),
+                      frac_burst=achieved_tf / peaks["bf16_burst"], peak_burst=peaks["bf16_burst"],
+                      frac_spec_2250=achieved_tf / 2250.0,
+                      traffic=args.traffic_bytes if args.traffic_bytes is not None else load_traffic(wl.name),
                       timed="CUDA events around pulsar_phase1_attn (prefix gather + attention kernel)"),
         e2e=dict(value=world * wl.L / (e2e_ms * 1e-3), unit=UNIT, ms_per_step=e2e_ms,
                  h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h, steps=e2e_steps_report,
@@ -349,7 +431,9 @@ def run_gpu(args, w):
     )
     if cpu is not None:
         line["cpu_baseline"] = dict(value=cpu["value"], unit=UNIT, cores=cpu["cores"], kind="oracle",
-                                    sample=cpu["sample"], seconds_measured=cpu["seconds_measured"])
+                                    sample=cpu["sample"], seconds_measured=cpu["seconds_measured"],
+                                    fixed_seconds=cpu["fixed_seconds"])
+        line["parity"] = parity_of_last_step(enc.slots[0], cpu["outputs"])
     if extras:
         line["extras"] = extras
     print(json.dumps(line), flush=True)
@@ -377,11 +461,12 @@ def run_gpu_blocks(args, w):
         raise SystemExit(f"--shard blocks needs the {w.n_blocks} blocks to divide over {world} ranks")
     lay = ShardLayout.make(w.n_blocks, world, w.block_size, w.chunk, w.k, w.sink, args.mapping)
     coll = TorchCollective() if world > 1 else SingleRankCollective()
-    enc = ShardedContextEncoder(lay, rank, w.Hq, w.Hkv, w.d, w.vocab_size, dev, coll)
     peers = None
     if args.exchange == "fused":                      # Phase-2 partials read in place by the merge kernel
         from paper_2607_20457_b200.sharding import LocalPeers, SymmetricMemoryPeers
         peers = SymmetricMemoryPeers() if world > 1 else LocalPeers(1)
+    # every buffer of a step is allocated here, and the peer buffers meet here: a step allocates nothing
+    enc = ShardedContextEncoder(lay, rank, w.Hq, w.Hkv, w.d, w.vocab_size, dev, coll, nq=w.nq, peers=peers)
 
     # every rank generates the same sequence and keeps its own blocks (pinned host copies for e2e)
     ids = W.token_ids(w)
@@ -580,6 +665,20 @@ def run_extras(binding, w, dev, K_d, V_d, peaks):
     return out
 
 
+def self_launch(n_gpus: int) -> int:
+    """Re-runs this command line as ``n_gpus`` ranks under torch.distributed.run on this node and
+    returns its exit code; rank 0 prints the JSON line."""
+    import socket
+    if torch.cuda.is_available() and torch.cuda.device_count() < n_gpus:
+        raise SystemExit(f"--gpus {n_gpus}: this node shows {torch.cuda.device_count()} GPU(s)")
+    with socket.socket() as sock:                      # a free port for the rendezvous
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -596,10 +695,23 @@ def main():
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--traffic-bytes", type=float, default=None,
                     help="DRAM bytes per Phase-1 launch from an ncu capture (reported as roofline.traffic)")
+    ap.add_argument("--traffic-from-ncu-csv", default=None, metavar="CSV",
+                    help="no benchmark: read an ncu --csv log of dram__bytes_read.sum,dram__bytes_write.sum taken on "
+                         "this command and record the Phase-1 launch's bytes for --workload")
     args = ap.parse_args()
+    if args.traffic_from_ncu_csv:
+        traffic_from_ncu_csv(args.traffic_from_ncu_csv, args.workload)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "pulsar" else args.warmup
     w = W.CONFIGS[args.workload]
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # Started by hand with --gpus N: start the N ranks ourselves (one process per GPU, NCCL over
+        # 127.0.0.1), which is what a launch under torch.distributed.run does.
+        raise SystemExit(self_launch(args.gpus))
     world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world != args.gpus and args.impl == "pulsar":
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}: launch one rank per GPU "
+                         f"(python -m torch.distributed.run --nproc-per-node {args.gpus} bench.py --gpus {args.gpus} ...)")
     if args.impl == "reference":
         run_reference(args, w)
         return

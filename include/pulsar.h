@@ -19,7 +19,8 @@
  *    no pointer after the work enqueued on `stream` has finished.  Scratch comes from the
  *    `workspace` argument, whose minimum size the matching *_workspace_bytes function returns
  *    (256-byte aligned base required).  The workspace may be reused by the next call on the
- *    same stream.
+ *    same stream.  The one exception is pulsar_maxidf_select_noalloc, whose scratch is a fixed
+ *    array inside the library image (see there).
  *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls
  *    only enqueue work and never synchronise the host; inputs and outputs must stay alive
  *    until the stream reaches the end of the call.
@@ -181,8 +182,14 @@ int32_t pulsar_chunk_select(const uint32_t *token_ids, int64_t L, int32_t vocab_
  *    configuration needs about 0.5 MiB; roughly, B * vocab_size / 8 + 2 * vocab_size +
  *    2 * L / chunk bytes must stay below 4 MiB.
  *  - The first call on each device looks up the device address of the scratch array (one
- *    cudaGetSymbolAddress with that device current).  Make that first call outside any stream
- *    capture; later calls only enqueue kernels.
+ *    cudaGetSymbolAddress with that device current).  If the CUDA runtime loads modules lazily,
+ *    that look-up is also what makes the runtime place the library's image -- and with it the
+ *    4 MiB array -- on the device: the call allocates nothing itself, but the first one can be
+ *    the moment those bytes get taken.  Make that first call outside any stream capture; later
+ *    calls only enqueue kernels.
+ *  - The address is remembered per device for the life of the process.  After a
+ *    cudaDeviceReset, or when the device's primary context is destroyed and created again, it
+ *    is stale: do not call this entry point again in such a process.
  *  - All calls on a device share the one array.  Nothing in it has to be cleared between calls
  *    (each region is written in full before it is read), but two calls whose kernels may run
  *    at the same time (different streams without an ordering between them) race on it and

@@ -208,19 +208,24 @@ def pulsar_maxidf_select(token_ids: torch.Tensor, vocab_size: int, block_size: i
 
 def pulsar_maxidf_select_noalloc(token_ids: torch.Tensor, vocab_size: int, block_size: int, chunk: int, k: int,
                                  sink: int, sel_chunks: torch.Tensor, prefix_idx: torch.Tensor,
-                                 prefix_len: torch.Tensor, status=None):
+                                 prefix_len: torch.Tensor, status=None, df_out=None, idf_out=None):
     """Selection through the entry point that needs no workspace (its scratch is built into the
     library, 4 MiB per GPU).  The caller passes every buffer: token_ids int32 [L] in, and the
     outputs sel_chunks [B*k], prefix_idx [sink+(B-1)*k*chunk], prefix_len [B] (CUDA int32).
+    ``df_out`` (int32 [vocab]) and ``idf_out`` (float32 [vocab]) optionally receive the tables.
     Raises PulsarError(PULSAR_ERR_WORKSPACE) if the problem does not fit the built-in scratch.
     Calls that may overlap on the GPU share that scratch and must be ordered by the caller."""
     lib = load_library()
     for t, n in ((token_ids, "token_ids"), (sel_chunks, "sel_chunks"), (prefix_idx, "prefix_idx"),
                  (prefix_len, "prefix_len")):
         _need(t, torch.int32, n)
+    if df_out is not None:
+        _need(df_out, torch.int32, "df_out")
+    if idf_out is not None:
+        _need(idf_out, torch.float32, "idf_out")
     rc = lib.pulsar_maxidf_select_noalloc(_p(token_ids), token_ids.numel(), vocab_size, block_size, chunk, k, sink,
-                                          _p(sel_chunks), _p(prefix_idx), _p(prefix_len), None, None, _p(status),
-                                          _stream())
+                                          _p(sel_chunks), _p(prefix_idx), _p(prefix_len), _p(df_out), _p(idf_out),
+                                          _p(status), _stream())
     _check("pulsar_maxidf_select_noalloc", rc)
 
 
@@ -324,10 +329,11 @@ def phase2_workspace_bytes(nq, B, block_size, Hq, Hkv, d, n_splits=0) -> int:
 
 def pulsar_phase2_attn(Qq, Kblocks, Vblocks, n_blocks: int, block_size: int, softmax_scale: float = 0.0,
                        n_splits: int = 0, want_partials: bool = False, out=None, lse_out=None, workspace=None,
-                       status=None):
+                       status=None, partials=None):
     """Phase-2 query attention with exact LSE merge.  Qq [nq,Hq,d], K/V [n_blocks*block_size,Hkv,d]
     CUDA bf16.  Returns (O bf16 [nq,Hq,d], LSE f32 [nq,Hq]) and, with ``want_partials``
-    (needs n_splits > 0), also (part_O f32 [J,nq,Hq,d], part_LSE f32 [J,nq,Hq])."""
+    (needs n_splits > 0), also (part_O f32 [J,nq,Hq,d], part_LSE f32 [J,nq,Hq]); ``partials`` may
+    give those two tensors preallocated."""
     lib = load_library()
     for t, n in ((Qq, "Qq"), (Kblocks, "Kblocks"), (Vblocks, "Vblocks")):
         _need(t, torch.bfloat16, n)
@@ -337,7 +343,12 @@ def pulsar_phase2_attn(Qq, Kblocks, Vblocks, n_blocks: int, block_size: int, sof
     O = torch.empty_like(Qq) if out is None else out
     LSE = lse_out if lse_out is not None else torch.empty((nq, Hq), dtype=torch.float32, device=dev)
     pO = pL = None
-    if want_partials:
+    if partials is not None:
+        pO, pL = partials
+        want_partials = True
+        _need(pO, torch.float32, "part_O")
+        _need(pL, torch.float32, "part_LSE")
+    elif want_partials:
         pO = torch.empty((n_splits, nq, Hq, d), dtype=torch.float32, device=dev)
         pL = torch.empty((n_splits, nq, Hq), dtype=torch.float32, device=dev)
     if workspace is None:

@@ -67,7 +67,8 @@ struct AttnArgs {
     int pairs_last;        // phase 1: query-tile pairs of the last block
     int n_items;           // work items in total
     int n_blocks;          // phase 1
-    int32_t* counter;      // phase 1: work counter (zeroed before the launch); null = fixed round order
+    int32_t* counter;      // work counter (zeroed before the launch): items are drawn in index order as CTAs
+                           // become free; null = fixed round order
     float scale_log2;      // softmax scale * log2(e)
     uint16_t* O;           // bf16 [tokens, Hq, d]   (final output mode)
     float* LSE;            // f32  [tokens, Hq] or null
@@ -101,8 +102,18 @@ gather_prefix_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V, c
         s_src = src;
     }
     __syncthreads();
-    if (s_src < 0) return;
-    const size_t src = static_cast<size_t>(s_src) * row_vecs, dst = static_cast<size_t>(j) * row_vecs;
+    const size_t dst = static_cast<size_t>(j) * row_vecs;
+    if (s_src < 0) {
+        // An entry no block uses still shares a key tile with used ones: the attention kernel masks
+        // its logits, but the PV product multiplies whatever the row holds by zero, and 0 * NaN
+        // is NaN.  The workspace is the caller's and may hold anything, so the row is cleared.
+        for (int v = threadIdx.x; v < row_vecs; v += blockDim.x) {
+            Kp[dst + v] = make_uint4(0u, 0u, 0u, 0u);
+            Vp[dst + v] = make_uint4(0u, 0u, 0u, 0u);
+        }
+        return;
+    }
+    const size_t src = static_cast<size_t>(s_src) * row_vecs;
     for (int v = threadIdx.x; v < row_vecs; v += blockDim.x) {
         Kp[dst + v] = K[src + v];
         Vp[dst + v] = V[src + v];
@@ -510,8 +521,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 // the lanes that went ahead (two phases behind, its parity test would read "not yet"
                 // again and it would stall until the bound expires).
                 __syncwarp();
-                // Next work item: drawn from the global counter (phase 1: items differ in cost, so
-                // they are handed out as CTAs become free) or the fixed round order (phase 2).
+                // Next work item: drawn from the global counter (items differ in cost or outnumber the
+                // CTAs, so they are handed out as CTAs become free) or the fixed round order.
                 // It is published through a small queue for the MMA issuer and the softmax warps.
                 const uint32_t slot = seq % kItemQueue;
                 ok = mbar_wait_a(bar0 + 8 * (SL::bItemEmpty + slot), ((seq / kItemQueue) & 1) ^ 1, abort_flag, a.status);
@@ -1366,7 +1377,7 @@ extern "C" size_t pulsar_phase2_workspace_bytes(int32_t nq, int32_t B, int32_t b
     size_t a, b;
     if (plan_phase2(nq, B, block_size, Hq, Hkv, d, n_splits, a, b) != PULSAR_OK) return 0;
     if (phase2_quad(nq, Hq / Hkv)) return 4 * (a + b);
-    return n_splits == 1 ? 256 : a + b;
+    return n_splits == 1 ? 256 : a + b + 256;              // partials and the work counter
 }
 
 extern "C" int32_t pulsar_phase2_attn(const uint16_t* Qq, int32_t nq, const uint16_t* Kb, const uint16_t* Vb,
@@ -1390,7 +1401,7 @@ extern "C" int32_t pulsar_phase2_attn(const uint16_t* Qq, int32_t nq, const uint
     po_bytes *= copies;                                        // both stay multiples of 256
     pl_bytes *= copies;
     const bool need_ws = (n_splits > 1 || quad) && !user_parts;
-    if (need_ws && (!workspace || workspace_bytes < po_bytes + pl_bytes)) return PULSAR_ERR_WORKSPACE;
+    if (need_ws && (!workspace || workspace_bytes < po_bytes + pl_bytes + (quad ? 0 : 256))) return PULSAR_ERR_WORKSPACE;
     rc = check_device();
     if (rc != PULSAR_OK) return rc;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -1429,6 +1440,13 @@ extern "C" int32_t pulsar_phase2_attn(const uint16_t* Qq, int32_t nq, const uint
     a.Hkv = Hkv;
     a.pairs = (row_tiles + 1) / 2;
     a.n_items = a.pairs * Hkv * n_splits;
+    if (a.n_items > sm_count() && need_ws && !quad && workspace_bytes >= po_bytes + pl_bytes + 256) {
+        // More items than CTAs: hand them out as CTAs become free (the last part is shorter, and the
+        // last round would otherwise leave CTAs idle behind the slowest one).  The result of an
+        // item does not depend on which CTA computes it.
+        a.counter = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + po_bytes + pl_bytes);
+        PULSAR_CUDA_OK(cudaMemsetAsync(a.counter, 0, sizeof(int32_t), stream));
+    }
     rc = d == 128 ? launch_attn<128>(tmQ, tmK, tmV, tmK, tmV, a, stream)
                   : launch_attn<64>(tmQ, tmK, tmV, tmK, tmV, a, stream);
     if (rc != PULSAR_OK) return rc;

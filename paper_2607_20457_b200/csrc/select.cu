@@ -541,7 +541,9 @@ void* g_scratch_ptr[kMaxDevices] = {};
 
 // Device address of g_select_scratch on the current device.  In host code the symbol's name is
 // only a stand-in; the address a kernel can use comes from cudaGetSymbolAddress, looked up once
-// per device with that device current.
+// per device with that device current and remembered for the life of the process.  (A device
+// reset, or a primary context torn down and created again, would leave the remembered address
+// stale: the header tells callers not to use this entry point across one.)
 int32_t static_scratch(void** out) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {

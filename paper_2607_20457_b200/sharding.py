@@ -73,6 +73,14 @@ class ShardLayout:
     def prefix_len_local(self, h: int) -> np.ndarray:
         return np.array([0 if i == 0 else self.sink + i * self.sigma for i in self.local_blocks(h)], np.int32)
 
+    def row_slice(self, h: int, rows: int):
+        """Rows of a [rows, d] result that rank h merges when the Phase-2 exchange is fused into the
+        merge: (first row, count).  ceil(rows / H) rows per rank, the last ranks taking what is left
+        (possibly nothing)."""
+        per = (rows + self.n_hosts - 1) // self.n_hosts
+        begin = min(h * per, rows)
+        return begin, min(per, rows - begin)
+
     def prefix_order(self) -> np.ndarray:
         """For each position of the prefix list, its row in the all-gathered send buffers, the
         buffer of rank h holding [K rows | V rows], ``send_rows`` each (so rank h's K rows start at
@@ -100,10 +108,12 @@ class TorchCollective:
         self.world = dist.get_world_size(group)
         self.rank = dist.get_rank(group)
 
-    def all_gather(self, send: torch.Tensor) -> torch.Tensor:
+    def all_gather(self, send: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:
+        """``out`` (optional): a preallocated contiguous tensor of world * send.numel() elements."""
         flat = send.contiguous().view(-1)
-        out = torch.empty(self.world * flat.numel(), dtype=send.dtype, device=send.device)
-        self._dist.all_gather_into_tensor(out, flat, group=self._group)
+        if out is None:
+            out = torch.empty(self.world * flat.numel(), dtype=send.dtype, device=send.device)
+        self._dist.all_gather_into_tensor(out.view(-1), flat, group=self._group)
         return out.view((self.world,) + tuple(send.shape))
 
 
@@ -111,7 +121,7 @@ class SingleRankCollective:
     """The all_gather of a one-rank job: the send buffer with a leading dimension of 1."""
     world, rank = 1, 0
 
-    def all_gather(self, send: torch.Tensor) -> torch.Tensor:
+    def all_gather(self, send: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:
         return send.unsqueeze(0)
 
 
@@ -159,28 +169,84 @@ class SymmetricMemoryPeers:
 
 
 class ShardedContextEncoder:
-    """One rank's part of the sharded context encoding.  ``collective`` supplies all_gather."""
+    """One rank's part of the sharded context encoding.  ``collective`` supplies all_gather.
+
+    Every buffer a step needs -- selection outputs and workspace, exchange buffers, Phase-1 outputs,
+    Phase-2 partials, send and receive buffers, results -- is allocated here (the Phase-2 ones for
+    ``nq`` query rows, by ``plan_phase2``), and with ``peers`` the peer-visible buffer is allocated
+    and its rendezvous done here too: a step allocates nothing and meets no other rank outside its
+    collectives.  A Phase-2 call with a different number of query rows re-plans first."""
 
     def __init__(self, layout: ShardLayout, rank: int, Hq: int, Hkv: int, d: int, vocab_size: int, device,
-                 collective=None):
+                 collective=None, nq: int | None = None, peers=None, phase2_splits: int = 0):
         from . import binding
         self.b = binding
         self.lay, self.rank, self.Hq, self.Hkv, self.d, self.V = layout, rank, Hq, Hkv, d, vocab_size
-        self.dev = torch.device(device)
+        self.dev = dev = torch.device(device)
         self.coll = collective
-        self.status = binding.new_status(self.dev)
-        self.block_ids = torch.tensor(layout.local_blocks(rank), dtype=torch.int32, device=self.dev)
-        self.plen_local = torch.from_numpy(layout.prefix_len_local(rank)).to(self.dev)
-        self.order = torch.from_numpy(layout.prefix_order()).to(self.dev)
-        self.send_kv = torch.empty((2, layout.send_rows, Hkv, d), dtype=torch.bfloat16, device=self.dev)
-        self.Kp = torch.empty((max(layout.prefix_total, 1), Hkv, d), dtype=torch.bfloat16, device=self.dev)
+        self.status = binding.new_status(dev)
+        self.block_ids = torch.tensor(layout.local_blocks(rank), dtype=torch.int32, device=dev)
+        self.plen_local = torch.from_numpy(layout.prefix_len_local(rank)).to(dev)
+        self.order = torch.from_numpy(layout.prefix_order()).to(dev)
+        self.send_kv = torch.empty((2, layout.send_rows, Hkv, d), dtype=torch.bfloat16, device=dev)
+        self.Kp = torch.empty((max(layout.prefix_total, 1), Hkv, d), dtype=torch.bfloat16, device=dev)
         self.Vp = torch.empty_like(self.Kp)
+        L = layout.n_blocks * layout.block_size
+        L_local = layout.n_local * layout.block_size
+        self.ws_select = binding._workspace(binding.maxidf_select_workspace_bytes(
+            L, vocab_size, layout.block_size, layout.chunk, layout.k, layout.sink), dev)
+        self.sel_out = (torch.empty(layout.n_blocks * layout.k + 4, dtype=torch.int32, device=dev),
+                        torch.empty(layout.prefix_total + 4, dtype=torch.int32, device=dev),
+                        torch.empty(max(layout.n_blocks, 1), dtype=torch.int32, device=dev))
+        self.gathered_kv = torch.empty((layout.n_hosts,) + tuple(self.send_kv.shape), dtype=torch.bfloat16, device=dev)
+        self.O1 = torch.empty((L_local, Hq, d), dtype=torch.bfloat16, device=dev)
+        self.LSE1 = torch.empty((L_local, Hq), dtype=torch.float32, device=dev)
+        self.ws_p1 = binding._workspace(256, dev)
+        self._p2 = None
+        self._peers = peers
+        if nq is not None:
+            self.plan_phase2(nq, phase2_splits)
+
+    def plan_phase2(self, nq: int, n_splits: int = 0):
+        """Allocates what Phase 2 needs for ``nq`` query rows; with peers, also the peer-visible
+        buffer (all ranks must call this together: the rendezvous is a collective)."""
+        lay, dev, rows = self.lay, self.dev, nq * self.Hq
+        J = n_splits or self.b.phase2_choose_splits(nq, lay.n_local, lay.block_size, self.Hq, self.Hkv, self.d)
+        per = (rows + lay.n_hosts - 1) // lay.n_hosts
+        _, n_mine = self.row_slice(nq)
+        p = dict(nq=nq, J=J,
+                 pO=torch.empty((J, nq, self.Hq, self.d), dtype=torch.float32, device=dev),
+                 pL=torch.empty((J, nq, self.Hq), dtype=torch.float32, device=dev),
+                 ws=self.b._workspace(256, dev),
+                 O_local=torch.empty((nq, self.Hq, self.d), dtype=torch.bfloat16, device=dev),
+                 L_local=torch.empty((nq, self.Hq), dtype=torch.float32, device=dev),
+                 send=torch.empty(self.partial_stride(nq), dtype=torch.float32, device=dev),
+                 gathered=torch.empty((lay.n_hosts, self.partial_stride(nq)), dtype=torch.float32, device=dev),
+                 O=torch.empty((nq, self.Hq, self.d), dtype=torch.bfloat16, device=dev),
+                 LSE=torch.empty((nq, self.Hq), dtype=torch.float32, device=dev),
+                 O_slice=torch.empty((max(n_mine, 1), self.d), dtype=torch.bfloat16, device=dev),
+                 L_slice=torch.empty(max(n_mine, 1), dtype=torch.float32, device=dev),
+                 o_pad=torch.zeros((per, self.d), dtype=torch.bfloat16, device=dev),
+                 l_pad=torch.zeros(per, dtype=torch.float32, device=dev),
+                 o_all=torch.empty((lay.n_hosts, per, self.d), dtype=torch.bfloat16, device=dev),
+                 l_all=torch.empty((lay.n_hosts, per), dtype=torch.float32, device=dev),
+                 peer_buf=None)
+        if self._peers is not None:
+            p["peer_buf"] = self._peers.alloc(self.rank, self.partial_stride(nq), dev)
+        self._p2 = p
+        return p
+
+    def _plan_for(self, nq: int, n_splits: int = 0):
+        p = self._p2
+        if p is None or p["nq"] != nq or (n_splits and p["J"] != n_splits):
+            p = self.plan_phase2(nq, n_splits)
+        return p
 
     # ---- selection: replicated, no communication ------------------------------------------------
     def select(self, token_ids: torch.Tensor):
         lay = self.lay
         self.sel = self.b.pulsar_maxidf_select(token_ids, self.V, lay.block_size, lay.chunk, lay.k, lay.sink,
-                                               status=self.status)
+                                               workspace=self.ws_select, status=self.status, out=self.sel_out)
         return self.sel
 
     # ---- Phase 1 ---------------------------------------------------------------------------------
@@ -203,10 +269,19 @@ class ShardedContextEncoder:
         else:
             Kp = Vp = None
         return self.b.pulsar_phase1_attn_sharded(Q, K, V, lay.block_size, Kp, Vp, self.plen_local,
-                                                 softmax_scale=softmax_scale, status=self.status)
+                                                 softmax_scale=softmax_scale, out=self.O1, lse_out=self.LSE1,
+                                                 workspace=self.ws_p1, status=self.status)
 
     def phase1(self, Q, K, V, softmax_scale: float = 0.0):
-        return self.phase1_finish(self.coll.all_gather(self.phase1_pack(K, V)), Q, K, V, softmax_scale)
+        gathered = self._all_gather(self.phase1_pack(K, V), self.gathered_kv)
+        return self.phase1_finish(gathered, Q, K, V, softmax_scale)
+
+    def _all_gather(self, send, out):
+        """The collective's all_gather into a preallocated buffer where it takes one."""
+        try:
+            return self.coll.all_gather(send, out=out)
+        except TypeError:                      # a test collective with the one-argument form
+            return self.coll.all_gather(send)
 
     # ---- Phase 2 ---------------------------------------------------------------------------------
     def partial_stride(self, nq: int) -> int:
@@ -216,13 +291,18 @@ class ShardedContextEncoder:
 
     def phase2_local(self, Qq, K, V, softmax_scale: float = 0.0, n_splits: int = 0) -> torch.Tensor:
         """(o_h, l_h) of this rank's retained KV as one float32 buffer."""
+        return self._phase2_local(Qq, K, V, softmax_scale, n_splits, into_peer_buffer=False)
+
+    def _phase2_local(self, Qq, K, V, softmax_scale, n_splits, into_peer_buffer: bool):
         lay = self.lay
         nq = Qq.shape[0]
         rows = nq * self.Hq
-        J = n_splits or self.b.phase2_choose_splits(nq, lay.n_local, lay.block_size, self.Hq, self.Hkv, self.d)
-        _, _, pO, pL = self.b.pulsar_phase2_attn(Qq, K, V, lay.n_local, lay.block_size, softmax_scale, n_splits=J,
-                                                 want_partials=True, status=self.status)
-        send = torch.empty(self.partial_stride(nq), dtype=torch.float32, device=self.dev)
+        p = self._plan_for(nq, n_splits)
+        J, pO, pL = p["J"], p["pO"], p["pL"]
+        self.b.pulsar_phase2_attn(Qq, K, V, lay.n_local, lay.block_size, softmax_scale, n_splits=J,
+                                  partials=(pO, pL), out=p["O_local"], lse_out=p["L_local"], workspace=p["ws"],
+                                  status=self.status)
+        send = p["peer_buf"] if into_peer_buffer else p["send"]
         self.b.pulsar_lse_merge_strided(pO.view(-1), pL.view(-1), J, rows * self.d, rows, rows, self.d,
                                         send[: rows * self.d].view(rows, self.d), send[rows * self.d:])
         return send
@@ -232,8 +312,8 @@ class ShardedContextEncoder:
         rows = nq * self.Hq
         stride = self.partial_stride(nq)
         flat = gathered.reshape(-1)
-        O = torch.empty((nq, self.Hq, self.d), dtype=torch.bfloat16, device=self.dev)
-        LSE = torch.empty((nq, self.Hq), dtype=torch.float32, device=self.dev)
+        p = self._plan_for(nq)
+        O, LSE = p["O"], p["LSE"]
         self.b.pulsar_lse_merge_strided(flat, flat[rows * self.d:], gathered.shape[0], stride, stride, rows, self.d,
                                         O.view(rows, self.d), LSE.view(rows))
         return O, LSE
@@ -241,25 +321,14 @@ class ShardedContextEncoder:
     # ---- Phase 2 with the exchange fused into the merge (each rank reduces 1/H of the rows) --------
     def row_slice(self, nq: int):
         """Rows of the [nq*Hq, d] result this rank merges: (first row, count)."""
-        rows = nq * self.Hq
-        per = (rows + self.lay.n_hosts - 1) // self.lay.n_hosts
-        begin = min(self.rank * per, rows)
-        return begin, min(per, rows - begin)
+        return self.lay.row_slice(self.rank, nq * self.Hq)
 
     def phase2_local_into(self, peers, Qq, K, V, softmax_scale: float = 0.0, n_splits: int = 0):
         """As phase2_local, with (o_h, l_h) written to this rank's peer-visible buffer."""
-        nq = Qq.shape[0]
-        if getattr(self, "_peer_buf_nq", None) != nq:
-            self._peer_buf = peers.alloc(self.rank, self.partial_stride(nq), self.dev)
-            self._peer_buf_nq = nq
-        lay, rows = self.lay, nq * self.Hq
-        J = n_splits or self.b.phase2_choose_splits(nq, lay.n_local, lay.block_size, self.Hq, self.Hkv, self.d)
-        _, _, pO, pL = self.b.pulsar_phase2_attn(Qq, K, V, lay.n_local, lay.block_size, softmax_scale, n_splits=J,
-                                                 want_partials=True, status=self.status)
-        send = self._peer_buf
-        self.b.pulsar_lse_merge_strided(pO.view(-1), pL.view(-1), J, rows * self.d, rows, rows, self.d,
-                                        send[: rows * self.d].view(rows, self.d), send[rows * self.d:])
-        return send
+        if self._peers is not peers:           # first use with these peers: allocate and meet (a collective)
+            self._peers = peers
+            self._p2 = None
+        return self._phase2_local(Qq, K, V, softmax_scale, n_splits, into_peer_buffer=True)
 
     def phase2_merge_slice(self, peers, nq: int):
         """This rank's slice of the merged result, read from every rank's buffer in place
@@ -267,8 +336,8 @@ class ShardedContextEncoder:
         first row)."""
         rows = nq * self.Hq
         begin, n = self.row_slice(nq)
-        O = torch.empty((max(n, 1), self.d), dtype=torch.bfloat16, device=self.dev)
-        LSE = torch.empty(max(n, 1), dtype=torch.float32, device=self.dev)
+        p = self._plan_for(nq)
+        O, LSE = p["O_slice"], p["L_slice"]
         if n > 0:
             self.b.pulsar_lse_merge_peers(peers.ptrs(), rows, begin, n, self.d, O, LSE)
         return O[:n], LSE[:n], begin
@@ -281,16 +350,15 @@ class ShardedContextEncoder:
         self.phase2_local_into(peers, Qq, K, V, softmax_scale, n_splits)
         peers.barrier()                                     # stream-ordered: every buffer is complete before it is read
         O, LSE, _ = self.phase2_merge_slice(peers, nq)
-        per = (rows + self.lay.n_hosts - 1) // self.lay.n_hosts
-        o_pad = torch.zeros((per, self.d), dtype=torch.bfloat16, device=self.dev)
-        l_pad = torch.zeros(per, dtype=torch.float32, device=self.dev)
-        o_pad[: O.shape[0]] = O
-        l_pad[: LSE.shape[0]] = LSE
-        Oall = self.coll.all_gather(o_pad).reshape(-1, self.d)[:rows].view(nq, self.Hq, self.d)
-        Lall = self.coll.all_gather(l_pad).reshape(-1)[:rows].view(nq, self.Hq)
+        p = self._p2
+        o_pad, l_pad = p["o_pad"], p["l_pad"]                # padded to ceil(rows / H) rows; the padding stays zero
+        o_pad[: O.shape[0]].copy_(O)
+        l_pad[: LSE.shape[0]].copy_(LSE)
+        Oall = self._all_gather(o_pad, p["o_all"]).reshape(-1, self.d)[:rows].view(nq, self.Hq, self.d)
+        Lall = self._all_gather(l_pad, p["l_all"]).reshape(-1)[:rows].view(nq, self.Hq)
         peers.barrier()                                     # nobody overwrites its buffer while others still read
         return Oall, Lall
 
     def phase2(self, Qq, K, V, softmax_scale: float = 0.0, n_splits: int = 0):
         send = self.phase2_local(Qq, K, V, softmax_scale, n_splits)
-        return self.phase2_finish(self.coll.all_gather(send), Qq.shape[0])
+        return self.phase2_finish(self._all_gather(send, self._p2["gathered"]), Qq.shape[0])

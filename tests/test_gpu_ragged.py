@@ -73,8 +73,12 @@ def test_selection_phase1_phase2(shape):
     Q, K, V = W.qkv(w, q_scale=2.0)
     status = binding.new_status(DEV)
     Kd, Vd = K.to(DEV), V.to(DEV)
+    # the workspace arrives full of NaN patterns: prefix entries that no block uses (a short chunk was
+    # selected, so the list is shorter than its buffer) must not reach the result through 0 * NaN
+    ws = torch.full((binding.phase1_workspace_bytes(w.L, w.Hq, w.Hkv, w.d, w.block_size, out["prefix_idx"].numel()),),
+                    0xFF, dtype=torch.uint8, device=DEV)
     O, LSE, Kr, Vr = binding.pulsar_phase1_attn(Q.to(DEV), Kd, Vd, w.block_size, out["prefix_idx"], out["prefix_len"],
-                                                status=status, retain_copy=True)
+                                                status=status, retain_copy=True, workspace=ws)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     assert torch.equal(Kr, Kd) and torch.equal(Vr, Vd) and Kr.shape[0] == w.L

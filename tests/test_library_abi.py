@@ -43,7 +43,7 @@ def test_workspace_sizes(lib):
     # phase 1: gathered prefix K and V + the work counter
     assert binding.phase1_workspace_bytes(131072, 32, 8, 128, 8192, 7744) == 2 * 7744 * 8 * 128 * 2 + 256
     # phase 2: fp32 partials for the chosen number of parts
-    assert binding.phase2_workspace_bytes(512, 16, 8192, 32, 8, 128, 4) == 4 * 512 * 32 * 129 * 4
+    assert binding.phase2_workspace_bytes(512, 16, 8192, 32, 8, 128, 4) == 4 * 512 * 32 * 129 * 4 + 256   # + work counter
     assert binding.phase2_workspace_bytes(512, 16, 8192, 32, 8, 128, 1) == 256
     # a sequence that ends inside a block: ceil(100/64) = 2 blocks of ceil(64/8) = 8 chunk slots
     assert binding.maxidf_select_workspace_bytes(100, 128, 64, 8, 1, 0) == 3 * 256

@@ -117,3 +117,74 @@ def test_two_gloo_ranks_exchange_and_merge(tmp_path):
     for r in range(2):
         z = np.load(tmp_path / f"r{r}.npz")
         assert z["dO"] < 1e-12 and z["dL"] < 1e-12 and bool(z["ok_prefix"])
+
+
+@pytest.mark.parametrize("H", [1, 2, 3, 4, 8])
+@pytest.mark.parametrize("rows", [1, 4, 15, 20, 21, 128, 2048 + 5])
+def test_row_slices_of_the_fused_exchange_tile_the_rows(H, rows):
+    lay = ShardLayout.make(8 * H, H, 64, 8, 2, 8, "zigzag")
+    slices = [lay.row_slice(h, rows) for h in range(H)]
+    per = -(-rows // H)
+    covered = []
+    for begin, n in slices:
+        assert 0 <= n <= per and 0 <= begin <= rows
+        covered += list(range(begin, begin + n))
+    assert covered == list(range(rows))                       # in rank order, no gap, no overlap
+
+
+def _worker_fused(rank, world, port, out_dir, Hq, Hkv, nq):
+    """The fused Phase-2 exchange and the Phase-1 prefix exchange on `world` gloo ranks with several
+    blocks per rank, the oracle standing in for the kernels."""
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    coll = TorchCollective()
+    w = W.shrink(W.CONFIGS["tiny"], L=6 * 128, block_size=128, chunk=8, k=3, sink=8, vocab_size=4096, Hq=Hq, Hkv=Hkv,
+                 d=16, nq=nq)
+    ids = W.needle_ids(w)
+    ref = oracle.maxidf_select(ids, w.vocab_size, w.block_size, w.chunk, w.k, w.sink)
+    Q, K, V = W.qkv(w)
+    Qq = W.phase2_query(w)
+    ok_prefix = {}
+    res = {}
+    for kind in cm.MAPPINGS:
+        lay = ShardLayout.make(w.n_blocks, world, w.block_size, w.chunk, w.k, w.sink, kind)
+        assert lay.n_local == 6 // world > 1
+        rows_local = lay.local_token_rows(rank)
+        # Phase-1 exchange: pack, all-gather, reorder -> the rows the prefix list names
+        Kb = K.view(torch.int16).reshape(w.L, -1).long().numpy()
+        mine = numpy_pack(lay, rank, Kb, ref["sel_chunks"])
+        gk = coll.all_gather(torch.from_numpy(np.concatenate([mine, -mine]))).numpy().reshape(-1, Kb.shape[1])
+        ok_prefix[kind] = bool(np.array_equal(gk[lay.prefix_order()], Kb[ref["prefix_idx"]]) and
+                               np.array_equal(gk[lay.prefix_order() + lay.send_rows], -Kb[ref["prefix_idx"]]))
+        # Phase 2, exchange fused into the merge: every rank's partial is visible to all (here: gathered),
+        # rank r merges only its slice of the rows, the merged slices are gathered
+        o_h, l_h = oracle.phase2_attn(Qq, K[rows_local], V[rows_local], lay.n_local, w.block_size)
+        n = nq * Hq
+        pO = coll.all_gather(torch.from_numpy(o_h.reshape(n, w.d))).numpy()
+        pL = coll.all_gather(torch.from_numpy(l_h.reshape(n))).numpy()
+        begin, cnt = lay.row_slice(rank, n)
+        per = -(-n // world)
+        o_pad, l_pad = np.zeros((per, w.d)), np.zeros(per)
+        if cnt:
+            o_pad[:cnt], l_pad[:cnt] = oracle.lse_merge(pO[:, begin: begin + cnt], pL[:, begin: begin + cnt])
+        O = coll.all_gather(torch.from_numpy(o_pad)).numpy().reshape(-1, w.d)[:n]
+        LSE = coll.all_gather(torch.from_numpy(l_pad)).numpy().reshape(-1)[:n]
+        O_ref, LSE_ref = oracle.phase2_attn(Qq, K, V, w.n_blocks, w.block_size)
+        res[kind] = (float(np.abs(O - O_ref.reshape(n, w.d)).max()), float(np.abs(LSE - LSE_ref.reshape(n)).max()), cnt)
+    np.savez(os.path.join(out_dir, f"r{rank}.npz"), ok=np.array([ok_prefix[k] for k in cm.MAPPINGS]),
+             dO=np.array([res[k][0] for k in cm.MAPPINGS]), dL=np.array([res[k][1] for k in cm.MAPPINGS]),
+             cnt=np.array([res[k][2] for k in cm.MAPPINGS]))
+    dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("world,Hq,Hkv,nq", [(2, 3, 1, 5), (3, 4, 2, 5)])
+def test_gloo_ranks_fused_exchange_rows_that_do_not_divide(tmp_path, world, Hq, Hkv, nq):
+    assert (nq * Hq) % world != 0
+    port = 33500 + os.getpid() % 2000 + world
+    mp.spawn(_worker_fused, args=(world, port, str(tmp_path), Hq, Hkv, nq), nprocs=world, join=True)
+    counts = np.zeros(len(cm.MAPPINGS), int)
+    for r in range(world):
+        z = np.load(tmp_path / f"r{r}.npz")
+        assert z["ok"].all() and (z["dO"] < 1e-12).all() and (z["dL"] < 1e-12).all()
+        counts += z["cnt"]
+    assert (counts == nq * Hq).all()

@@ -32,16 +32,20 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point():
              (W.CONFIGS["tiny"], W.token_ids(W.shrink(W.CONFIGS["tiny"], zipf_s=2.0)))]
     for w, ids in cases:
         ids_d = to_dev_ids(ids, DEV)
-        ref = binding.pulsar_maxidf_select(ids_d, w.vocab_size, w.block_size, w.chunk, w.k, w.sink)
+        ref = binding.pulsar_maxidf_select(ids_d, w.vocab_size, w.block_size, w.chunk, w.k, w.sink,
+                                           want_df=True, want_idf=True)
         status = binding.new_status(DEV)
         sel, pidx, plen = _buffers(w)
+        df = torch.full((w.vocab_size,), -7, dtype=torch.int32, device=DEV)
+        idf = torch.full((w.vocab_size,), -7.0, dtype=torch.float32, device=DEV)
         binding.pulsar_maxidf_select_noalloc(ids_d, w.vocab_size, w.block_size, w.chunk, w.k, w.sink,
-                                             sel, pidx, plen, status=status)
+                                             sel, pidx, plen, status=status, df_out=df, idf_out=idf)
         torch.cuda.synchronize()
         assert int(status.item()) == 0
         assert torch.equal(sel.view(w.n_blocks, w.k), ref["sel_chunks"])
         assert torch.equal(pidx, ref["prefix_idx"])
         assert torch.equal(plen, ref["prefix_len"])
+        assert torch.equal(df, ref["df"]) and torch.equal(idf, ref["idf"])      # the optional tables too
     # and the first problem once more, after the smaller one has overwritten part of the scratch
     w, ids = cases[0]
     ids_d = to_dev_ids(ids, DEV)
