@@ -241,6 +241,10 @@ constexpr float kRescaleThreshold = 8.0f;      // in log2 units
 #ifndef PULSAR_SPECULATE
 #define PULSAR_SPECULATE 0
 #endif
+#ifndef PULSAR_SPLIT_LD
+#define PULSAR_SPLIT_LD 0
+#endif
+constexpr bool kSplitLd = PULSAR_SPLIT_LD && !PULSAR_SPECULATE;   // read S in two halves, the second in flight during the first half's maximum
 constexpr int kPolyPairs = PULSAR_POLY_PAIRS;  // of every four column pairs, how many use the polynomial exp2
 constexpr bool kSpeculate = PULSAR_SPECULATE;  // form P with the maximum in use while the tile maximum is computed
 // Registers per thread: the kernel is compiled for 168 (twelve warps).  setmaxnreg moves
@@ -390,6 +394,20 @@ __device__ __forceinline__ void decode_item(const AttnArgs& a, const VarlenTable
         it.n_tiles_b = it.has1 ? n : 0;
     }
     it.n_load = max(it.n_tiles_a, it.n_tiles_b);
+}
+
+// Row maximum of logits [kBegin, kBegin + 64) (3-input max, four independent chains).
+template <int kBegin>
+__device__ __forceinline__ float row_max64(const uint32_t (&r)[kTileN]) {
+    float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+    for (int c = kBegin; c < kBegin + 64; c += 8) {
+        m0 = max3(m0, __uint_as_float(r[c]), __uint_as_float(r[c + 1]));
+        m1 = max3(m1, __uint_as_float(r[c + 2]), __uint_as_float(r[c + 3]));
+        m2 = max3(m2, __uint_as_float(r[c + 4]), __uint_as_float(r[c + 5]));
+        m3 = max3(m3, __uint_as_float(r[c + 6]), __uint_as_float(r[c + 7]));
+    }
+    return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
 }
 
 // Row maximum of 128 raw logits (3-input max, four independent chains).
@@ -865,11 +883,31 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 }
 
                 uint32_t r[kTileN];
+                float m_split = -INFINITY;                    // kSplitLd: the tile maximum, formed while S arrives
                 PULSAR_TMEM_LD32_AT(tS + 0, r, 0);
                 PULSAR_TMEM_LD32_AT(tS + 32, r, 32);
-                PULSAR_TMEM_LD32_AT(tS + 64, r, 64);
-                PULSAR_TMEM_LD32_AT(tS + 96, r, 96);
-                tmem_wait_ld();
+                if (kSplitLd) {
+                    tmem_wait_ld();
+                    PULSAR_TMEM_LD32_AT(tS + 64, r, 64);
+                    PULSAR_TMEM_LD32_AT(tS + 96, r, 96);
+                    if (masked) {
+#pragma unroll
+                        for (int c = 0; c < 64; ++c)
+                            if (c >= n_vis) r[c] = 0xff800000u;          // -inf
+                    }
+                    m_split = row_max64<0>(r);
+                    tmem_wait_ld();
+                    if (masked) {
+#pragma unroll
+                        for (int c = 64; c < kTileN; ++c)
+                            if (c >= n_vis) r[c] = 0xff800000u;
+                    }
+                    m_split = fmaxf(m_split, row_max64<64>(r));
+                } else {
+                    PULSAR_TMEM_LD32_AT(tS + 64, r, 64);
+                    PULSAR_TMEM_LD32_AT(tS + 96, r, 96);
+                    tmem_wait_ld();
+                }
 
                 // Fast path (unmasked tile, not the first): the first half of the probabilities is
                 // formed with the maximum already in use while the tile's own maximum is computed
@@ -891,12 +929,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                     }
                 }
                 if (exact) {
-                    if (masked) {
+                    if (masked && !kSplitLd) {
 #pragma unroll
                         for (int c = 0; c < kTileN; ++c)
                             if (c >= n_vis) r[c] = 0xff800000u;          // -inf
                     }
-                    const float m_tile = row_max128(r) * a.scale_log2;
+                    const float m_tile = (kSplitLd ? m_split : row_max128(r)) * a.scale_log2;
                     const bool need = m_tile > m_used + kRescaleThreshold;   // always true on the first tile
                     if (__any_sync(0xffffffffu, need)) {
                         const float m_new = need ? m_tile : m_used;
