@@ -244,6 +244,14 @@ constexpr float kRescaleThreshold = 8.0f;      // in log2 units
 #ifndef PULSAR_SPLIT_LD
 #define PULSAR_SPLIT_LD 0
 #endif
+#ifndef PULSAR_MUFU_TURNS
+#define PULSAR_MUFU_TURNS 0
+#endif
+// The two softmax warps that share a scheduler (warp w of query tile 0 and warp w + 4 of query tile 1)
+// take turns at the exponentials of a key tile instead of interleaving them on the MUFU pipe.
+// Measured at the 128K step, 40 steps alternated twice: 17.09 ms against 15.75 ms for Phase 1 (and 2.12
+// against 1.92 us per pair of tiles on long causal blocks): off.  See mufu_turn_take.
+constexpr bool kMufuTurns = PULSAR_MUFU_TURNS;
 constexpr bool kSplitLd = PULSAR_SPLIT_LD && !PULSAR_SPECULATE;   // read S in two halves, the second in flight during the first half's maximum
 constexpr int kPolyPairs = PULSAR_POLY_PAIRS;  // of every four column pairs, how many use the polynomial exp2
 constexpr bool kSpeculate = PULSAR_SPECULATE;  // form P with the maximum in use while the tile maximum is computed
@@ -269,7 +277,8 @@ struct SmemLayout {
     static constexpr int kTmemPtr = kBars + kNumBars * 8;
     static constexpr int kAbort = kTmemPtr + 4;
     static constexpr int kItemQ = kAbort + 4;                      // int [kItemQueue]: published work items
-    static constexpr int kTotal = kItemQ + 4 * kItemQueue;
+    static constexpr int kMufuTurn = kItemQ + 4 * kItemQueue;      // int [4]: per scheduler, 1 while a softmax warp exponentiates
+    static constexpr int kTotal = kMufuTurn + 16;
     static constexpr int kDynBytes = kTotal + 1024;                // room to align the base to 1024 bytes
 };
 
@@ -454,6 +463,41 @@ __device__ __forceinline__ float exp_row128(const uint32_t (&r)[kTileN], float s
     return (acc0.x + acc0.y) + (acc1.x + acc1.y);
 }
 
+// Turn-taking on the MUFU pipe (compile-time option, off: it lost).  Both softmax warps of a
+// scheduler spend two thirds of a key tile's chain (S ready -> P handed over -> PV and next S issued)
+// exponentiating.  The idea: interleaved instruction by instruction they would each run at half the
+// pipe's rate while they overlap, so let one warp run its 128 exponentials alone while the other
+// waits.  The measurement says the opposite: one warp alone does not fill the pipe (its own
+// dependency chains leave it idle), two interleaved warps hide each other's latencies, and taking
+// turns made the kernel 8.5 % slower.  The turn protects no data, only the pipe: one word per
+// scheduler in shared memory, taken with a compare-and-swap by lane 0 and given back with a plain
+// store; nothing blocks while it is held.  The wait is bounded like every other.
+__device__ __forceinline__ bool mufu_turn_take(volatile int* turn, int lane, volatile int* abort_flag, int32_t* status) {
+    bool ok = true;
+    if (lane == 0) {
+        uint32_t polls = 0;
+        uint64_t t0 = 0;
+        while (atomicCAS(const_cast<int*>(turn), 0, 1) != 0) {
+            if ((++polls & 0xffu) == 0) {
+                if (*abort_flag) { ok = false; break; }
+                const uint64_t now = globaltimer_ns();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > kWaitLimitNs) {
+                    *abort_flag = 1;
+                    report(status, PULSAR_DEV_TIMEOUT);
+                    ok = false;
+                    break;
+                }
+            }
+        }
+    }
+    return __all_sync(0xffffffffu, ok);
+}
+__device__ __forceinline__ void mufu_turn_give(volatile int* turn, int lane) {
+    __syncwarp();
+    if (lane == 0) *turn = 0;
+}
+
 // kQuad: the decode-shaped instance (AttnArgs::quad); a separate instantiation keeps its code out
 // of the Phase-1 kernel's register allocation.
 template <int D, bool kQuad>
@@ -476,6 +520,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     // SMs become free; it waits for this grid to finish before it reads anything.
     grid_launch_dependents();
 
+    if (tid < 4) reinterpret_cast<volatile int*>(smem + SL::kMufuTurn)[tid] = 0;
     if (tid == 0) {
         *abort_flag = 0;
         for (int s = 0; s < 2; ++s) {
@@ -768,6 +813,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         uint64_t* bar_p2 = bars + SL::bPFull2 + s;
         uint64_t* bar_of = bars + SL::bOFull + s;
         uint64_t* bar_oe = bars + SL::bOEmpty + s;
+        volatile int* mufu_turn = reinterpret_cast<volatile int*>(smem + SL::kMufuTurn) + (warp & 3);
         uint32_t s_cnt = 0, o_cnt = 0;
         bool ok = true;
 
@@ -957,6 +1003,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                     // P goes to the MMA issuer in two halves of 64 keys, so that the first half
                     // of the PV product runs while the second half of the row is exponentiated.
                     // (The rescale above has stored its O columns before the first hand-over.)
+                    if (kMufuTurns && !kQuad) {
+                        ok = mufu_turn_take(mufu_turn, lane, abort_flag, a.status);
+                        if (!ok) break;
+                    }
                     if (masked) l_run += exp_row128<0, 0, 64>(r, a.scale_log2, neg_m, tS);
                     else l_run += exp_row128<kSpeculate ? 0 : kPolyPairs, 0, 64>(r, a.scale_log2, neg_m, tS);
                     tmem_wait_st();
@@ -965,6 +1015,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                     if (lane == 0) mbar_arrive(bar_p);
                     if (masked) l_run += exp_row128<0, 64, 128>(r, a.scale_log2, neg_m, tS);
                     else l_run += exp_row128<kSpeculate ? 0 : kPolyPairs, 64, 128>(r, a.scale_log2, neg_m, tS);
+                    if (kMufuTurns && !kQuad) mufu_turn_give(mufu_turn, lane);
                 }
 
                 tmem_wait_st();
