@@ -244,6 +244,13 @@ constexpr float kRescaleThreshold = 8.0f;      // in log2 units
 #ifndef PULSAR_SPLIT_LD
 #define PULSAR_SPLIT_LD 0
 #endif
+#ifndef PULSAR_EARLY_RELEASE
+#define PULSAR_EARLY_RELEASE 1
+#endif
+// Hand a query tile's shared memory back to the loader when its last S product has been issued (the PV
+// products that follow do not read Q), and the O accumulator back to the issuer as soon as the epilogue has
+// read it into registers (before the rows are scaled and stored): both shorten the gap between work items.
+constexpr bool kEarlyRelease = PULSAR_EARLY_RELEASE;
 #ifndef PULSAR_MUFU_TURNS
 #define PULSAR_MUFU_TURNS 0
 #endif
@@ -735,12 +742,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 if (!ok) break;
                 tc_fence_after();
                 PULSAR_ISSUE_S(tS0, descQ0, descK + static_cast<uint64_t>(ks * kStageStep), 0);
+                if (kEarlyRelease && n0 == 1 && leader) umma_commit_a(bar0 + 8 * (SL::bQEmpty + 0));
                 if (it.has1) {
                     ok = mbar_wait_a(bar0 + 8 * (SL::bQFull + 1), q_use1 & 1, abort_flag, a.status);
                     ++q_use1;
                     if (!ok) break;
                     tc_fence_after();
                     PULSAR_ISSUE_S(tS1, descQ1, descK + static_cast<uint64_t>(ks * kStageStep), 1);
+                    if (kEarlyRelease && n1 == 1 && leader) umma_commit_a(bar0 + 8 * (SL::bQEmpty + 1));
                 }
                 if (leader) umma_commit_a(bar0 + 8 * (SL::bKvEmpty + ks));
                 for (int t = 0; t < it.n_load; ++t) {
@@ -767,14 +776,18 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                         if (!ok) break;
                         if (t == n0 - 1) {
                             if (leader) umma_commit_a(bar0 + 8 * (SL::bOFull + 0));
-                            if (leader) umma_commit_a(bar0 + 8 * (SL::bQEmpty + 0));
+                            if (!kEarlyRelease && leader) umma_commit_a(bar0 + 8 * (SL::bQEmpty + 0));
                         }
                     }
                     if (more) {
                         ok = mbar_wait_a(bar0 + 8 * (SL::bKvFull + ks), kp, abort_flag, a.status);
                         if (!ok) break;
                         tc_fence_after();
-                        if (t + 1 < n0) PULSAR_ISSUE_S(tS0, descQ0, dk, 0);
+                        if (t + 1 < n0) {
+                            PULSAR_ISSUE_S(tS0, descQ0, dk, 0);
+                            // the tile's last S: nothing reads its Q any more
+                            if (kEarlyRelease && t + 2 == n0 && leader) umma_commit_a(bar0 + 8 * (SL::bQEmpty + 0));
+                        }
                     }
                     if (t < n1) {
                         if (t == 0) {
@@ -786,12 +799,15 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                         if (!ok) break;
                         if (t == n1 - 1) {
                             if (leader) umma_commit_a(bar0 + 8 * (SL::bOFull + 1));
-                            if (leader) umma_commit_a(bar0 + 8 * (SL::bQEmpty + 1));
+                            if (!kEarlyRelease && leader) umma_commit_a(bar0 + 8 * (SL::bQEmpty + 1));
                         }
                     }
                     if (leader) umma_commit_a(bar0 + 8 * (SL::bKvEmpty + vs));
                     if (more) {
-                        if (t + 1 < n1) PULSAR_ISSUE_S(tS1, descQ1, dk, 1);
+                        if (t + 1 < n1) {
+                            PULSAR_ISSUE_S(tS1, descQ1, dk, 1);
+                            if (kEarlyRelease && t + 2 == n1 && leader) umma_commit_a(bar0 + 8 * (SL::bQEmpty + 1));
+                        }
                         if (leader) umma_commit_a(bar0 + 8 * (SL::bKvEmpty + ks));
                     }
                 }
@@ -1039,23 +1055,30 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 const float inv_l = l_run > 0.f ? 1.f / l_run : 0.f;
                 const float lse = (l_run > 0.f) ? (m_used + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
                 const size_t orow = static_cast<size_t>(token) * a.Hq + head;
+                // The whole accumulator row goes to registers first (the logits' registers are free by
+                // now), so that the accumulator can be handed back before the row is scaled and stored.
+                uint32_t o[D];
 #pragma unroll
-                for (int c0 = 0; c0 < D; c0 += 32) {
-                    uint32_t o[32];
-                    tmem_ld32(tO + c0, o);
-                    tmem_wait_ld();
-                    if (!store) continue;
+                for (int c0 = 0; c0 < D; c0 += 32) PULSAR_TMEM_LD32_AT(tO + c0, o, c0);
+                tmem_wait_ld();
+                if (kEarlyRelease) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_oe);
+                }
+                if (store) {
                     if (a.part_O != nullptr) {
                         float4* dst = reinterpret_cast<float4*>(
-                            a.part_O + (static_cast<size_t>(part) * a.n_tokens * a.Hq + orow) * D + c0);
+                            a.part_O + (static_cast<size_t>(part) * a.n_tokens * a.Hq + orow) * D);
 #pragma unroll
-                        for (int c = 0; c < 32; c += 4)
+                        for (int c = 0; c < D; c += 4)
                             dst[c >> 2] = make_float4(__uint_as_float(o[c]) * inv_l, __uint_as_float(o[c + 1]) * inv_l,
                                                       __uint_as_float(o[c + 2]) * inv_l, __uint_as_float(o[c + 3]) * inv_l);
+                        a.part_LSE[static_cast<size_t>(part) * a.n_tokens * a.Hq + orow] = lse;
                     } else {
-                        uint4* dst = reinterpret_cast<uint4*>(a.O + orow * D + c0);
+                        uint4* dst = reinterpret_cast<uint4*>(a.O + orow * D);
 #pragma unroll
-                        for (int c = 0; c < 32; c += 8) {
+                        for (int c = 0; c < D; c += 8) {
                             uint4 v;
                             v.x = pack_bf16x2(__uint_as_float(o[c]) * inv_l, __uint_as_float(o[c + 1]) * inv_l);
                             v.y = pack_bf16x2(__uint_as_float(o[c + 2]) * inv_l, __uint_as_float(o[c + 3]) * inv_l);
@@ -1063,18 +1086,15 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                             v.w = pack_bf16x2(__uint_as_float(o[c + 6]) * inv_l, __uint_as_float(o[c + 7]) * inv_l);
                             dst[c >> 3] = v;
                         }
+                        if (a.LSE != nullptr) a.LSE[orow] = lse;
                     }
                 }
-                if (store) {
-                    if (a.part_O != nullptr)
-                        a.part_LSE[static_cast<size_t>(part) * a.n_tokens * a.Hq + orow] = lse;
-                    else if (a.LSE != nullptr)
-                        a.LSE[orow] = lse;
-                }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_oe);
+            if (!kEarlyRelease) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_oe);
+            }
         }
     }
 
