@@ -715,7 +715,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="128k", choices=list(W.CONFIGS))
+    ap.add_argument("--workload", default="128k", choices=list(W.CONFIGS) + list(W.MORE_WORKLOADS))
     ap.add_argument("--impl", default="pulsar", choices=["pulsar", "reference"])
     ap.add_argument("--shard", default="sequences", choices=["sequences", "blocks"],
                     help="sequences: every GPU encodes its own sequence; blocks: one sequence, blocks spread over GPUs")
@@ -734,7 +734,7 @@ def main():
         traffic_from_ncu_csv(args.traffic_from_ncu_csv, args.workload)
         return
     args.warmup = max(args.warmup, 3) if args.impl == "pulsar" else args.warmup
-    w = W.CONFIGS[args.workload]
+    w = W.CONFIGS.get(args.workload) or W.MORE_WORKLOADS[args.workload]
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         # Started by hand with --gpus N: start the N ranks ourselves (one process per GPU, NCCL over
         # 127.0.0.1), which is what a launch under torch.distributed.run does.

@@ -57,6 +57,11 @@ CONFIGS = {
     "128k": Workload("128k", 131072, 8192, 32, 16, 64, 128256, 32, 8, 128, 512),
 }
 CONFIG_ORDER = ["tiny", "16k", "32k", "64k", "128k"]
+# Beside the five configurations: the 32K shape with head dimension 64 (the tiny configuration is the only one of
+# the five with d = 64 and is too small to time anything but launches).
+MORE_WORKLOADS = {
+    "32k_d64": Workload("32k_d64", 32768, 4096, 32, 8, 64, 128256, 32, 8, 64, 64),
+}
 
 
 def zipf_ids(L: int, vocab_size: int, s: float = 1.1, seed: int = 0) -> np.ndarray:
