@@ -32,6 +32,7 @@ __global__ void __launch_bounds__(kPresenceThreads)
 presence_kernel(const uint32_t* __restrict__ ids, int64_t L, int block_size, int vocab_size, int words,
                 uint32_t* __restrict__ bitmaps, int32_t* status) {
     extern __shared__ uint32_t bits[];
+    grid_launch_dependents();          // the next launch of the chain may be placed; it waits for this grid itself
     const int b = blockIdx.x;
     for (int w = threadIdx.x; w < words; w += blockDim.x) bits[w] = 0u;
     __syncthreads();
@@ -50,6 +51,8 @@ presence_kernel(const uint32_t* __restrict__ ids, int64_t L, int block_size, int
 __global__ void df_idf_kernel(const uint32_t* __restrict__ bitmaps, int n_blocks, int words, int vocab_size,
                               uint16_t* __restrict__ df_table, uint32_t* __restrict__ df_out,
                               float* __restrict__ idf_out) {
+    grid_launch_dependents();
+    grid_dependency_wait();            // the presence sets are complete
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= vocab_size) return;
     const int w = t >> 5, bit = t & 31;
@@ -92,6 +95,8 @@ __global__ void __launch_bounds__(256)
 chunk_level_kernel(const uint32_t* __restrict__ ids, const uint16_t* __restrict__ df_table, int64_t L,
                    int block_size, int chunks_per_block, int n_slots_total, int chunk, int vocab_size, int worst,
                    uint16_t* __restrict__ level) {
+    grid_launch_dependents();
+    grid_dependency_wait();            // the df table is complete
     const int lane = threadIdx.x & 31;
     const int slot = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (slot >= n_slots_total) return;
@@ -200,6 +205,7 @@ topk_kernel(const uint16_t* __restrict__ level_all, int n_blocks, int64_t L, int
     const int k = geo.k_b;                   // a short last block may have fewer than k_all chunks
 
     for (int i = threadIdx.x; i < n_blocks + 3; i += blockDim.x) hist[i] = 0;
+    grid_dependency_wait();                  // the chunk levels are complete
     __syncthreads();
     for (int c = threadIdx.x; c < C; c += blockDim.x) {
         const int lv = level_all[static_cast<size_t>(b) * C + c];
@@ -419,19 +425,17 @@ extern "C" int32_t pulsar_maxidf_select(const uint32_t* token_ids, int64_t L, in
         token_ids, L, block_size, vocab_size, p.words, bitmaps, device_status);
     PULSAR_CUDA_OK(cudaGetLastError());
     count_launch();
-    df_idf_kernel<<<(vocab_size + 255) / 256, 256, 0, stream>>>(bitmaps, p.n_blocks, p.words, vocab_size, df_table,
-                                                                df_out, idf_out);
-    PULSAR_CUDA_OK(cudaGetLastError());
+    // The three launches that follow are programmatic dependents of the one before them: they are placed
+    // while it runs and wait for it on the device, which takes the launch gaps out of the chain.
+    PULSAR_CUDA_OK(launch_kernel(df_idf_kernel, dim3((vocab_size + 255) / 256), dim3(256), 0, stream, true, bitmaps,
+                                 p.n_blocks, p.words, vocab_size, df_table, df_out, idf_out));
     count_launch();
     const int n_chunks_total = p.n_blocks * p.C;
-    chunk_level_kernel<<<(n_chunks_total + 7) / 8, 256, 0, stream>>>(token_ids, df_table, L, block_size, p.C,
-                                                                     n_chunks_total, chunk, vocab_size,
-                                                                     p.n_blocks + 1, level);
-    PULSAR_CUDA_OK(cudaGetLastError());
+    PULSAR_CUDA_OK(launch_kernel(chunk_level_kernel, dim3((n_chunks_total + 7) / 8), dim3(256), 0, stream, true, token_ids,
+                                 df_table, L, block_size, p.C, n_chunks_total, chunk, vocab_size, p.n_blocks + 1, level));
     count_launch();
-    topk_kernel<<<p.n_blocks, kTopkThreads, p.topk_smem, stream>>>(level, p.n_blocks, L, block_size, chunk, k, sink,
-                                                                   sel_chunks, prefix_idx, prefix_len);
-    PULSAR_CUDA_OK(cudaGetLastError());
+    PULSAR_CUDA_OK(launch_kernel(topk_kernel, dim3(p.n_blocks), dim3(kTopkThreads), p.topk_smem, stream, true, level,
+                                 p.n_blocks, L, block_size, chunk, k, sink, sel_chunks, prefix_idx, prefix_len));
     count_launch();
     return PULSAR_OK;
 }

@@ -76,3 +76,27 @@ def test_gpus_flag_starts_the_ranks_itself():
     assert len(lines) == 1
     line = json.loads(lines[0])
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["cpu_baseline"]["fixed_seconds"] >= 0
+
+
+def test_traffic_json_is_written_from_an_ncu_csv(tmp_path, monkeypatch):
+    """`bench.py --traffic-from-ncu-csv`: the Phase-1 attention launches are the attention launches with
+    the large DRAM reads; their median bytes land in the tracked JSON, and load_traffic reads them back."""
+    import bench
+    head = ('"ID","Process ID","Process Name","Host Name","Kernel Name","Context","Stream","Block Size","Grid Size",'
+            '"Device","CC","Section Name","Metric Name","Metric Unit","Metric Value"')
+    def row(i, kernel, metric, unit, value):
+        return f'"{i}","1","python","box","{kernel}","1","7","(384, 1, 1)","(148, 1, 1)","0","10.0","Command line profiler metrics","{metric}","{unit}","{value}"'
+    lines = ["==PROF== Connected to process 1", head]
+    launches = [("gather_prefix_kernel", 31.5e6, 0.9e6), ("attn_kernel<128, 0>", 2.26e9, 1.078e9), ("attn_kernel<128, 0>", 0.571e9, 0.063e9),
+                ("lse_merge_kernel<0>", 76e6, 0.1e6), ("attn_kernel<128, 0>", 2.27e9, 1.080e9), ("attn_kernel<128, 0>", 0.571e9, 0.063e9)]
+    for i, (k, rd, wr) in enumerate(launches):
+        lines.append(row(i, k, "dram__bytes_read.sum", "byte", f"{int(rd):,}"))
+        lines.append(row(i, k, "dram__bytes_write.sum", "Mbyte", f"{wr / 1e6:.3f}"))
+    csv_path = tmp_path / "dram.csv"
+    csv_path.write_text("\n".join(lines) + "\n")
+    monkeypatch.setattr(bench, "TRAFFIC_JSON", str(tmp_path / "traffic.json"))
+    bench.traffic_from_ncu_csv(str(csv_path), "128k")
+    rec = json.load(open(tmp_path / "traffic.json"))["128k"]
+    assert rec["launches"] == 2 and rec["dram_bytes_read"] == 2.265e9 and abs(rec["dram_bytes_write"] - 1.079e9) < 1e3
+    assert bench.load_traffic("128k") == rec["dram_bytes_read"] + rec["dram_bytes_write"]
+    assert bench.load_traffic("16k") is None
