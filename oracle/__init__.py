@@ -204,10 +204,11 @@ SCORE_MODES = {"max_idf": 0, "tf_idf": 1, "bm25": 2, "type_token": 3}
 
 def chunk_select(token_ids, vocab_size, block_size, chunk, k, sink, mode):
     """Chunk selection under one of the Appendix C heuristics (``mode`` a key of SCORE_MODES or
-    its number).  Returns sel_chunks [B,k], prefix_idx, prefix_len and score [B,C] (float64)."""
+    its number).  Returns sel_chunks [B,k], prefix_idx, prefix_len and score [B,C] (float64);
+    B = ceil(L/block_size), C = ceil(block_size/chunk), padding as in :func:`maxidf_select`."""
     ids = np.ascontiguousarray(np.asarray(token_ids, dtype=np.uint32))
     L = ids.shape[0]
-    B, C = L // block_size, block_size // chunk
+    B, C = -(-L // block_size), -(-block_size // chunk)
     m = SCORE_MODES.get(mode, mode)
     sel = np.zeros((B, k), np.int32)
     pidx = np.zeros(sink + max(B - 1, 0) * k * chunk, np.int32)

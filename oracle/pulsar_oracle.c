@@ -383,16 +383,17 @@ int oracle_generate_step(const uint16_t *Qnew, const uint16_t *Knew, const uint1
  *                     IDF_BM25(t) = ln((N - df + 0.5)/(df + 0.5) + 1)      (Eq. 7)
  *   mode 3  type-token ratio ("Entropy")  score = distinct tokens / |C|    (Eq. 8)
  * IDF(t) = ln(N / max(df, 1)) (Eq. 5).  Sums run over the chunk's positions in order (BM25:
- * over its types in order of first occurrence), in float64.  Top-k, tie rule, positional order
- * and the prefix list are those of oracle_maxidf_select.
- * Outputs as there; score_out [B*C] float64.
+ * over its types in order of first occurrence), in float64.  Top-k, tie rule, positional order,
+ * the prefix list and the treatment of lengths that do not divide are those of
+ * oracle_maxidf_select: |C| is the number of tokens the chunk has (a short last chunk is scored
+ * on those), lbar = L / (number of chunks in the sequence).
+ * Outputs as there; score_out [B*C] float64 (-inf for a slot without a chunk).
  */
 int oracle_chunk_select(const uint32_t *token_ids, int64_t L, int32_t vocab_size, int32_t block_size,
                         int32_t chunk, int32_t k, int32_t sink, int32_t mode,
                         int32_t *sel_chunks, int32_t *prefix_idx, int32_t *prefix_len, double *score_out) {
     if (L <= 0 || block_size <= 0 || chunk <= 0 || vocab_size <= 0 || mode < 0 || mode > 3) return -1;
-    if (L % block_size != 0 || block_size % chunk != 0) return -1;
-    const int64_t B = L / block_size, C = block_size / chunk;
+    const int64_t B = (L + block_size - 1) / block_size, C = (block_size + chunk - 1) / chunk;
     if (k < 0 || k > C || sink < 0 || sink > block_size) return -1;
     for (int64_t p = 0; p < L; ++p)
         if (token_ids[p] >= (uint32_t)vocab_size) return -1;
@@ -402,70 +403,88 @@ int oracle_chunk_select(const uint32_t *token_ids, int64_t L, int32_t vocab_size
     char *taken = (char *)malloc((size_t)C);
     if (!df || !last_block || !score || !taken) return -2;
     for (int64_t t = 0; t < vocab_size; ++t) last_block[t] = -1;
-    for (int64_t b = 0; b < B; ++b)
-        for (int64_t p = b * block_size; p < (b + 1) * block_size; ++p) {
-            uint32_t t = token_ids[p];
-            if (last_block[t] != b) { last_block[t] = b; df[t] += 1; }
-        }
+    for (int64_t p = 0; p < L; ++p) {
+        const int64_t b = p / block_size;
+        uint32_t t = token_ids[p];
+        if (last_block[t] != b) { last_block[t] = b; df[t] += 1; }
+    }
     const double N = (double)B, k1 = 1.2, bb = 0.75;
-    const double lbar = (double)chunk;                     /* every chunk has the same length */
-    const double Dc = 1.0 - bb + bb * ((double)chunk / lbar);
-    if (prefix_idx) for (int32_t j = 0; j < sink; ++j) prefix_idx[j] = j;
+    /* mean chunk length over the sequence: full blocks have C chunks, the last block what it needs */
+    const int64_t last_len = L - (B - 1) * block_size;
+    const int64_t n_chunks = (B - 1) * C + (last_len + chunk - 1) / chunk;
+    const double lbar = (double)L / (double)n_chunks;
+    const int64_t cap = sink + (B - 1) * (int64_t)k * chunk;
+    const int64_t len0 = L < block_size ? L : block_size;
+    int64_t used = sink < len0 ? sink : len0;
+    if (prefix_idx) for (int64_t j = 0; j < used; ++j) prefix_idx[j] = (int32_t)j;
     for (int64_t b = 0; b < B; ++b) {
+        const int64_t lo = b * block_size;
+        const int64_t hi = lo + block_size < L ? lo + block_size : L;
+        const int64_t Cb = (hi - lo + chunk - 1) / chunk;
+        if (prefix_len) prefix_len[b] = b == 0 ? 0 : (int32_t)used;
         for (int64_t c = 0; c < C; ++c) {
-            const uint32_t *tok = token_ids + b * block_size + c * chunk;
+            const uint32_t *tok = token_ids + lo + c * chunk;
+            int64_t len = hi - (lo + c * chunk);
+            if (len > chunk) len = chunk;
             double s = 0.0;
-            if (mode == 0) {
+            if (len <= 0) {
                 s = -INFINITY;
-                for (int32_t p = 0; p < chunk; ++p) {
+            } else if (mode == 0) {
+                s = -INFINITY;
+                for (int64_t p = 0; p < len; ++p) {
                     uint32_t f = df[tok[p]] > 1 ? df[tok[p]] : 1;
                     double v = log(N / (double)f);
                     if (v > s) s = v;
                 }
             } else if (mode == 1) {
-                for (int32_t p = 0; p < chunk; ++p) {
+                for (int64_t p = 0; p < len; ++p) {
                     uint32_t f = df[tok[p]] > 1 ? df[tok[p]] : 1;
                     s = s + log(N / (double)f);
                 }
-                s = s / (double)chunk;
+                s = s / (double)len;
             } else {
+                const double Dc = (1.0 - bb) + bb * ((double)len / lbar);
                 int32_t distinct = 0;
-                for (int32_t p = 0; p < chunk; ++p) {
+                for (int64_t p = 0; p < len; ++p) {
                     int first = 1;
-                    for (int32_t q = 0; q < p; ++q) if (tok[q] == tok[p]) first = 0;
+                    for (int64_t q = 0; q < p; ++q) if (tok[q] == tok[p]) first = 0;
                     if (!first) continue;
                     ++distinct;
                     if (mode == 2) {
                         int32_t tf = 0;
-                        for (int32_t q = 0; q < chunk; ++q) if (tok[q] == tok[p]) ++tf;
+                        for (int64_t q = 0; q < len; ++q) if (tok[q] == tok[p]) ++tf;
                         double f = (double)df[tok[p]];
                         double idf = log((N - f + 0.5) / (f + 0.5) + 1.0);
                         s = s + (idf * ((double)tf * (k1 + 1.0))) / ((double)tf + k1 * Dc);
                     }
                 }
-                if (mode == 3) s = (double)distinct / (double)chunk;
+                if (mode == 3) s = (double)distinct / (double)len;
             }
             score[c] = s;
             if (score_out) score_out[b * C + c] = s;
         }
         memset(taken, 0, (size_t)C);
-        for (int32_t j = 0; j < k; ++j) {
+        for (int32_t j = 0; j < k && j < Cb; ++j) {
             int64_t best = -1;
-            for (int64_t c = 0; c < C; ++c)
+            for (int64_t c = 0; c < Cb; ++c)
                 if (!taken[c] && (best < 0 || score[c] > score[best])) best = c;
             if (best >= 0) taken[best] = 1;
         }
         int32_t j = 0;
-        for (int64_t c = 0; c < C; ++c) {
+        for (int64_t c = 0; c < Cb; ++c) {
             if (!taken[c]) continue;
             if (sel_chunks) sel_chunks[b * k + j] = (int32_t)c;
-            if (prefix_idx && b < B - 1)
-                for (int64_t p = 0; p < chunk; ++p)
-                    prefix_idx[sink + (b * k + j) * chunk + p] = (int32_t)(b * block_size + c * chunk + p);
+            if (b < B - 1)
+                for (int64_t p = lo + c * chunk; p < lo + (c + 1) * chunk && p < hi; ++p) {
+                    if (prefix_idx) prefix_idx[used] = (int32_t)p;
+                    ++used;
+                }
             ++j;
         }
-        if (prefix_len) prefix_len[b] = b == 0 ? 0 : (int32_t)(sink + b * k * chunk);
+        for (; j < k; ++j)
+            if (sel_chunks) sel_chunks[b * k + j] = -1;
     }
+    if (prefix_idx) for (int64_t j = used; j < cap; ++j) prefix_idx[j] = -1;
     free(df); free(last_block); free(score); free(taken);
     return 0;
 }

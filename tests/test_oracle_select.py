@@ -142,7 +142,7 @@ def test_rejects_shapes_outside_the_definition():
     with pytest.raises(ValueError):
         oracle.maxidf_select(ids, 8, 32, 4, 2, 33)      # sink longer than a block
     with pytest.raises(ValueError):
-        oracle.chunk_select(ids, 8, 24, 4, 1, 0, "bm25")   # the other scores keep whole blocks
+        oracle.chunk_select(ids, 8, 32, 4, 9, 0, "bm25")   # k above chunks per block, any score
 
 
 # ---- lengths that do not divide ---------------------------------------------------------------
@@ -279,3 +279,75 @@ def test_heuristic_closed_forms():
     idf1 = math.log((4 - 1 + 0.5) / (1 + 0.5) + 1)
     assert abs(bm[0, 1] - idf1 * 4 * 2.2 / (4 + 1.2)) < 1e-15  # one type with tf = 4
     assert abs(bm[0, 0] - 4 * idf1 * 2.2 / (1 + 1.2)) < 1e-14  # four types with tf = 1
+
+
+def ragged_scores(ids, nb, m, mode):
+    """Eq. 6-9 on a sequence cut by Python slices: |C| is whatever the slice holds, the mean chunk
+    length is taken over all chunks of the sequence."""
+    from collections import Counter
+    blocks = [ids[s: s + nb].tolist() for s in range(0, len(ids), nb)]
+    B = len(blocks)
+    df = Counter(t for blk in blocks for t in set(blk))
+    chunks = [[blk[s: s + m] for s in range(0, len(blk), m)] for blk in blocks]
+    lbar = len(ids) / sum(len(cs) for cs in chunks)
+    out = []
+    for cs in chunks:
+        row = []
+        for ch in cs:
+            if mode == "max_idf":
+                row.append(max(math.log(B / df[t]) for t in ch))
+            elif mode == "tf_idf":
+                acc = 0.0
+                for t in ch:
+                    acc = acc + math.log(B / df[t])
+                row.append(acc / len(ch))
+            elif mode == "type_token":
+                row.append(len(set(ch)) / len(ch))
+            else:
+                D = (1 - 0.75) + 0.75 * (len(ch) / lbar)
+                acc = 0.0
+                for t in dict.fromkeys(ch):                    # types in order of first occurrence
+                    tf = ch.count(t)
+                    acc = acc + (math.log((B - df[t] + 0.5) / (df[t] + 0.5) + 1) * (tf * 2.2)) / (tf + 1.2 * D)
+                row.append(acc)
+        out.append(row)
+    return out
+
+
+@pytest.mark.parametrize("mode", ["max_idf", "tf_idf", "bm25", "type_token"])
+@pytest.mark.parametrize("L,nb,m,k,sink", [(50, 16, 5, 2, 3), (61, 20, 4, 3, 6), (100, 33, 7, 5, 0), (9, 16, 4, 2, 12)])
+def test_heuristics_on_lengths_that_do_not_divide(mode, L, nb, m, k, sink):
+    ids = np.random.default_rng(L).integers(0, 11, size=L).astype(np.uint32)
+    r = oracle.chunk_select(ids, 11, nb, m, k, sink, mode)
+    sc = ragged_scores(ids, nb, m, mode)
+    B = len(sc)
+    prefix, plen, sel = list(range(min(sink, min(nb, L)))), [], []
+    for b, row in enumerate(sc):
+        for c, v in enumerate(row):
+            assert r["score"][b, c] == v or abs(r["score"][b, c] - v) <= 1e-15 * abs(v)
+        assert np.isneginf(r["score"][b, len(row):]).all()
+        plen.append(0 if b == 0 else len(prefix))
+        best = sorted(sorted(range(len(row)), key=lambda c: (-r["score"][b, c], c))[:k])
+        sel.append(best + [-1] * (k - len(best)))
+        if b < B - 1:
+            for c in best:
+                prefix += list(range(b * nb + c * m, min(b * nb + (c + 1) * m, (b + 1) * nb)))
+    np.testing.assert_array_equal(r["sel_chunks"], np.asarray(sel))
+    np.testing.assert_array_equal(r["prefix_len"], np.asarray(plen))
+    cap = sink + (B - 1) * k * m
+    np.testing.assert_array_equal(r["prefix_idx"], np.asarray(prefix + [-1] * (cap - len(prefix))))
+
+
+def test_bm25_length_normaliser_by_hand():
+    # 10 tokens in chunks of 4: chunks of 4, 4 and 2 tokens, mean length 10/3.  One block, so N = 1 and
+    # every token has df = 1: IDF_BM25 = ln((1 - 1 + 0.5)/(1 + 0.5) + 1) = ln(4/3).
+    ids = np.asarray([1, 1, 1, 1, 2, 3, 4, 5, 6, 6], np.uint32)
+    r = oracle.chunk_select(ids, 8, 10, 4, 1, 0, "bm25")
+    idf, lbar = math.log(4.0 / 3.0), 10.0 / 3.0
+    D4, D2 = 0.25 + 0.75 * (4 / lbar), 0.25 + 0.75 * (2 / lbar)
+    assert abs(r["score"][0, 0] - idf * (4 * 2.2) / (4 + 1.2 * D4)) < 1e-15        # one type, tf = 4
+    assert abs(r["score"][0, 1] - 4 * idf * 2.2 / (1 + 1.2 * D4)) < 1e-15          # four types, tf = 1
+    assert abs(r["score"][0, 2] - idf * (2 * 2.2) / (2 + 1.2 * D2)) < 1e-15        # the short chunk: smaller D
+    assert r["sel_chunks"].tolist() == [[1]]
+    tt = oracle.chunk_select(ids, 8, 10, 4, 1, 0, "type_token")["score"]
+    assert tt[0].tolist() == [0.25, 1.0, 0.5]                                      # the short chunk divides by 2
