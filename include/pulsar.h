@@ -131,15 +131,20 @@ int32_t pulsar_maxidf_select(const uint32_t *token_ids, int64_t L, int32_t vocab
  *   PULSAR_SCORE_TF_IDF      (1/|C|) * sum over the chunk's positions of IDF(t_p)
  *   PULSAR_SCORE_BM25        sum over the chunk's distinct tokens of
  *                            ln((B - df + 0.5)/(df + 0.5) + 1) * tf (k1 + 1) / (tf + k1 D),
- *                            k1 = 1.2, b = 0.75, D = 1 - b + b |C| / mean chunk length (= 1 here,
- *                            all chunks having one length), tf = occurrences within the chunk
+ *                            k1 = 1.2, b = 0.75, D = (1 - b) + b |C| / mean chunk length (the mean over
+ *                            all chunks of the sequence; D = 1 when every chunk has `chunk` tokens),
+ *                            tf = occurrences within the chunk
  *   PULSAR_SCORE_TYPE_TOKEN  distinct tokens in the chunk / |C|
  *
  * with IDF(t) = ln(B / max(df(t),1)).  Scores are float64, accumulated left to right over the
  * positions (BM25: over the types in order of first occurrence) with one rounding per add,
  * multiply and divide; chunks whose scores are the same double tie and the lower index wins.
  *
- *   score_out   out [B*C] float64 device, or NULL
+ * Lengths that do not divide are taken as in pulsar_maxidf_select: |C| is the number of tokens a
+ * chunk has (the last chunk of a block may be short and is scored on those, as Eq. 6-8 divide by
+ * |C|), C = ceil(block_size / chunk) slots per block.
+ *
+ *   score_out   out [B*C] float64 device, or NULL; -inf for a slot without a chunk
  *
  * Requirements beyond pulsar_maxidf_select's (else PULSAR_ERR_SHAPE): B <= 1024, chunk <= 1024,
  * C <= 4096.  score_mode outside the enum: PULSAR_ERR_INVALID_ARG.

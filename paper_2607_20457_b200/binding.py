@@ -242,8 +242,8 @@ def pulsar_chunk_select(token_ids: torch.Tensor, vocab_size: int, block_size: in
     mode = SCORE_MODES.get(score_mode, score_mode)
     L = token_ids.numel()
     dev = token_ids.device
-    B = L // block_size if block_size > 0 else 0
-    C = block_size // chunk if chunk > 0 else 0
+    B = -(-L // block_size) if block_size > 0 else 0
+    C = -(-block_size // chunk) if chunk > 0 else 0
     sel_buf = torch.empty(max(B, 0) * max(k, 0) + 4, dtype=torch.int32, device=dev)
     pidx = torch.empty(max(sink, 0) + max(B - 1, 0) * max(k, 0) * max(chunk, 0) + 4, dtype=torch.int32, device=dev)
     plen = torch.empty(max(B, 1), dtype=torch.int32, device=dev)

@@ -256,41 +256,54 @@ topk_kernel(const uint16_t* __restrict__ level_all, int n_blocks, int64_t L, int
 // Scores are float64 and every operation is an explicitly rounded add, multiply or divide in
 // the order the equations are written (positions left to right, types by first occurrence), so
 // two chunks tie exactly when their scores are the same double.  The logarithms are a table over
-// df = 0..B that the host fills (B + 1 values) and passes as a kernel parameter.
+// df = 0..B that the host fills (B + 1 values) and passes as a kernel parameter.  |C| is the number
+// of tokens the chunk has (the last chunk of a block may be short), the mean chunk length of the
+// BM25 normaliser is L over the number of chunks of the sequence.
 // ---------------------------------------------------------------------------------------------
 constexpr int kMaxScoreBlocks = 1024;
 constexpr int kMaxScoreChunk = 1024;
 constexpr int kMaxScoreChunksPerBlock = 4096;
 struct ScoreTable {
     double by_df[kMaxScoreBlocks + 1];   // Eq. 5 (TF-IDF, Max-IDF) or the BM25 IDF of Eq. 7, per df
-    double k1_plus_1, k1_times_D;        // BM25 constants: k1 + 1 and k1 * D(C)
+    double k1_plus_1, k1, b, one_minus_b, mean_len;   // BM25: D(C) = (1 - b) + b * (|C| / mean chunk length)
 };
 
-// One thread per chunk.
+// One thread per chunk slot.  Slot c of block b covers the tokens [b*block_size + c*chunk, +chunk)
+// that lie inside the block and the sequence (|C| = len); a slot without a chunk scores -inf.
 __global__ void __launch_bounds__(128)
-chunk_score_kernel(const uint32_t* __restrict__ ids, const uint16_t* __restrict__ df_table, int n_chunks_total,
-                   int chunk, int vocab_size, int mode, const __grid_constant__ ScoreTable tab,
-                   double* __restrict__ score) {
-    const int c = blockIdx.x * blockDim.x + threadIdx.x;
-    if (c >= n_chunks_total) return;
-    const uint32_t* tok = ids + static_cast<size_t>(c) * chunk;
+chunk_score_kernel(const uint32_t* __restrict__ ids, const uint16_t* __restrict__ df_table, int64_t L,
+                   int block_size, int chunks_per_block, int n_slots_total, int chunk, int vocab_size, int mode,
+                   const __grid_constant__ ScoreTable tab, double* __restrict__ score) {
+    const int slot = blockIdx.x * blockDim.x + threadIdx.x;
+    if (slot >= n_slots_total) return;
+    const int b = slot / chunks_per_block, c = slot - b * chunks_per_block;
+    const int64_t lo = static_cast<int64_t>(b) * block_size;
+    const int64_t start = lo + static_cast<int64_t>(c) * chunk;
+    const int len = static_cast<int>(max(static_cast<int64_t>(0),
+                                         min(static_cast<int64_t>(chunk), min(lo + block_size, L) - start)));
+    const uint32_t* tok = ids + start;
     const uint32_t V = static_cast<uint32_t>(vocab_size);
     double s = 0.0;
-    if (mode == PULSAR_SCORE_MAX_IDF) {
+    if (len == 0) {
         s = -CUDART_INF;
-        for (int p = 0; p < chunk; ++p) {
+    } else if (mode == PULSAR_SCORE_MAX_IDF) {
+        s = -CUDART_INF;
+        for (int p = 0; p < len; ++p) {
             const uint32_t t = tok[p];
             if (t < V) s = fmax(s, tab.by_df[df_table[t]]);
         }
     } else if (mode == PULSAR_SCORE_TF_IDF) {
-        for (int p = 0; p < chunk; ++p) {
+        for (int p = 0; p < len; ++p) {
             const uint32_t t = tok[p];
             if (t < V) s = __dadd_rn(s, tab.by_df[df_table[t]]);
         }
-        s = __ddiv_rn(s, static_cast<double>(chunk));
+        s = __ddiv_rn(s, static_cast<double>(len));
     } else {
+        // D(C) = (1 - b) + b * (|C| / mean chunk length), then k1 * D(C): one rounding per operation
+        const double k1_times_D =
+            __dmul_rn(tab.k1, __dadd_rn(tab.one_minus_b, __dmul_rn(tab.b, __ddiv_rn(static_cast<double>(len), tab.mean_len))));
         int distinct = 0;
-        for (int p = 0; p < chunk; ++p) {
+        for (int p = 0; p < len; ++p) {
             const uint32_t t = tok[p];
             bool first = true;
             for (int q = 0; q < p; ++q) first = first && (tok[q] != t);
@@ -298,39 +311,44 @@ chunk_score_kernel(const uint32_t* __restrict__ ids, const uint16_t* __restrict_
             ++distinct;
             if (mode == PULSAR_SCORE_BM25 && t < V) {
                 int tf = 0;
-                for (int q = p; q < chunk; ++q) tf += (tok[q] == t) ? 1 : 0;
+                for (int q = p; q < len; ++q) tf += (tok[q] == t) ? 1 : 0;
                 const double tfd = static_cast<double>(tf);
                 const double num = __dmul_rn(tab.by_df[df_table[t]], __dmul_rn(tfd, tab.k1_plus_1));
-                s = __dadd_rn(s, __ddiv_rn(num, __dadd_rn(tfd, tab.k1_times_D)));
+                s = __dadd_rn(s, __ddiv_rn(num, __dadd_rn(tfd, k1_times_D)));
             }
         }
-        if (mode == PULSAR_SCORE_TYPE_TOKEN) s = __ddiv_rn(static_cast<double>(distinct), static_cast<double>(chunk));
+        if (mode == PULSAR_SCORE_TYPE_TOKEN) s = __ddiv_rn(static_cast<double>(distinct), static_cast<double>(len));
     }
-    score[c] = s;
+    score[slot] = s;
 }
 
 // One CTA per block: chunk c is taken when fewer than k chunks beat it (a larger score, or the
 // same score at a lower index); the taken chunks are compacted in index order.
 __global__ void __launch_bounds__(kTopkThreads)
-topk_score_kernel(const double* __restrict__ score_all, int n_blocks, int block_size, int chunk, int k, int sink,
-                  int32_t* __restrict__ sel_chunks, int32_t* __restrict__ prefix_idx,
+topk_score_kernel(const double* __restrict__ score_all, int n_blocks, int64_t L, int block_size, int chunk, int k_all,
+                  int sink, int32_t* __restrict__ sel_chunks, int32_t* __restrict__ prefix_idx,
                   int32_t* __restrict__ prefix_len) {
     extern __shared__ double smem_d[];
-    const int C = block_size / chunk;
+    const int C = (block_size + chunk - 1) / chunk;
     double* sc = smem_d;                                   // [C]
     int* chosen = reinterpret_cast<int*>(sc + C);          // [k]
     __shared__ int warp_sums[kTopkThreads / 32];
+    __shared__ int s_short;
     const int b = blockIdx.x;
+    const PrefixGeometry geo = prefix_geometry(b, n_blocks, L, block_size, chunk, k_all, sink);
+    const int k = geo.k_b;                                 // a short last block may have fewer than k_all chunks
+    const int64_t lo = static_cast<int64_t>(b) * block_size;
+    const int Cb = static_cast<int>((min(static_cast<int64_t>(block_size), L - lo) + chunk - 1) / chunk);
     for (int c = threadIdx.x; c < C; c += blockDim.x) sc[c] = score_all[static_cast<size_t>(b) * C + c];
     __syncthreads();
     int taken_before = 0;
     for (int c0 = 0; c0 < C; c0 += kTopkThreads) {
         const int c = c0 + threadIdx.x;
         int take = 0;
-        if (c < C) {
+        if (c < Cb) {
             const double mine = sc[c];
             int better = 0;
-            for (int o = 0; o < C; ++o) {
+            for (int o = 0; o < Cb; ++o) {
                 const double v = sc[o];
                 better += (v > mine || (v == mine && o < c)) ? 1 : 0;
             }
@@ -340,16 +358,32 @@ topk_score_kernel(const double* __restrict__ score_all, int n_blocks, int block_
         const int pos = taken_before + block_exclusive_scan(take, warp_sums, tot);
         if (take && pos < k) {
             chosen[pos] = c;
-            sel_chunks[static_cast<size_t>(b) * k + pos] = c;
+            sel_chunks[static_cast<size_t>(b) * k_all + pos] = c;
         }
         taken_before += tot;
     }
     __syncthreads();
-    // this entry point takes whole blocks and chunks only: every summary has k * chunk tokens
-    const PrefixGeometry geo = prefix_geometry(b, n_blocks, static_cast<int64_t>(n_blocks) * block_size, block_size,
-                                               chunk, k, sink);
-    write_block_prefix(b, n_blocks, block_size, chunk, k, geo, sink + b * k * chunk, chosen, sel_chunks, prefix_idx,
-                       prefix_len);
+    // Entry of prefix_idx at which this block's summary starts: as in prefix_offset, with the scores
+    // deciding whether an earlier (full) block selected its short last chunk -- it did iff fewer
+    // than k of its other chunks, which all have a lower index, score at least as much.
+    int offset = geo.sink_eff + b * k_all * chunk;
+    if (geo.tail != chunk && k_all > 0 && b > 0) {
+        if (threadIdx.x == 0) s_short = 0;
+        __syncthreads();
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+        for (int j = warp; j < b; j += n_warps) {
+            const double* sj = score_all + static_cast<size_t>(j) * C;
+            const double last = sj[C - 1];
+            int before = 0;
+            for (int c = lane; c < C - 1; c += 32) before += (sj[c] >= last) ? 1 : 0;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
+            if (lane == 0 && before < k_all) atomicAdd(&s_short, 1);
+        }
+        __syncthreads();
+        offset -= s_short * (chunk - geo.tail);
+    }
+    write_block_prefix(b, n_blocks, block_size, chunk, k_all, geo, offset, chosen, sel_chunks, prefix_idx, prefix_len);
 }
 
 struct SelectPlan {
@@ -358,11 +392,9 @@ struct SelectPlan {
     size_t presence_smem, topk_smem;
 };
 
-// whole_only: the entry point takes only lengths that divide (L by block_size, block_size by chunk).
 int32_t plan_select(int64_t L, int32_t vocab_size, int32_t block_size, int32_t chunk, int32_t k, int32_t sink,
-                    SelectPlan& p, bool whole_only = false) {
+                    SelectPlan& p) {
     if (L <= 0 || vocab_size <= 0 || block_size <= 0 || chunk <= 0 || k < 0 || sink < 0) return PULSAR_ERR_INVALID_ARG;
-    if (whole_only && (L % block_size != 0 || block_size % chunk != 0)) return PULSAR_ERR_SHAPE;
     if (L >= (1ll << 31)) return PULSAR_ERR_SHAPE;
     const int64_t B = (L + block_size - 1) / block_size;
     p.C = (block_size + chunk - 1) / chunk;
@@ -451,7 +483,7 @@ struct ScorePlan {
 int32_t plan_score(int64_t L, int32_t vocab_size, int32_t block_size, int32_t chunk, int32_t k, int32_t sink,
                    int32_t mode, ScorePlan& p) {
     if (mode < PULSAR_SCORE_MAX_IDF || mode > PULSAR_SCORE_TYPE_TOKEN) return PULSAR_ERR_INVALID_ARG;
-    int32_t rc = plan_select(L, vocab_size, block_size, chunk, k, sink, p.base, /*whole_only=*/true);
+    int32_t rc = plan_select(L, vocab_size, block_size, chunk, k, sink, p.base);
     if (rc != PULSAR_OK) return rc;
     if (p.base.n_blocks > kMaxScoreBlocks || chunk > kMaxScoreChunk || p.base.C > kMaxScoreChunksPerBlock)
         return PULSAR_ERR_SHAPE;
@@ -501,10 +533,14 @@ extern "C" int32_t pulsar_chunk_select(const uint32_t* token_ids, int64_t L, int
                                                        : std::log(N / static_cast<double>(f > 1 ? f : 1));
     }
     const double k1 = 1.2, bb = 0.75;
-    const double mean_len = static_cast<double>(chunk);          // all chunks have one length
-    const double D = 1.0 - bb + bb * (static_cast<double>(chunk) / mean_len);
+    // mean chunk length over the sequence: full blocks have C chunks, a short last block what it needs
+    const int64_t last_len = L - static_cast<int64_t>(b.n_blocks - 1) * block_size;
+    const int64_t n_chunks = static_cast<int64_t>(b.n_blocks - 1) * b.C + (last_len + chunk - 1) / chunk;
     tab.k1_plus_1 = k1 + 1.0;
-    tab.k1_times_D = k1 * D;
+    tab.k1 = k1;
+    tab.b = bb;
+    tab.one_minus_b = 1.0 - bb;
+    tab.mean_len = static_cast<double>(L) / static_cast<double>(n_chunks);
 
     if (b.presence_smem > 48 * 1024)
         PULSAR_CUDA_OK(cudaFuncSetAttribute(presence_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -518,11 +554,12 @@ extern "C" int32_t pulsar_chunk_select(const uint32_t* token_ids, int64_t L, int
     PULSAR_CUDA_OK(cudaGetLastError());
     count_launch();
     const int n_chunks_total = b.n_blocks * b.C;
-    chunk_score_kernel<<<(n_chunks_total + 127) / 128, 128, 0, stream>>>(token_ids, df_table, n_chunks_total, chunk,
-                                                                         vocab_size, score_mode, tab, score);
+    chunk_score_kernel<<<(n_chunks_total + 127) / 128, 128, 0, stream>>>(token_ids, df_table, L, block_size, b.C,
+                                                                         n_chunks_total, chunk, vocab_size, score_mode,
+                                                                         tab, score);
     PULSAR_CUDA_OK(cudaGetLastError());
     count_launch();
-    topk_score_kernel<<<b.n_blocks, kTopkThreads, p.topk_smem, stream>>>(score, b.n_blocks, block_size, chunk, k,
+    topk_score_kernel<<<b.n_blocks, kTopkThreads, p.topk_smem, stream>>>(score, b.n_blocks, L, block_size, chunk, k,
                                                                          sink, sel_chunks, prefix_idx, prefix_len);
     PULSAR_CUDA_OK(cudaGetLastError());
     count_launch();

@@ -68,6 +68,22 @@ def test_edge_shapes(shape, mode):
     run_and_compare(ids, shape["vocab_size"], shape["block_size"], shape["chunk"], shape["k"], shape["sink"], mode)
 
 
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("shape", [
+    dict(L=1000, block_size=256, chunk=16, k=3, sink=20),      # short last block, chunks divide
+    dict(L=777, block_size=200, chunk=7, k=5, sink=13),        # nothing divides: 4-token last chunks, BM25's D varies
+    dict(L=530, block_size=512, chunk=32, k=4, sink=64),       # last block of 18 tokens: one chunk, fewer than k
+    dict(L=300, block_size=512, chunk=24, k=3, sink=400),      # one block shorter than block and sink
+    dict(L=2049, block_size=128, chunk=9, k=2, sink=5),        # 17 blocks, 2-token last chunks, 1-token last block
+    dict(L=131000, block_size=8192, chunk=32, k=16, sink=64),  # the 128K shape cut short
+])
+def test_lengths_that_do_not_divide(shape, mode):
+    rng = np.random.default_rng(shape["L"])
+    ids = rng.integers(0, 9, size=shape["L"]).astype(np.uint32)          # few types: ties and repeated tokens
+    ids[rng.integers(0, shape["L"], size=shape["L"] // 50)] = rng.integers(9, 4000, size=shape["L"] // 50)
+    run_and_compare(ids, 4096, shape["block_size"], shape["chunk"], shape["k"], shape["sink"], mode)
+
+
 def test_rejections():
     ids = to_dev_ids(np.zeros(1 << 16, np.uint32), DEV)
     with pytest.raises(binding.PulsarError):                  # 2048 blocks: beyond the per-df table

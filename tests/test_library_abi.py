@@ -49,7 +49,7 @@ def test_workspace_sizes(lib):
     assert binding.maxidf_select_workspace_bytes(100, 128, 64, 8, 1, 0) == 3 * 256
     # shapes the kernels do not cover give 0
     assert binding.maxidf_select_workspace_bytes(128, 128, 64, 8, 9, 0) == 0
-    assert lib.pulsar_chunk_select_workspace_bytes(100, 128, 64, 8, 1, 0, 2) == 0     # other scores: whole blocks only
+    assert lib.pulsar_chunk_select_workspace_bytes(100, 128, 64, 8, 1, 0, 2) == 3 * 256   # the other scores too
     assert binding.phase1_workspace_bytes(4096, 4, 1, 96, 1024, 0) == 0
 
 
