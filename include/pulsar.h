@@ -478,7 +478,9 @@ int32_t pulsar_lse_merge_peers(const float *const *part_bases, int32_t n_parts, 
  *                          entry its prefix_idx value, row r of block i the position i*block_size+r
  *   PULSAR_POS_CONTIGUOUS  each input is renumbered 0 .. n_i - 1
  *   pos_out  out [sum_i (prefix_len[i] + block_size)] int32 device; writes beyond pos_capacity
- *            entries are dropped.  A prefix_len outside [0, prefix_total] sets PULSAR_DEV_BAD_LENGTH.
+ *            entries are dropped -- which is also how a sequence that ends inside its last block is
+ *            given: pos_capacity = sum_i prefix_len[i] + L, the last input then ends with the
+ *            sequence.  A prefix_len outside [0, prefix_total] sets PULSAR_DEV_BAD_LENGTH.
  *
  * pulsar_rope_apply: rotary embedding with explicit position ids, rotate-half pairing (element j
  * with element j + d/2), angle = position * theta^(-2j/d):

@@ -121,3 +121,23 @@ def test_rope_full_size_rows_sampled_against_the_oracle():
         bound = 2.0 ** -8 * np.concatenate([mag, mag], axis=-1) + 1e-6
         err = np.abs(Y[torch.from_numpy(pick).to(DEV)].double().cpu().numpy() - ref)
         assert (err <= bound).all(), float((err / bound).max())
+
+
+def test_position_ids_of_a_sequence_with_a_short_last_block():
+    """The last assembled input of a sequence that ends inside a block is shorter: the call takes the
+    total number of rows, and what lies beyond it is not written.  Expected ids written out directly
+    from the definition (sparse: a prefix entry keeps its position, row r of block i is i*n_b + r)."""
+    w = W.shrink(W.CONFIGS["tiny"], L=3000, block_size=1024, chunk=24, k=5, sink=64, vocab_size=4096)
+    ids = W.zipf_ids(w.L, w.vocab_size, 1.3, 9)
+    sel = binding.pulsar_maxidf_select(to_dev_ids(ids, DEV), w.vocab_size, w.block_size, w.chunk, w.k, w.sink)
+    ref = oracle.maxidf_select(ids, w.vocab_size, w.block_size, w.chunk, w.k, w.sink)
+    lens = [min(w.block_size, w.L - i * w.block_size) for i in range(w.n_blocks)]
+    total = int(ref["prefix_len"].sum()) + sum(lens)
+    for mode in ("sparse", "contiguous"):
+        want = []
+        for i, n in enumerate(lens):
+            P = int(ref["prefix_len"][i])
+            want += (ref["prefix_idx"][:P].tolist() if mode == "sparse" else list(range(P)))
+            want += [i * w.block_size + r if mode == "sparse" else P + r for r in range(n)]
+        pos = binding.pulsar_assemble_positions(sel["prefix_idx"], sel["prefix_len"], w.n_blocks, w.block_size, total, mode)
+        assert pos.cpu().tolist() == want
