@@ -110,7 +110,8 @@ int32_t pulsar_wait_selftest(int32_t *device_status, uint64_t limit_ns, int32_t 
  *
  * Requirements (else PULSAR_ERR_SHAPE): 0 <= k <= C, 0 <= sink <= block_size, B <= 65533,
  * L < 2^31, vocab_size <= 1,800,000 (one block's presence bitmap must fit in shared memory),
- * C <= 32768.
+ * C <= 32768, and C + B + k + 3 <= 58,112 (the top-k kernel's per-block tables, 4 bytes each,
+ * must fit in 227 KB of shared memory).
  * ------------------------------------------------------------------------------------------ */
 size_t pulsar_maxidf_select_workspace_bytes(int64_t L, int32_t vocab_size, int32_t block_size,
                                             int32_t chunk, int32_t k, int32_t sink);

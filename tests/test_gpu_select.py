@@ -83,3 +83,15 @@ def test_two_runs_are_identical():
     b = binding.pulsar_maxidf_select(ids, w.vocab_size, w.block_size, w.chunk, w.k, w.sink)
     for key in ("sel_chunks", "prefix_idx", "prefix_len"):
         assert torch.equal(a[key], b[key])
+
+
+def test_many_blocks():
+    """50,000 blocks of one 2-token chunk each: the level histogram of the top-k kernel (one counter per
+    possible df value) nearly fills shared memory; beyond that the call is rejected on the host."""
+    w = W.shrink(W.CONFIGS["tiny"], L=100000, block_size=2, chunk=2, k=1, sink=1, vocab_size=97)
+    rng = np.random.default_rng(1)
+    run_and_compare(rng.integers(0, 97, size=w.L).astype(np.uint32), w, want_tables=True)
+    ids = to_dev_ids(np.zeros(65533, np.uint32), DEV)
+    with pytest.raises(binding.PulsarError) as e:            # 65,533 blocks: within the 16-bit levels, beyond shared memory
+        binding.pulsar_maxidf_select(ids, 97, 1, 1, 1, 0)
+    assert e.value.status == 2
