@@ -36,10 +36,10 @@ from paper_2607_20457_b200 import workloads as W
 
 METRIC = "context_tokens_per_s_per_layer"
 UNIT = "tokens/s"
-# Measured DRAM bytes of the dominant kernel, per workload: a small JSON written by
+# Measured DRAM bytes of the dominant kernel, per workload: a small text file (JSON) written by
 # `bench.py --traffic-from-ncu-csv <csv>` from an ncu capture of dram__bytes_read.sum and
 # dram__bytes_write.sum of this bench command.  Absent or for another workload: traffic is null.
-TRAFFIC_JSON = os.path.join(os.path.dirname(os.path.abspath(__file__)), "profiles", "phase1_attn_dram_traffic.json")
+TRAFFIC_JSON = os.path.join(os.path.dirname(os.path.abspath(__file__)), "profiles", "phase1_attn_dram_traffic.txt")
 
 
 # --------------------------------------------------------------------------------------------
