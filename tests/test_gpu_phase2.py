@@ -71,6 +71,29 @@ def test_small_shapes(shape, n_splits):
     print(run_phase2(w, W.phase2_query(w, q_scale=2.0), K, V, n_splits, what=f"{shape} J={n_splits}", scale=0.2))
 
 
+@pytest.mark.parametrize("nq", [1, 8, 20, 32, 40])
+@pytest.mark.parametrize("n_splits", [1, 2])
+def test_row_maximum_jumps_at_late_key_tiles(nq, n_splits):
+    """One query row's logits jump by far more than the kernel's lazy-rescale threshold at two later
+    key tiles, so the accumulated output is rescaled there while the other rows of the same warp --
+    near-uniform attention, every key tile counts -- pass through the same rescale step with factor 1.
+    Covers the decode mode (nq * g <= 32), the one-tile mode (<= 128 rows) and the two-tile mode."""
+    L, Hq, Hkv, d, tile = 6 * 128 + 40, 8, 2, 128, 128
+    w = W.shrink(W.CONFIGS["tiny"], L=L, block_size=L, Hq=Hq, Hkv=Hkv, d=d, nq=nq)
+    gen = torch.Generator().manual_seed(1234 + nq)
+    u = torch.zeros(d)
+    u[::2] = 1.0 / (d // 2) ** 0.5                                   # unit direction
+    Qq = 0.05 * torch.randn(nq, Hq, d, generator=gen)
+    K = 0.05 * torch.randn(L, Hkv, d, generator=gen)
+    V = torch.randn(L, Hkv, d, generator=gen)
+    for h in (0, Hq - 1):                                            # one row in each KV head's group
+        Qq[nq // 2, h] = 12.0 * u
+    K[3 * tile:, :, :] += 3.0 * u                                    # logit + 36 * scale from key tile 3 on
+    K[5 * tile + 7:, :, :] += 4.0 * u                                # and + 48 * scale more inside key tile 5
+    Qq, K, V = Qq.bfloat16(), K.bfloat16(), V.bfloat16()
+    print(run_phase2(w, Qq, K, V, n_splits, what=f"late maximum nq={nq} J={n_splits}", scale=0.5))
+
+
 def test_per_block_partials_match_oracle_partials():
     w = W.CONFIGS["tiny"]
     _, K, V = W.qkv(w)
