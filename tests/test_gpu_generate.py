@@ -68,3 +68,51 @@ def test_capacity_is_checked_on_the_host():
         binding.pulsar_phase2_generate_step(z(4, w.Hq), z(4, w.Hkv), z(4, w.Hkv), K.to(DEV), V.to(DEV), w.n_blocks,
                                             w.block_size, z(8, w.Hkv), z(8, w.Hkv), gen_len=6)
     assert e.value.status == 2
+
+
+def test_step_captured_as_a_cuda_graph_replays_to_the_same_results():
+    """One generation step (append, attention started beside it, merge started beside the attention)
+    recorded as a CUDA graph: the replay equals the call-by-call step bit for bit, also after the
+    inputs in the captured buffers have changed."""
+    w = W.CONFIGS["tiny"]
+    _, K, V = W.qkv(w)
+    Kd, Vd = K.to(DEV), V.to(DEV)
+    gen = torch.Generator().manual_seed(5)
+    cap, gen_len, n_new = 64, 9, 1
+    rnd = lambda n, h: torch.randn(n, h, w.d, generator=gen).to(torch.bfloat16).to(DEV)
+    Kgen, Vgen = rnd(cap, w.Hkv), rnd(cap, w.Hkv)
+    Qn, Kn, Vn = rnd(n_new, w.Hq), rnd(n_new, w.Hkv), rnd(n_new, w.Hkv)
+    status = binding.new_status(DEV)
+    n_splits = binding.phase2_choose_splits(n_new, w.n_blocks, w.block_size, w.Hq, w.Hkv, w.d)
+    ws = binding._workspace(binding.load_library().pulsar_phase2_generate_workspace_bytes(
+        n_new, w.n_blocks, w.block_size, w.Hq, w.Hkv, w.d, n_splits), DEV)
+    O = torch.empty_like(Qn)
+
+    def step():
+        return binding.pulsar_phase2_generate_step(Qn, Kn, Vn, Kd, Vd, w.n_blocks, w.block_size, Kgen, Vgen, gen_len,
+                                                   n_splits=n_splits, out=O, workspace=ws, status=status)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        _, LSE_g = step()
+    for fresh in (False, True):
+        if fresh:                                       # new token in the captured buffers
+            Qn.copy_(rnd(n_new, w.Hq)); Kn.copy_(rnd(n_new, w.Hkv)); Vn.copy_(rnd(n_new, w.Hkv))
+        O.zero_(); LSE_g.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        O_replay, LSE_replay, K_row = O.clone(), LSE_g.clone(), Kgen[gen_len].clone()
+        _, LSE_e = step()
+        torch.cuda.synchronize()
+        assert torch.equal(O_replay, O) and torch.equal(LSE_replay, LSE_e)
+        assert torch.equal(K_row, Kn[0]) and torch.equal(Kgen[gen_len], Kn[0])
+        to_np = lambda t: t.cpu().view(torch.int16).numpy().view(np.uint16)
+        Oref, Lref = oracle.generate_step(Qn.cpu(), Kn.cpu(), Vn.cpu(), K, V, to_np(Kgen).copy(), to_np(Vgen).copy(),
+                                          gen_len)
+        print(check_attention(O_replay, LSE_replay, Oref, Lref, f"graph replay fresh={fresh}"))
+    assert int(status.item()) == 0
