@@ -599,7 +599,7 @@ def run_extras(binding, w, dev, K_d, V_d, peaks):
     how = ("L2 flushed before every call by writing a 512 MiB buffer and reading it back (clean lines); "
            "events around the call only; ms_after_write_only_flush: the same after a memset alone, whose "
            "dirty lines are written back during the call")
-    for name, nq in (("phase2_decode_8x1", 8), ("phase2_decode_1x1", 1)):
+    for name, nq in (("phase2_decode_8x1", 8), ("phase2_decode_1x1", 1), ("phase2_decode_32x1", 32)):
         Qd = W.phase2_query(w, nq=nq).to(dev)
         J = binding.phase2_choose_splits(nq, w.n_blocks, w.block_size, w.Hq, w.Hkv, w.d)
         ws = binding._workspace(binding.phase2_workspace_bytes(nq, w.n_blocks, w.block_size, w.Hq, w.Hkv, w.d, J), dev)
@@ -609,7 +609,8 @@ def run_extras(binding, w, dev, K_d, V_d, peaks):
             binding.pulsar_phase2_attn(Qd, K_d, V_d, w.n_blocks, w.block_size, n_splits=J, out=O, workspace=ws)
         ms = time_after_flush(call, flush_clean, 12)["median_ms"]
         ms_dirty = time_after_flush(call, flush_dirty, 12)["median_ms"]
-        nbytes = cm.phase2_hbm_bytes(nq, w.L, w.Hq, w.Hkv, w.d, 4 * J)       # four partials per KV part in this mode
+        # four partials per KV part while all query rows of a KV head fit a quarter tile (8 and 1 tokens)
+        nbytes = cm.phase2_hbm_bytes(nq, w.L, w.Hq, w.Hkv, w.d, (4 if nq * (w.Hq // w.Hkv) <= 32 else 1) * J)
         out[name] = dict(ms=ms, splits=J, gbs=nbytes / (ms * 1e-3) / 1e9,
                          frac_of_measured_hbm=nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                          ms_after_write_only_flush=ms_dirty,

@@ -63,6 +63,11 @@ def test_tiny_peaked():
     dict(L=512, block_size=256, Hq=2, Hkv=2, d=64, nq=33),        # g = 1, one row too many for that mode
     dict(L=1152, block_size=384, Hq=4, Hkv=2, d=128, nq=16),      # g = 2, 32 rows
     dict(L=90, block_size=45, Hq=4, Hkv=1, d=64, nq=5),           # fewer keys than one tile
+    # one or two query tiles per KV head and several parts
+    dict(L=1280, block_size=640, Hq=8, Hkv=2, d=128, nq=40),      # g = 4, 160 rows: two query tiles, the second ragged
+    dict(L=1280, block_size=640, Hq=8, Hkv=2, d=64, nq=64),       # 256 rows exactly
+    dict(L=256, block_size=128, Hq=4, Hkv=1, d=128, nq=20),       # two parts of one key tile
+    dict(L=1000, block_size=500, Hq=16, Hkv=4, d=128, nq=33),     # odd key-tile counts per part, ragged last tile
 ])
 @pytest.mark.parametrize("n_splits", [1, 2])
 def test_small_shapes(shape, n_splits):
@@ -71,13 +76,14 @@ def test_small_shapes(shape, n_splits):
     print(run_phase2(w, W.phase2_query(w, q_scale=2.0), K, V, n_splits, what=f"{shape} J={n_splits}", scale=0.2))
 
 
-@pytest.mark.parametrize("nq", [1, 8, 20, 32, 40])
+@pytest.mark.parametrize("nq", [1, 8, 20, 32, 40, 64, 70])
 @pytest.mark.parametrize("n_splits", [1, 2])
 def test_row_maximum_jumps_at_late_key_tiles(nq, n_splits):
     """One query row's logits jump by far more than the kernel's lazy-rescale threshold at two later
     key tiles, so the accumulated output is rescaled there while the other rows of the same warp --
     near-uniform attention, every key tile counts -- pass through the same rescale step with factor 1.
-    Covers the decode mode (nq * g <= 32), the one-tile mode (<= 128 rows) and the two-tile mode."""
+    Covers the decode mode (nq * g <= 32), the one-tile schedule (<= 128 rows) and two and three query
+    tiles per KV head."""
     L, Hq, Hkv, d, tile = 6 * 128 + 40, 8, 2, 128, 128
     w = W.shrink(W.CONFIGS["tiny"], L=L, block_size=L, Hq=Hq, Hkv=Hkv, d=d, nq=nq)
     gen = torch.Generator().manual_seed(1234 + nq)
