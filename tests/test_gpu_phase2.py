@@ -122,6 +122,21 @@ def test_full_size_kv(name, nq):
     print(run_phase2(w, Qq, K, V, 0, what=f"{name} nq={Qq.shape[0]}"))
 
 
+@pytest.mark.parametrize("nq", [1, 24])
+def test_twice_the_largest_configuration_and_a_ragged_end(nq):
+    """262,181 keys (2049 key tiles, the last one of 37 keys) as one block: twice the KV of the largest
+    configuration, through the decode mode (1 token) and the one-tile schedule (24 tokens = 96 rows per
+    KV head), with the split the library picks."""
+    L = 2 * 131072 + 37
+    w = W.shrink(W.CONFIGS["128k"], L=L, block_size=L)
+    gen = torch.Generator().manual_seed(99)
+    K = torch.randn(L, w.Hkv, w.d, generator=gen).to(torch.bfloat16)
+    V = torch.randn(L, w.Hkv, w.d, generator=gen).to(torch.bfloat16)
+    Qq = W.phase2_query(w, nq=nq, seed=17)
+    rows = None if nq == 1 else [0, nq // 2, nq - 1]
+    print(run_phase2(w, Qq, K, V, 0, what=f"256K+37 keys nq={nq}", rows=rows))
+
+
 @pytest.mark.parametrize("n_splits", [0, 9])
 def test_128k_config_own_query(n_splits):
     """The 128K configuration's own Phase-2 call -- 8 queries x 64 tokens = 512 rows, i.e. 16 row
