@@ -98,6 +98,16 @@ def test_full_size_configs_on_sampled_rows(name):
     print(run_phase1(w, Q, K, V, pidx, plen, rows=rows, what=name))
 
 
+def test_twice_the_largest_configuration_on_sampled_rows():
+    """262,144 tokens in 32 blocks of 8192: prefixes up to 15,936 rows (125 key tiles before the block's
+    own 64), 65,536 work items; the prefix is the one the sequence's own token ids select."""
+    w = W.shrink(W.CONFIGS["128k"], L=262144)
+    sel = oracle.maxidf_select(W.token_ids(w), w.vocab_size, w.block_size, w.chunk, w.k, w.sink)
+    Q, K, V = W.qkv(w)
+    rows = W.sample_rows(w, per_block=10)
+    print(run_phase1(w, Q, K, V, sel["prefix_idx"], sel["prefix_len"], rows=rows, what="256k"))
+
+
 def test_64k_star_anchor_sampled_rows():
     w = W.CONFIGS["64k"]
     pidx, plen = W.star_anchor_prefix(w)
