@@ -58,9 +58,11 @@ CONFIGS = {
 }
 CONFIG_ORDER = ["tiny", "16k", "32k", "64k", "128k"]
 # Beside the five configurations: the 32K shape with head dimension 64 (the tiny configuration is the only one of
-# the five with d = 64 and is too small to time anything but launches).
+# the five with d = 64 and is too small to time anything but launches), and the 128K shape at twice the length
+# (32 blocks of 8192: the prefixes grow to 15,936 rows).
 MORE_WORKLOADS = {
     "32k_d64": Workload("32k_d64", 32768, 4096, 32, 8, 64, 128256, 32, 8, 64, 64),
+    "256k": Workload("256k", 262144, 8192, 32, 16, 64, 128256, 32, 8, 128, 512),
 }
 
 
