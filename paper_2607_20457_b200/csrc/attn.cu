@@ -248,9 +248,6 @@ constexpr float kRescaleThreshold = 8.0f;      // in log2 units
 #ifndef PULSAR_SPECULATE
 #define PULSAR_SPECULATE 0
 #endif
-#ifndef PULSAR_SPLIT_LD
-#define PULSAR_SPLIT_LD 0
-#endif
 #ifndef PULSAR_EARLY_RELEASE
 #define PULSAR_EARLY_RELEASE 1
 #endif
@@ -258,15 +255,11 @@ constexpr float kRescaleThreshold = 8.0f;      // in log2 units
 // products that follow do not read Q), and the O accumulator back to the issuer as soon as the epilogue has
 // read it into registers (before the rows are scaled and stored): both shorten the gap between work items.
 constexpr bool kEarlyRelease = PULSAR_EARLY_RELEASE;
-#ifndef PULSAR_MUFU_TURNS
-#define PULSAR_MUFU_TURNS 0
-#endif
-// The two softmax warps that share a scheduler (warp w of query tile 0 and warp w + 4 of query tile 1)
-// take turns at the exponentials of a key tile instead of interleaving them on the MUFU pipe.
-// Measured at the 128K step, 40 steps alternated twice: 17.09 ms against 15.75 ms for Phase 1 (and 2.12
-// against 1.92 us per pair of tiles on long causal blocks): off.  See mufu_turn_take.
-constexpr bool kMufuTurns = PULSAR_MUFU_TURNS;
-constexpr bool kSplitLd = PULSAR_SPLIT_LD && !PULSAR_SPECULATE;   // read S in two halves, the second in flight during the first half's maximum
+// Two more variants were built, measured at the 128K step and taken out again: the two softmax warps of a
+// scheduler taking turns at a key tile's exponentials instead of interleaving them on the MUFU pipe (Phase 1
+// 17.09 ms against 15.75 ms: one warp alone does not fill the pipe, two interleaved warps hide each other's
+// latencies), and reading S from TMEM in two halves with the first half's maximum formed while the second
+// arrives (0.6-1 % slower at the power limit).
 constexpr int kPolyPairs128 = PULSAR_POLY_PAIRS;  // of every four column pairs, how many use the polynomial exp2 (d = 128)
 // Head dimension 64 halves the tensor work per exponential, the GPU stays below its power limit there,
 // and one polynomial pair in four is 3.6 % faster (32K shape with d = 64: 1.228 against 1.272 ms; two pairs
@@ -298,8 +291,7 @@ struct SmemLayout {
     static constexpr int kTmemPtr = kBars + kNumBars * 8;
     static constexpr int kAbort = kTmemPtr + 4;
     static constexpr int kItemQ = kAbort + 4;                      // int [kItemQueue]: published work items
-    static constexpr int kMufuTurn = kItemQ + 4 * kItemQueue;      // int [4]: per scheduler, 1 while a softmax warp exponentiates
-    static constexpr int kTotal = kMufuTurn + 16;
+    static constexpr int kTotal = kItemQ + 4 * kItemQueue;
     static constexpr int kDynBytes = kTotal + 1024;                // room to align the base to 1024 bytes
 };
 
@@ -426,20 +418,6 @@ __device__ __forceinline__ void decode_item(const AttnArgs& a, const VarlenTable
     it.n_load = max(it.n_tiles_a, it.n_tiles_b);
 }
 
-// Row maximum of logits [kBegin, kBegin + 64) (3-input max, four independent chains).
-template <int kBegin>
-__device__ __forceinline__ float row_max64(const uint32_t (&r)[kTileN]) {
-    float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
-#pragma unroll
-    for (int c = kBegin; c < kBegin + 64; c += 8) {
-        m0 = max3(m0, __uint_as_float(r[c]), __uint_as_float(r[c + 1]));
-        m1 = max3(m1, __uint_as_float(r[c + 2]), __uint_as_float(r[c + 3]));
-        m2 = max3(m2, __uint_as_float(r[c + 4]), __uint_as_float(r[c + 5]));
-        m3 = max3(m3, __uint_as_float(r[c + 6]), __uint_as_float(r[c + 7]));
-    }
-    return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
-}
-
 // Row maximum of 128 raw logits (3-input max, four independent chains).
 __device__ __forceinline__ float row_max128(const uint32_t (&r)[kTileN]) {
     float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
@@ -484,41 +462,6 @@ __device__ __forceinline__ float exp_row128(const uint32_t (&r)[kTileN], float s
     return (acc0.x + acc0.y) + (acc1.x + acc1.y);
 }
 
-// Turn-taking on the MUFU pipe (compile-time option, off: it lost).  Both softmax warps of a
-// scheduler spend two thirds of a key tile's chain (S ready -> P handed over -> PV and next S issued)
-// exponentiating.  The idea: interleaved instruction by instruction they would each run at half the
-// pipe's rate while they overlap, so let one warp run its 128 exponentials alone while the other
-// waits.  The measurement says the opposite: one warp alone does not fill the pipe (its own
-// dependency chains leave it idle), two interleaved warps hide each other's latencies, and taking
-// turns made the kernel 8.5 % slower.  The turn protects no data, only the pipe: one word per
-// scheduler in shared memory, taken with a compare-and-swap by lane 0 and given back with a plain
-// store; nothing blocks while it is held.  The wait is bounded like every other.
-__device__ __forceinline__ bool mufu_turn_take(volatile int* turn, int lane, volatile int* abort_flag, int32_t* status) {
-    bool ok = true;
-    if (lane == 0) {
-        uint32_t polls = 0;
-        uint64_t t0 = 0;
-        while (atomicCAS(const_cast<int*>(turn), 0, 1) != 0) {
-            if ((++polls & 0xffu) == 0) {
-                if (*abort_flag) { ok = false; break; }
-                const uint64_t now = globaltimer_ns();
-                if (t0 == 0) t0 = now;
-                else if (now - t0 > kWaitLimitNs) {
-                    *abort_flag = 1;
-                    report(status, PULSAR_DEV_TIMEOUT);
-                    ok = false;
-                    break;
-                }
-            }
-        }
-    }
-    return __all_sync(0xffffffffu, ok);
-}
-__device__ __forceinline__ void mufu_turn_give(volatile int* turn, int lane) {
-    __syncwarp();
-    if (lane == 0) *turn = 0;
-}
-
 // kQuad: the decode-shaped instance (AttnArgs::quad); a separate instantiation keeps its code out
 // of the Phase-1 kernel's register allocation.
 // kSingle: every work item of the launch has one query tile (AttnArgs::single).  With a second tile the
@@ -553,7 +496,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     // SMs become free; it waits for this grid to finish before it reads anything.
     grid_launch_dependents();
 
-    if (tid < 4) reinterpret_cast<volatile int*>(smem + SL::kMufuTurn)[tid] = 0;
     if (tid == 0) {
         *abort_flag = 0;
         for (int s = 0; s < 2; ++s) {
@@ -908,7 +850,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         uint64_t* bar_pv = bars + SL::bOFull + 1;              // kSingle: one completion per PV product
         uint32_t g_tile = 0;                                   // kSingle: key tiles this CTA has walked
         uint64_t* bar_oe = bars + SL::bOEmpty + s;
-        volatile int* mufu_turn = reinterpret_cast<volatile int*>(smem + SL::kMufuTurn) + (warp & 3);
         uint32_t s_cnt = 0, o_cnt = 0;
         bool ok = true;
 
@@ -1041,31 +982,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 }
 
                 uint32_t r[kTileN];
-                float m_split = -INFINITY;                    // kSplitLd: the tile maximum, formed while S arrives
                 PULSAR_TMEM_LD32_AT(tS + 0, r, 0);
                 PULSAR_TMEM_LD32_AT(tS + 32, r, 32);
-                if (kSplitLd) {
-                    tmem_wait_ld();
-                    PULSAR_TMEM_LD32_AT(tS + 64, r, 64);
-                    PULSAR_TMEM_LD32_AT(tS + 96, r, 96);
-                    if (masked) {
-#pragma unroll
-                        for (int c = 0; c < 64; ++c)
-                            if (c >= n_vis) r[c] = 0xff800000u;          // -inf
-                    }
-                    m_split = row_max64<0>(r);
-                    tmem_wait_ld();
-                    if (masked) {
-#pragma unroll
-                        for (int c = 64; c < kTileN; ++c)
-                            if (c >= n_vis) r[c] = 0xff800000u;
-                    }
-                    m_split = fmaxf(m_split, row_max64<64>(r));
-                } else {
-                    PULSAR_TMEM_LD32_AT(tS + 64, r, 64);
-                    PULSAR_TMEM_LD32_AT(tS + 96, r, 96);
-                    tmem_wait_ld();
-                }
+                PULSAR_TMEM_LD32_AT(tS + 64, r, 64);
+                PULSAR_TMEM_LD32_AT(tS + 96, r, 96);
+                tmem_wait_ld();
 
                 // Fast path (unmasked tile, not the first): the first half of the probabilities is
                 // formed with the maximum already in use while the tile's own maximum is computed
@@ -1087,12 +1008,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                     }
                 }
                 if (exact) {
-                    if (masked && !kSplitLd) {
+                    if (masked) {
 #pragma unroll
                         for (int c = 0; c < kTileN; ++c)
                             if (c >= n_vis) r[c] = 0xff800000u;          // -inf
                     }
-                    const float m_tile = (kSplitLd ? m_split : row_max128(r)) * a.scale_log2;
+                    const float m_tile = row_max128(r) * a.scale_log2;
                     const bool need = m_tile > m_used + kRescaleThreshold;   // always true on the first tile
                     if (__any_sync(0xffffffffu, need)) {
                         if (kSingle && t > 0) {
@@ -1124,10 +1045,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                     // P goes to the MMA issuer in two halves of 64 keys, so that the first half
                     // of the PV product runs while the second half of the row is exponentiated.
                     // (The rescale above has stored its O columns before the first hand-over.)
-                    if (kMufuTurns && !kQuad) {
-                        ok = mufu_turn_take(mufu_turn, lane, abort_flag, a.status);
-                        if (!ok) break;
-                    }
                     if (masked) l_run += exp_row128<0, 0, 64>(r, a.scale_log2, neg_m, tS);
                     else l_run += exp_row128<kSpeculate ? 0 : kPolyPairsFor<D>, 0, 64>(r, a.scale_log2, neg_m, tS);
                     tmem_wait_st();
@@ -1136,7 +1053,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                     if (lane == 0) mbar_arrive(bar_p);
                     if (masked) l_run += exp_row128<0, 64, 128>(r, a.scale_log2, neg_m, tS);
                     else l_run += exp_row128<kSpeculate ? 0 : kPolyPairsFor<D>, 64, 128>(r, a.scale_log2, neg_m, tS);
-                    if (kMufuTurns && !kQuad) mufu_turn_give(mufu_turn, lane);
                 }
 
                 tmem_wait_st();
