@@ -239,14 +239,13 @@ constexpr int kMmaWarp = 8;
 constexpr int kLoadWarp = 9;
 constexpr float kRescaleThreshold = 8.0f;      // in log2 units
 // Tuning knobs (overridable at build time with -D).  Measured on a 1000 W B200 running the 128K
-// step back to back (power-capped, SM clock ~1.56 GHz): both off 1060 TFLOP/s, speculation only
-// 1048, polynomial only 1032, both on 1020 -- under the power cap the variant that executes the
-// fewest instructions wins, although both options shorten the per-tile latency in short runs.
+// step back to back (power-capped, SM clock ~1.56 GHz): without the polynomial exponential 1060 TFLOP/s,
+// with one pair in four 1032 -- under the power cap the variant that executes the fewest instructions
+// wins, although the option shortens the per-tile latency in short runs.  (Forming the first half of P
+// with the maximum in use while the tile maximum is computed alongside was a second such option: 1048,
+// and 1020 with both; taken out of the source.)
 #ifndef PULSAR_POLY_PAIRS
 #define PULSAR_POLY_PAIRS 0
-#endif
-#ifndef PULSAR_SPECULATE
-#define PULSAR_SPECULATE 0
 #endif
 #ifndef PULSAR_EARLY_RELEASE
 #define PULSAR_EARLY_RELEASE 1
@@ -268,7 +267,6 @@ constexpr int kPolyPairs128 = PULSAR_POLY_PAIRS;  // of every four column pairs,
 #define PULSAR_POLY_PAIRS_D64 1
 #endif
 template <int D> constexpr int kPolyPairsFor = D == 64 ? PULSAR_POLY_PAIRS_D64 : kPolyPairs128;
-constexpr bool kSpeculate = PULSAR_SPECULATE;  // form P with the maximum in use while the tile maximum is computed
 // Registers per thread: the kernel is compiled for 168 (twelve warps).  setmaxnreg moves
 // registers inside the CTA's own pool of 12 * 168 per lane slot and acts on whole warpgroups:
 // warpgroup 2 (MMA issuer, TMA loader and two spare warps) hands back all but kRegsIssuer,
@@ -988,72 +986,51 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 PULSAR_TMEM_LD32_AT(tS + 96, r, 96);
                 tmem_wait_ld();
 
-                // Fast path (unmasked tile, not the first): the first half of the probabilities is
-                // formed with the maximum already in use while the tile's own maximum is computed
-                // alongside (independent instruction streams); only if that maximum exceeds the
-                // one in use by more than the threshold (rare) is the tile redone on the exact
-                // path below.  Either way P is handed over in two halves of 64 keys.
-                bool exact = masked || t == 0 || !kSpeculate;
-                if (!exact) {
-                    const float l_lo = exp_row128<kPolyPairsFor<D>, 0, 64>(r, a.scale_log2, -m_used, tS);
-                    const float m_tile = row_max128(r) * a.scale_log2;
-                    if (__any_sync(0xffffffffu, m_tile > m_used + kRescaleThreshold)) {
-                        exact = true;
-                    } else {
-                        tmem_wait_st();
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(bar_p);
-                        l_run += l_lo + exp_row128<kPolyPairsFor<D>, 64, 128>(r, a.scale_log2, -m_used, tS);
-                    }
+                if (masked) {
+#pragma unroll
+                    for (int c = 0; c < kTileN; ++c)
+                        if (c >= n_vis) r[c] = 0xff800000u;          // -inf
                 }
-                if (exact) {
-                    if (masked) {
-#pragma unroll
-                        for (int c = 0; c < kTileN; ++c)
-                            if (c >= n_vis) r[c] = 0xff800000u;          // -inf
+                const float m_tile = row_max128(r) * a.scale_log2;
+                const bool need = m_tile > m_used + kRescaleThreshold;   // always true on the first tile
+                if (__any_sync(0xffffffffu, need)) {
+                    if (kSingle && t > 0) {
+                        // O may be rescaled once the PV product of the previous key tile is complete.
+                        // This is key tile g_tile - 1 of the CTA; completions 0 .. g_tile - 3 are certain
+                        // (this tile's S was issued after them), so the barrier is in phase g_tile - 2
+                        // or g_tile - 1 and the parity of g_tile - 2 tells the two apart.
+                        ok = __all_sync(0xffffffffu, mbar_wait(bar_pv, g_tile & 1u, abort_flag, a.status));
+                        if (!ok) break;
+                        tc_fence_after();
                     }
-                    const float m_tile = row_max128(r) * a.scale_log2;
-                    const bool need = m_tile > m_used + kRescaleThreshold;   // always true on the first tile
-                    if (__any_sync(0xffffffffu, need)) {
-                        if (kSingle && t > 0) {
-                            // O may be rescaled once the PV product of the previous key tile is complete.
-                            // This is key tile g_tile - 1 of the CTA; completions 0 .. g_tile - 3 are certain
-                            // (this tile's S was issued after them), so the barrier is in phase g_tile - 2
-                            // or g_tile - 1 and the parity of g_tile - 2 tells the two apart.
-                            ok = __all_sync(0xffffffffu, mbar_wait(bar_pv, g_tile & 1u, abort_flag, a.status));
-                            if (!ok) break;
-                            tc_fence_after();
-                        }
-                        const float m_new = need ? m_tile : m_used;
-                        const float alpha = (m_new == -INFINITY) ? 1.f : ex2(m_used - m_new);
-                        l_run *= alpha;
-                        m_used = m_new;
-                        if (t > 0) {
+                    const float m_new = need ? m_tile : m_used;
+                    const float alpha = (m_new == -INFINITY) ? 1.f : ex2(m_used - m_new);
+                    l_run *= alpha;
+                    m_used = m_new;
+                    if (t > 0) {
 #pragma unroll
-                            for (int c0 = 0; c0 < D; c0 += 32) {
-                                uint32_t o[32];
-                                tmem_ld32(tO + c0, o);
-                                tmem_wait_ld();
+                        for (int c0 = 0; c0 < D; c0 += 32) {
+                            uint32_t o[32];
+                            tmem_ld32(tO + c0, o);
+                            tmem_wait_ld();
 #pragma unroll
-                                for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-                                tmem_st32(tO + c0, o);
-                            }
+                            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                            tmem_st32(tO + c0, o);
                         }
                     }
-                    const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
-                    // P goes to the MMA issuer in two halves of 64 keys, so that the first half
-                    // of the PV product runs while the second half of the row is exponentiated.
-                    // (The rescale above has stored its O columns before the first hand-over.)
-                    if (masked) l_run += exp_row128<0, 0, 64>(r, a.scale_log2, neg_m, tS);
-                    else l_run += exp_row128<kSpeculate ? 0 : kPolyPairsFor<D>, 0, 64>(r, a.scale_log2, neg_m, tS);
-                    tmem_wait_st();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_p);
-                    if (masked) l_run += exp_row128<0, 64, 128>(r, a.scale_log2, neg_m, tS);
-                    else l_run += exp_row128<kSpeculate ? 0 : kPolyPairsFor<D>, 64, 128>(r, a.scale_log2, neg_m, tS);
                 }
+                const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
+                // P goes to the MMA issuer in two halves of 64 keys, so that the first half
+                // of the PV product runs while the second half of the row is exponentiated.
+                // (The rescale above has stored its O columns before the first hand-over.)
+                if (masked) l_run += exp_row128<0, 0, 64>(r, a.scale_log2, neg_m, tS);
+                else l_run += exp_row128<kPolyPairsFor<D>, 0, 64>(r, a.scale_log2, neg_m, tS);
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_p);
+                if (masked) l_run += exp_row128<0, 64, 128>(r, a.scale_log2, neg_m, tS);
+                else l_run += exp_row128<kPolyPairsFor<D>, 64, 128>(r, a.scale_log2, neg_m, tS);
 
                 tmem_wait_st();
                 tc_fence_before();
